@@ -1,0 +1,153 @@
+/*
+ * treewy.h -- C ABI of libtreewy: speculative draft-tree verification and commit for
+ * Gated DeltaNet (GDN) layers through the tree-structured WY transform of the gated
+ * delta rule, as hand-written CUDA kernels for NVIDIA B200 (sm_100a).
+ *
+ * The method (TreeWY paper, Section 3).  A GDN head keeps a state S in R^{d_v x d_k} that
+ * evolves by the gated delta rule (Eq. 1)
+ *       S_t = alpha_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T ,   o_t = S_t q_t .
+ * Writing it as S_t = alpha_t S_{t-1} + u_t k_t^T with the pseudo-value
+ *       u_t = beta_t (v_t - alpha_t S_{t-1} k_t)                    ("Key rewrite")
+ * and chaining it along every root-to-node path of a draft tree of N nodes that hang off
+ * the committed state S0 gives ONE unit-lower-triangular system for all pseudo-values
+ * (Eq. 2):
+ *       (I + A) U = R ,   A[t,i] = beta_t (g_t/g_i) (k_t . k_i)  for i a proper ancestor of t,
+ *                         R[t]   = beta_t (v_t - g_t S0 k_t) ,
+ * with g_t the cumulative decay from S0 to t (the product of alpha over the root path,
+ * node t included).  Every node's output reads out from the same solve,
+ *       o_t = g_t S0 q_t + sum_{i ancestor-or-self of t} (g_t/g_i) (k_i . q_t) u_i ,
+ * and once node a is accepted the next committed state is rebuilt (Eq. 3) as
+ *       S_a = g_a S0 + sum_{i ancestor-or-self of a} (g_a/g_i) u_i k_i^T ,
+ * so no per-node state snapshot is ever stored.
+ *
+ * Conventions for every call
+ *   - d_k = d_v = 128 (both Qwen3.5 hybrids of the paper, Section 2).
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte aligned, and
+ *     must stay valid until the stream has passed the call.  The library allocates
+ *     nothing, frees nothing, keeps no global state and never synchronises the host:
+ *     each call enqueues its kernel(s) on `cuda_stream` (a cudaStream_t passed as
+ *     void*, NULL = the default stream) and returns.
+ *   - Trees are packed: sequence b owns nodes node_offsets[b] .. node_offsets[b+1]-1
+ *     (N_b = 1..64 of them), `parent` holds LOCAL indices, parent = -1 means the node
+ *     applies directly to S0, and parent[i] < i (any topological order, DFS pre-order
+ *     being one; Section 3, "Verifying a draft").  Several parent = -1 nodes are legal.
+ *   - Value head h reads q/k head h / (H_v / H_qk) (adjacent value heads share one).
+ *   - State layout: S0[b][h][r][c], r the d_v index, c the d_k index, c contiguous.
+ *   - Host-checkable misuse returns an error code and launches nothing.
+ *     Data-dependent errors never trap: the sequence is skipped (its rows of O / U, its
+ *     tree outputs and its state are left untouched) and, when `seq_status` is not NULL,
+ *     the reason is OR-ed into seq_status[b] (the caller zeroes the array).
+ */
+#ifndef TREEWY_H
+#define TREEWY_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TREEWY_D 128         /* d_k = d_v */
+#define TREEWY_MAX_NODES 64  /* nodes per sequence (one 64-bit ancestor mask per node) */
+
+typedef enum {
+    TREEWY_OK = 0,
+    TREEWY_ERR_INVALID_ARG = 1, /* NULL or misaligned pointer, negative size, H_v % H_qk != 0 */
+    TREEWY_ERR_UNSUPPORTED = 2, /* unknown dtype, max_nodes > 64, dtype combination not built */
+    TREEWY_ERR_CUDA = 3         /* launch failed; cudaGetLastError() still holds the reason */
+} treewy_status_t;
+
+typedef enum { TREEWY_F32 = 0, TREEWY_BF16 = 1 } treewy_dtype_t;
+
+/* per-sequence status bits, OR-ed into seq_status[b] */
+enum {
+    TREEWY_SEQ_BAD_PARENT = 1,     /* some parent[i] >= i or < -1 */
+    TREEWY_SEQ_TOO_MANY_NODES = 2, /* N_b outside 1..max_nodes */
+    TREEWY_SEQ_BAD_ACCEPTED = 4,   /* accepted[b] outside -1..N_b-1 */
+    TREEWY_SEQ_TIMEOUT = 8         /* a bounded wait inside a kernel gave up */
+};
+
+/*
+ * A packed batch of draft trees.  The first block is filled by the caller; the second
+ * is written by treewy_tree_prepare and read by treewy_verify / treewy_commit.
+ */
+typedef struct {
+    int32_t B;                   /* sequences */
+    int32_t T;                   /* packed nodes, = node_offsets[B] */
+    int32_t H_v;                 /* value heads */
+    int32_t max_nodes;           /* host-known upper bound on N_b, 1..64; 0 means 64.  Only
+                                    sizes launches; a longer sequence is flagged, not run */
+    const int32_t *node_offsets; /* [B+1] device, node_offsets[0] = 0 */
+    const int32_t *parent;       /* [T]   device, local parent index or -1 */
+    int32_t *depth;              /* [T]   device, out: 0 for parent = -1, else depth[parent]+1 */
+    uint64_t *anc_mask;          /* [T]   device, out: bit j set <=> local node j is an
+                                    ancestor of the node or the node itself */
+    float *cum_log_gate;         /* [T,H_v] device, out: L[i,h] = sum over the root path of i,
+                                    i included, of log(alpha[.,h])  (log of g_i in Eq. 2) */
+} treewy_tree_t;
+
+/*
+ * Tree indexing (Section 3, "Verifying a draft"; g_t of Eq. 2).
+ * Reads tree->node_offsets, tree->parent and alpha [T,H_v] (fp32, linear gates in (0,1]);
+ * writes tree->depth, tree->anc_mask (bit-exact, one correct value each) and
+ * tree->cum_log_gate (fp32 sums of logf).  One small kernel on `cuda_stream`.
+ * Malformed sequences get TREEWY_SEQ_BAD_PARENT / TREEWY_SEQ_TOO_MANY_NODES.
+ * Topology is per decoding step, the log-gates per layer: call it once per layer, or reuse
+ * depth / anc_mask across layers and let it rewrite only what changed.
+ */
+treewy_status_t treewy_tree_prepare(const treewy_tree_t *tree, const float *alpha,
+                                    int32_t *seq_status, void *cuda_stream);
+
+/*
+ * Verify (Section 3, Eq. 2 and the read-out "from that same solve").
+ *   S0   [B,H_v,128,128]  io_dtype, read only
+ *   q,k  [T,H_qk,128]     io_dtype;  v [T,H_v,128] io_dtype;  beta [T,H_v] fp32
+ *   tree                  prepared by treewy_tree_prepare with this layer's alpha
+ *   O    [T,H_v,128]      o_dtype, out: o_t for every node (post-update state times q_t,
+ *                         no 1/sqrt(d) scale and no normalisation are applied)
+ *   U    [T,H_v,128]      fp32, out: the pseudo-values; keep them until commit
+ * io_dtype = BF16 takes the tensor-core kernel; io_dtype = F32 takes the fp32 SIMT kernel.
+ * o_dtype may be F32 or BF16 (round-to-nearest-even of the fp32 result).
+ * Sequences flagged by prepare-time checks (repeated here) are skipped.
+ */
+treewy_status_t treewy_verify(const void *S0, const void *q, const void *k, const void *v,
+                              const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                              treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,
+                              int32_t *seq_status, void *cuda_stream);
+
+/*
+ * Same contract as treewy_verify, always through the portable fp32 SIMT kernel (one CTA
+ * per (sequence, value head), no tensor cores).  It is the path F32 inputs take and a
+ * cross-check for the tensor-core kernel on BF16 inputs.
+ */
+treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void *k, const void *v,
+                                      const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                                      treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                      float *U, int32_t *seq_status, void *cuda_stream);
+
+/*
+ * Commit (Section 3, Eq. 3, "Reconstruct on commit").
+ * For every sequence b with a = accepted[b] >= 0 and every value head h, in place:
+ *   S0[b,h] <- g_a S0[b,h] + sum_{i ancestor-or-self of a} (g_a/g_i) u_i k_i^T
+ * rounded once to io_dtype.  accepted[b] = -1 leaves the state as it is.
+ *   S0        [B,H_v,128,128] io_dtype, in/out
+ *   U         [T,H_v,128] fp32 from treewy_verify;  k [T,H_qk,128] io_dtype (same as verify)
+ *   accepted  [B] int32, local node index or -1
+ *   S_out_f32 optional [B,H_v,128,128] fp32: when not NULL the unrounded new state is ALSO
+ *             written there (for accepted = -1 the old state, widened); NULL to skip
+ * An accepted index outside -1..N_b-1 sets TREEWY_SEQ_BAD_ACCEPTED and skips the sequence.
+ */
+treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
+                              int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
+                              float *S_out_f32, int32_t *seq_status, void *cuda_stream);
+
+/* A short constant string for a status code. */
+const char *treewy_status_string(treewy_status_t status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int treewy_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREEWY_H */

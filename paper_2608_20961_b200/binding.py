@@ -1,0 +1,220 @@
+"""Thin ctypes binding of libtreewy's C ABI (``include/treewy.h``).
+
+Argument marshalling only: torch tensors supply device memory and the stream, every
+step of verify / commit runs inside the library's CUDA kernels.  There is no CPU or
+PyTorch fallback -- if ``libtreewy.so`` cannot be loaded the import of a function fails
+loudly.  Function names and argument order follow the C header.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtreewy.so")
+
+TREEWY_OK, TREEWY_ERR_INVALID_ARG, TREEWY_ERR_UNSUPPORTED, TREEWY_ERR_CUDA = 0, 1, 2, 3
+TREEWY_F32, TREEWY_BF16 = 0, 1
+SEQ_BAD_PARENT, SEQ_TOO_MANY_NODES, SEQ_BAD_ACCEPTED, SEQ_TIMEOUT = 1, 2, 4, 8
+D = 128
+MAX_NODES = 64
+
+_DTYPES = {torch.float32: TREEWY_F32, torch.bfloat16: TREEWY_BF16}
+
+
+class TreeStruct(ctypes.Structure):
+    """Mirror of ``treewy_tree_t``."""
+    _fields_ = [
+        ("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H_v", ctypes.c_int32),
+        ("max_nodes", ctypes.c_int32),
+        ("node_offsets", ctypes.c_void_p), ("parent", ctypes.c_void_p),
+        ("depth", ctypes.c_void_p), ("anc_mask", ctypes.c_void_p),
+        ("cum_log_gate", ctypes.c_void_p),
+    ]
+
+
+class TreewyError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__(f"{fn} returned {code} ({status_string(code)})")
+
+
+_lib = None
+
+
+def load_library(path: str | None = None):
+    """Load ``libtreewy.so`` (built in-tree by ``build.py``); raises if it is absent."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} not found: build it with `python -m paper_2608_20961_b200.build` "
+            "(nvcc, sm_100a). libtreewy has no CPU fallback.")
+    lib = ctypes.CDLL(path)
+    vp, i32 = ctypes.c_void_p, ctypes.c_int32
+    lib.treewy_tree_prepare.argtypes = [ctypes.POINTER(TreeStruct), vp, vp, vp]
+    lib.treewy_tree_prepare.restype = ctypes.c_int
+    verify_args = [vp, vp, vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int,
+                   vp, vp, vp, vp]
+    lib.treewy_verify.argtypes = verify_args
+    lib.treewy_verify.restype = ctypes.c_int
+    lib.treewy_verify_generic.argtypes = verify_args
+    lib.treewy_verify_generic.restype = ctypes.c_int
+    lib.treewy_commit.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, vp, ctypes.c_int,
+                                  vp, vp, vp]
+    lib.treewy_commit.restype = ctypes.c_int
+    lib.treewy_status_string.argtypes = [ctypes.c_int]
+    lib.treewy_status_string.restype = ctypes.c_char_p
+    lib.treewy_version.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().treewy_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(load_library().treewy_version())
+
+
+def _p(t: torch.Tensor | None):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(fn: str, code: int):
+    if code != TREEWY_OK:
+        raise TreewyError(fn, code)
+
+
+@dataclass
+class Tree:
+    """Device-side ``treewy_tree_t``: topology in, depth / mask / log-gates out."""
+    B: int
+    T: int
+    H_v: int
+    max_nodes: int
+    node_offsets: torch.Tensor   # int32 [B+1]
+    parent: torch.Tensor         # int32 [T]
+    depth: torch.Tensor          # int32 [T]
+    anc_mask: torch.Tensor       # int64 storage of the uint64 masks [T]
+    cum_log_gate: torch.Tensor   # fp32 [T, H_v]
+
+    @classmethod
+    def empty(cls, node_offsets: torch.Tensor, parent: torch.Tensor, H_v: int,
+              max_nodes: int = 0) -> "Tree":
+        dev = parent.device
+        T = int(parent.numel())
+        return cls(B=int(node_offsets.numel()) - 1, T=T, H_v=H_v, max_nodes=max_nodes,
+                   node_offsets=node_offsets, parent=parent,
+                   depth=torch.full((max(T, 1),), -1, dtype=torch.int32, device=dev),
+                   anc_mask=torch.zeros((max(T, 1),), dtype=torch.int64, device=dev),
+                   cum_log_gate=torch.zeros((max(T, 1), H_v), dtype=torch.float32, device=dev))
+
+    def struct(self) -> TreeStruct:
+        return TreeStruct(self.B, self.T, self.H_v, self.max_nodes,
+                          self.node_offsets.data_ptr(), self.parent.data_ptr(),
+                          self.depth.data_ptr(), self.anc_mask.data_ptr(),
+                          self.cum_log_gate.data_ptr())
+
+
+def treewy_tree_prepare(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tensor | None = None,
+                        stream=None) -> None:
+    lib = load_library()
+    ts = tree.struct()
+    _check("treewy_tree_prepare",
+           lib.treewy_tree_prepare(ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream)))
+
+
+def treewy_verify(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,
+                  seq_status: torch.Tensor | None = None, stream=None, generic: bool = False) -> None:
+    """O and U are written in place; io dtype comes from S0, the output dtype from O."""
+    lib = load_library()
+    ts = tree.struct()
+    fn = lib.treewy_verify_generic if generic else lib.treewy_verify
+    assert q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
+    _check("treewy_verify",
+           fn(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+              _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream)))
+
+
+def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
+                  seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """S0 is updated in place; S_out_f32, when given, also receives the unrounded state."""
+    lib = load_library()
+    ts = tree.struct()
+    _check("treewy_commit",
+           lib.treewy_commit(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+
+
+# --------------------------------------------------------------------------- user-level step
+
+class VerifyCommitLayer:
+    """One GDN layer's speculative state on a device: the committed state lives in HBM across
+    steps; each step uploads the draft window's inputs, verifies, returns the outputs to the
+    host, and commits the accepted node.  This is the call a serving loop makes."""
+
+    def __init__(self, S0: torch.Tensor, H_qk: int, max_T: int, max_nodes: int = 0,
+                 o_dtype: torch.dtype | None = None):
+        dev = S0.device
+        self.S0 = S0
+        self.B, self.H_v = int(S0.shape[0]), int(S0.shape[1])
+        self.H_qk, self.max_nodes = H_qk, max_nodes
+        io = S0.dtype
+        o_dtype = o_dtype or io
+        z = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        self.q, self.k = z((max_T, H_qk, D), io), z((max_T, H_qk, D), io)
+        self.v = z((max_T, self.H_v, D), io)
+        self.alpha, self.beta = z((max_T, self.H_v), torch.float32), z((max_T, self.H_v), torch.float32)
+        self.node_offsets = z((self.B + 1,), torch.int32)
+        self.parent = z((max_T,), torch.int32)
+        self.accepted = z((self.B,), torch.int32)
+        self.O = z((max_T, self.H_v, D), o_dtype)
+        self.U = z((max_T, self.H_v, D), torch.float32)
+        self.status = torch.zeros((self.B,), dtype=torch.int32, device=dev)
+        self.depth = z((max_T,), torch.int32)
+        self.anc_mask = z((max_T,), torch.int64)
+        self.cum_log_gate = z((max_T, self.H_v), torch.float32)
+
+    def tree(self, T: int) -> Tree:
+        return Tree(self.B, T, self.H_v, self.max_nodes, self.node_offsets, self.parent,
+                    self.depth, self.anc_mask, self.cum_log_gate)
+
+    def upload(self, host: dict) -> int:
+        """Host (pinned) tensors -> device buffers on the current stream; returns T."""
+        T = int(host["parent"].numel())
+        for name in ("q", "k", "v", "alpha", "beta", "parent"):
+            getattr(self, name)[:T].copy_(host[name], non_blocking=True)
+        self.node_offsets.copy_(host["node_offsets"], non_blocking=True)
+        return T
+
+    def verify(self, T: int) -> None:
+        tree = self.tree(T)
+        treewy_tree_prepare(tree, self.alpha, self.status)
+        treewy_verify(self.S0, self.q, self.k, self.v, self.beta, tree, self.H_qk, self.O, self.U,
+                      self.status)
+
+    def commit(self, T: int, accepted_host: torch.Tensor | None = None) -> None:
+        if accepted_host is not None:
+            self.accepted.copy_(accepted_host, non_blocking=True)
+        treewy_commit(self.S0, self.U, self.k, self.tree(T), self.H_qk, self.accepted, None,
+                      self.status)
+
+    def step(self, host: dict, O_host: torch.Tensor) -> None:
+        """upload -> prepare -> verify -> outputs to host -> commit, all on the current stream."""
+        T = self.upload(host)
+        self.verify(T)
+        O_host[:T].copy_(self.O[:T], non_blocking=True)
+        self.commit(T, host["accepted"])

@@ -1,0 +1,133 @@
+// C ABI of libtreewy: argument checks and kernel dispatch.  No allocation, no host
+// synchronisation, no state kept between calls.
+#include "treewy_kernels.cuh"
+
+using namespace treewy;
+
+namespace {
+
+inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+inline bool bad_ptr(const void *p) { return p == nullptr || misaligned(p); }
+inline bool bad_dtype(int d) { return d != TREEWY_F32 && d != TREEWY_BF16; }
+
+// Checks the caller-filled part of the tree; *max_nodes receives the launch bound.
+treewy_status_t check_tree(const treewy_tree_t *t, bool need_outputs, int *max_nodes)
+{
+    if (!t) return TREEWY_ERR_INVALID_ARG;
+    if (t->B < 0 || t->T < 0 || t->H_v < 1) return TREEWY_ERR_INVALID_ARG;
+    if (t->max_nodes < 0) return TREEWY_ERR_INVALID_ARG;
+    if (t->max_nodes > TREEWY_MAX_NODES) return TREEWY_ERR_UNSUPPORTED;
+    *max_nodes = t->max_nodes == 0 ? TREEWY_MAX_NODES : t->max_nodes;
+    if (t->B == 0) return TREEWY_OK;
+    if (bad_ptr(t->node_offsets)) return TREEWY_ERR_INVALID_ARG;
+    if (t->T > 0 && bad_ptr(t->parent)) return TREEWY_ERR_INVALID_ARG;
+    if (need_outputs && t->T > 0 &&
+        (bad_ptr(t->depth) || bad_ptr(t->anc_mask) || bad_ptr(t->cum_log_gate)))
+        return TREEWY_ERR_INVALID_ARG;
+    return TREEWY_OK;
+}
+
+treewy_status_t verify_common(bool force_generic, const void *S0, const void *q, const void *k,
+                              const void *v, const float *beta, const treewy_tree_t *tree,
+                              int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype,
+                              void *O, float *U, int32_t *seq_status, void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(io_dtype) || bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0 || tree->T == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(q) || bad_ptr(k) || bad_ptr(v) || bad_ptr(beta) || bad_ptr(O) ||
+        bad_ptr(U))
+        return TREEWY_ERR_INVALID_ARG;
+
+    VerifyArgs a;
+    a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.O = O, a.U = U, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    (void)force_generic;
+    e = launch_verify_generic(a, io_dtype, o_dtype, stream);
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+treewy_status_t treewy_tree_prepare(const treewy_tree_t *tree, const float *alpha,
+                                    int32_t *seq_status, void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0) return TREEWY_OK;
+    if (tree->T > 0 && bad_ptr(alpha)) return TREEWY_ERR_INVALID_ARG;
+    cudaError_t e =
+        launch_prepare(*tree, max_nodes, alpha, seq_status, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_verify(const void *S0, const void *q, const void *k, const void *v,
+                              const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                              treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,
+                              int32_t *seq_status, void *cuda_stream)
+{
+    return verify_common(false, S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status,
+                         cuda_stream);
+}
+
+treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void *k, const void *v,
+                                      const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                                      treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                      float *U, int32_t *seq_status, void *cuda_stream)
+{
+    return verify_common(true, S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status,
+                         cuda_stream);
+}
+
+treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
+                              int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
+                              float *S_out_f32, int32_t *seq_status, void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(io_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (S_out_f32 && misaligned(S_out_f32)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(accepted)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->T > 0 && (bad_ptr(U) || bad_ptr(k))) return TREEWY_ERR_INVALID_ARG;
+
+    CommitArgs a;
+    a.S0 = S0, a.U = U, a.k = k;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    cudaError_t e = launch_commit(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+const char *treewy_status_string(treewy_status_t status)
+{
+    switch (status) {
+    case TREEWY_OK: return "ok";
+    case TREEWY_ERR_INVALID_ARG: return "invalid argument";
+    case TREEWY_ERR_UNSUPPORTED: return "unsupported";
+    case TREEWY_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+int treewy_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,81 @@
+// Shared device helpers of libtreewy's kernels: storage-type conversion, per-sequence
+// validation, small warp utilities.  Nothing here is used by the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/treewy.h"
+
+namespace treewy {
+
+constexpr int D = TREEWY_D;
+constexpr int MAXN = TREEWY_MAX_NODES;
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x)
+{
+    return __float2bfloat16_rn(x);
+}
+
+// Two packed bf16 (low = first element) -> two floats.  bf16 -> fp32 is a 16-bit shift.
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&p);
+}
+
+// 128 consecutive elements (16-byte aligned) widened into registers with 128-bit loads.
+__device__ __forceinline__ void load_row128(const float *__restrict__ p, float (&s)[128])
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const float4 x = reinterpret_cast<const float4 *>(p)[i];
+        s[4 * i] = x.x, s[4 * i + 1] = x.y, s[4 * i + 2] = x.z, s[4 * i + 3] = x.w;
+    }
+}
+__device__ __forceinline__ void load_row128(const __nv_bfloat16 *__restrict__ p, float (&s)[128])
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const uint4 x = reinterpret_cast<const uint4 *>(p)[i];
+        s[8 * i] = bf16lo(x.x), s[8 * i + 1] = bf16hi(x.x);
+        s[8 * i + 2] = bf16lo(x.y), s[8 * i + 3] = bf16hi(x.y);
+        s[8 * i + 4] = bf16lo(x.z), s[8 * i + 5] = bf16hi(x.z);
+        s[8 * i + 6] = bf16lo(x.w), s[8 * i + 7] = bf16hi(x.w);
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Status bits of sequence [lo, lo+n): node count in 1..max_nodes, parent[i] in -1..i-1.
+// Called by every thread of a CTA with the same arguments; `scratch` is one shared int the
+// caller zeroed before a barrier.  Returns the same value in every thread.
+__device__ __forceinline__ int validate_sequence(const int32_t *__restrict__ parent, int lo, int n,
+                                                 int max_nodes, int *scratch)
+{
+    if (n < 1 || n > max_nodes) return TREEWY_SEQ_TOO_MANY_NODES;
+    int bad = 0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int p = parent[lo + i];
+        if (p < -1 || p >= i) bad = 1;
+    }
+    if (bad) atomicOr(scratch, TREEWY_SEQ_BAD_PARENT);
+    __syncthreads();
+    return *scratch;
+}
+
+}  // namespace treewy

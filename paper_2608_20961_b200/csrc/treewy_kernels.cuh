@@ -1,0 +1,42 @@
+// Argument blocks and launchers of libtreewy's kernels (internal to the library).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/treewy.h"
+
+namespace treewy {
+
+struct VerifyArgs {
+    const void *S0, *q, *k, *v;
+    const float *beta;
+    const int32_t *node_offsets, *parent;
+    const uint64_t *anc_mask;
+    const float *cum_log_gate;
+    void *O;
+    float *U;
+    int32_t *seq_status;
+    int B, H_v, H_qk, max_nodes;
+};
+
+struct CommitArgs {
+    void *S0;
+    const float *U;
+    const void *k;
+    const int32_t *node_offsets, *parent;
+    const uint64_t *anc_mask;
+    const float *cum_log_gate;
+    const int32_t *accepted;
+    float *S_out_f32;
+    int32_t *seq_status;
+    int B, H_v, H_qk, max_nodes;
+};
+
+cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha,
+                           int32_t *seq_status, cudaStream_t stream);
+cudaError_t launch_verify_generic(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od,
+                                  cudaStream_t stream);
+cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
+
+}  // namespace treewy

@@ -1,0 +1,153 @@
+"""GPU parity tests: libtreewy (through its C ABI) against the fp64 CPU oracle, element by
+element, on seeded inputs small enough for the oracle to finish in seconds yet spanning
+several CTAs, shared q/k heads and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_20961_b200 import workloads as wl
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+SMALL = {  # config id -> overrides that keep the structure but shrink the batch
+    0: {},
+    1: dict(B=6, H_v=8),
+    2: dict(B=5, H_v=8),
+    3: dict(B=3, H_v=4),
+    4: dict(B=21, H_v=4, prefix_tokens=32),
+    5: dict(B=3, H_v=4),
+}
+
+
+@pytest.mark.parametrize("generic", [True, False])
+@pytest.mark.parametrize("cid", sorted(SMALL))
+def test_configs_match_oracle(oracle, cid, generic):
+    w = wl.make_workload(cid, **SMALL[cid])
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    gpu = pu.run_gpu(w, torch.float32, generic=generic)
+    assert not gpu["status"].any()
+    errs = pu.assert_parity(w, gpu, tree_ref, ref)
+    print(f"config {cid} generic={generic}: worst (max-abs/rms, rel-fro) {errs}")
+    if w.io_dtype == torch.bfloat16:
+        gpu16 = pu.run_gpu(w, torch.bfloat16, generic=generic)
+        got, floor = pu.assert_bf16_outputs(w, gpu16, gpu, ref)
+        print(f"   bf16 O: {got} against rounding floor {floor}")
+        assert torch.equal(gpu16["S"], gpu["S"])
+
+
+@pytest.mark.parametrize("generic", [True, False])
+def test_fp32_inputs_bf16_heads_shared_by_four(oracle, generic):
+    w = wl.make_workload(2, B=3, H_v=8, H_qk=2)
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    gpu = pu.run_gpu(w, torch.float32, generic=generic)
+    pu.assert_parity(w, gpu, tree_ref, ref)
+    w32 = wl.make_workload(2, B=2, H_v=4, io_dtype=torch.float32)
+    tree_ref, ref = pu.run_oracle(oracle, w32)
+    gpu = pu.run_gpu(w32, torch.float32, generic=generic)
+    pu.assert_parity(w32, gpu, tree_ref, ref)
+
+
+def _custom(trees, H_v=2, H_qk=1, seed=1, dtype=torch.bfloat16, accepted=None):
+    """A workload with hand-made topologies and config-2 value distributions."""
+    base = wl.make_workload(2, B=1, H_v=H_v, H_qk=H_qk, seed=seed)
+    g = torch.Generator().manual_seed(seed)
+    off = [0]
+    for t in trees:
+        off.append(off[-1] + len(t))
+    T, B = off[-1], len(trees)
+    norm = lambda x: x / x.norm(dim=-1, keepdim=True)
+    return wl.Workload(
+        name="custom", config_id=-1, B=B, H_v=H_v, H_qk=H_qk, io_dtype=dtype,
+        node_offsets=torch.tensor(off, dtype=torch.int32),
+        parent=torch.tensor([p for t in trees for p in t], dtype=torch.int32),
+        q=norm(torch.randn(T, H_qk, 128, generator=g)).to(dtype),
+        k=norm(torch.randn(T, H_qk, 128, generator=g)).to(dtype),
+        v=torch.randn(T, H_v, 128, generator=g).to(dtype),
+        alpha=0.9 + 0.099 * torch.rand(T, H_v, generator=g),
+        beta=0.1 + 0.8 * torch.rand(T, H_v, generator=g),
+        S0=(0.05 * torch.randn(B, H_v, 128, 128, generator=g)).to(dtype),
+        accepted=torch.tensor(accepted if accepted is not None else [len(t) - 1 for t in trees],
+                              dtype=torch.int32), seed=seed)
+
+
+@pytest.mark.parametrize("generic", [True, False])
+def test_degenerate_topologies(oracle, generic):
+    chain64 = [i - 1 for i in range(64)]
+    star64 = [-1] + [0] * 63
+    forest = [-1, -1, 0, 1, -1, 4, 5]
+    single = [-1]
+    trees = [chain64, star64, forest, single, [-1, 0], chain64[:33]]
+    w = _custom(trees, H_v=4, H_qk=2, accepted=[63, 17, 6, 0, -1, 32])
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    gpu = pu.run_gpu(w, torch.float32, generic=generic)
+    assert not gpu["status"].any()
+    pu.assert_parity(w, gpu, tree_ref, ref)
+    # accepted = -1: the stored state is bit-identical to the input state
+    assert torch.equal(gpu["S"][4], w.S0[4])
+
+
+@pytest.mark.parametrize("generic", [True, False])
+def test_malformed_sequences_are_skipped_not_trapped(oracle, generic):
+    good = [-1, 0, 0, 2]
+    bad_parent = [-1, 2, 0]               # parent[1] = 2 >= 1
+    trees = [good, bad_parent, good, [-1, 0]]
+    w = _custom(trees, H_v=2, H_qk=2, accepted=[3, 1, 9, 1])   # sequence 2: accepted out of range
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    gpu = pu.run_gpu(w, torch.float32, generic=generic)
+    from paper_2608_20961_b200 import binding as tw
+    assert list(gpu["status"]) == [0, tw.SEQ_BAD_PARENT, tw.SEQ_BAD_ACCEPTED, 0]
+    assert list(ref.seq_status) == list(gpu["status"])
+    pu.assert_parity(w, gpu, tree_ref, ref, skip_seqs=(1, 2))
+    off = w.node_offsets.tolist()
+    # skipped sequence: outputs untouched (canary), state untouched
+    assert torch.all(gpu["O"][off[1]:off[2]] == gpu["canary"])
+    assert torch.all(gpu["U"][off[1]:off[2]] == gpu["canary"])
+    assert torch.equal(gpu["S"][1], w.S0[1]) and torch.equal(gpu["S"][2], w.S0[2])
+    # bad accepted only stops the commit: verify outputs of sequence 2 are right
+    sl = slice(off[2], off[3])
+    np.testing.assert_allclose(gpu["O"][sl].double().numpy(), ref_O_of(oracle, w, 2), atol=1e-4)
+
+
+def ref_O_of(oracle, w, b):
+    one = w.select_sequences([b])
+    one.accepted[:] = -1
+    return pu.run_oracle(oracle, one)[1].O
+
+
+def test_max_nodes_hint_flags_longer_sequences():
+    from paper_2608_20961_b200 import binding as tw
+    w = _custom([[-1, 0, 1], [i - 1 for i in range(20)]], H_v=2, H_qk=2)
+    gpu = pu.run_gpu(w, torch.float32, max_nodes=16)
+    assert list(gpu["status"]) == [0, tw.SEQ_TOO_MANY_NODES]
+
+
+def test_empty_batch_is_a_no_op():
+    from paper_2608_20961_b200 import binding as tw
+    dev = torch.device("cuda:0")
+    off = torch.zeros(1, dtype=torch.int32, device=dev)
+    par = torch.zeros(4, dtype=torch.int32, device=dev)[:0]
+    tree = tw.Tree.empty(off, par, 2)
+    z = torch.zeros(4, 2, 128, device=dev)
+    tw.treewy_tree_prepare(tree, z[:, :, 0], None)
+    tw.treewy_verify(z, z, z, z, z[:, :, 0], tree, 2, z.clone(), z.clone(), None)
+    tw.treewy_commit(z, z, z, tree, 2, off, None, None)
+    torch.cuda.synchronize()
+
+
+def test_metamorphic_commit_then_verify_on_gpu(oracle):
+    # commit node a on the GPU, then verify a's subtree from the new state: outputs of those
+    # nodes must reproduce the first verify (fp32 state hand-over keeps it tight)
+    tree = [-1, 0, 1, 1, 3, 0, 2]
+    w = _custom([tree], H_v=2, H_qk=1, dtype=torch.float32, accepted=[1])
+    first = pu.run_gpu(w, torch.float32)
+    sub = [2, 3, 4, 6]
+    w2 = _custom([[-1, -1, 1, 0]], H_v=2, H_qk=1, dtype=torch.float32, accepted=[-1])
+    idx = torch.tensor(sub)
+    w2.q, w2.k, w2.v = w.q[idx], w.k[idx], w.v[idx]
+    w2.alpha, w2.beta = w.alpha[idx], w.beta[idx]
+    w2.S0 = first["S"]
+    second = pu.run_gpu(w2, torch.float32)
+    torch.testing.assert_close(second["O"], first["O"][idx], rtol=0, atol=2e-5)
+    torch.testing.assert_close(second["U"], first["U"][idx], rtol=0, atol=2e-5)
