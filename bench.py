@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of GDN draft-tree verify + commit (libtreewy) on B200.
+
+A step is one pass of the whole hot path -- treewy_tree_prepare, treewy_verify,
+treewy_commit -- over one batch of the 35B-shaped workload (256 sequences x 32 value heads,
+16 shared q/k heads, random trees of 32 nodes).  Metric: node*heads/s per layer.
+
+Layer rotation: the bench keeps two independent layer buffer sets; step s prepares and
+verifies set s%2 and commits the other set (verified one step earlier).  Every step still
+does one prepare + one verify + one commit over a full batch, but a state is committed only
+after ~1 GB of other traffic has passed through the 126 MB L2 -- as in serving, where commit
+follows the rest of the forward pass -- so no kernel is timed on an L2-resident state.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config ID] [--impl reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange
+step, so there is no data-path collective (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_20961_b200 import footprint, replicas  # noqa: E402
+from paper_2608_20961_b200 import workloads as wl  # noqa: E402
+
+METRIC = "gdn_tree_verify_commit_node_heads_per_s_per_layer"
+UNIT = "node*heads/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the verify kernel on the bench workload, from one ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/.  None until captured.
+VERIFY_DRAM_TRAFFIC_BYTES = {2: None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 0.0)), "measured"
+    return FALLBACK_HBM_GBS, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                bits = get_reasons(self.h)
+                for name, bit in names.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+class LayerSet:
+    """Device buffers of one GDN layer for one batch of draft trees."""
+
+    def __init__(self, w: wl.Workload, dev: torch.device):
+        from paper_2608_20961_b200 import binding as tw
+        self.tw, self.w = tw, w
+        d = lambda t: t.to(dev)
+        self.off, self.par = d(w.node_offsets), d(w.parent)
+        self.alpha, self.beta = d(w.alpha), d(w.beta)
+        self.q, self.k, self.v, self.S0 = d(w.q), d(w.k), d(w.v), d(w.S0).clone()
+        self.acc = d(w.accepted)
+        self.O = torch.empty((w.T, w.H_v, 128), dtype=w.io_dtype, device=dev)
+        self.U = torch.empty((w.T, w.H_v, 128), dtype=torch.float32, device=dev)
+        self.status = torch.zeros(w.B, dtype=torch.int32, device=dev)
+        self.tree = tw.Tree.empty(self.off, self.par, w.H_v, w.max_nodes)
+
+    def prepare(self):
+        self.tw.treewy_tree_prepare(self.tree, self.alpha, self.status)
+
+    def verify(self):
+        self.tw.treewy_verify(self.S0, self.q, self.k, self.v, self.beta, self.tree, self.w.H_qk,
+                              self.O, self.U, self.status)
+
+    def commit(self):
+        self.tw.treewy_commit(self.S0, self.U, self.k, self.tree, self.w.H_qk, self.acc, None,
+                              self.status)
+
+
+def pass_bytes(w: wl.Workload) -> footprint.PassBytes:
+    off = w.node_offsets.tolist()
+    par = w.parent.tolist()
+    nodes, plen = [], []
+    for b in range(w.B):
+        t = par[off[b]:off[b + 1]]
+        depth = wl.tree_depths(t)
+        a = int(w.accepted[b])
+        nodes.append(len(t))
+        plen.append(depth[a] + 1 if a >= 0 else 0)
+    return footprint.algorithmic_bytes(nodes, plen, w.H_v, w.H_qk, io_elem=w.S0.element_size(),
+                                       o_elem=w.S0.element_size())
+
+
+def oracle_inputs(w: wl.Workload):
+    f = lambda t: t.to(torch.float64).numpy()
+    return (w.node_offsets.numpy(), w.parent.numpy(), f(w.S0), f(w.q), f(w.k), f(w.v), f(w.alpha),
+            f(w.beta), w.accepted.numpy())
+
+
+def time_oracle(w: wl.Workload, n_seq: int, min_seconds: float = 10.0):
+    """The CPU oracle, as it stands, on the first n_seq sequences, repeated until at least
+    min_seconds have passed; returns (units/s, seconds, passes, sub-batch, threads)."""
+    from oracle import treewy_oracle
+    treewy_oracle.build()
+    sub = w.select_sequences(range(min(n_seq, w.B)))
+    args = oracle_inputs(sub)
+    passes, t0 = 0, time.perf_counter()
+    while True:
+        treewy_oracle.prepare(args[0], args[1], args[6])
+        treewy_oracle.verify_commit(*args)
+        passes += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds or passes >= 64:
+            break
+    return passes * sub.T * sub.H_v / dt, dt, passes, sub, treewy_oracle.num_threads()
+
+
+def run_reference(args, rank: int):
+    """Reference arm: the fp64 CPU oracle on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    w = wl.make_workload(args.config, B=args.ref_seqs)
+    from oracle import treewy_oracle
+    treewy_oracle.build()
+    oargs = oracle_inputs(w)
+    units = w.T * w.H_v
+
+    def step():
+        treewy_oracle.prepare(oargs[0], oargs[1], oargs[6])
+        treewy_oracle.verify_commit(*oargs)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = units * args.steps / dt
+    full = wl._DEFAULTS[args.config]
+    sample = f"{w.B} of {full[1]} sequences of workload {full[0]} per step, all heads"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": full[0], "B": full[1], "H_v": w.H_v, "H_qk": w.H_qk,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": treewy_oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args, rank: int, size: int, local: int):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libtreewy has no CPU path")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    from paper_2608_20961_b200 import binding as tw
+    tw.load_library()
+
+    w = wl.make_workload(args.config, prefix_device=str(dev))
+    units = w.T * w.H_v
+    pb = pass_bytes(w)
+    sets = [LayerSet(w, dev) for _ in range(2)]
+    for s in sets:                       # every set holds a verified tree before step 0
+        s.prepare(), s.verify()
+    torch.cuda.synchronize(dev)
+
+    def step(i: int):
+        a, b = sets[i % 2], sets[(i + 1) % 2]
+        a.prepare()
+        a.verify()
+        b.commit()
+
+    stream = torch.cuda.current_stream(dev)
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize(dev)
+    replicas.barrier(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        e0.record(stream)
+        for i in range(args.steps):
+            step(args.warmup + i)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+    replicas.barrier(dev)
+    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
+    ms_per_step = ms / args.steps
+    value = size * units * args.steps / (ms * 1e-3)
+
+    # per-kernel durations, separate pass: events around every launch on the launching stream
+    kb = max(3, min(args.steps, 50))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb)]
+    for i in range(kb):
+        a, b = sets[i % 2], sets[(i + 1) % 2]
+        ev[i][0].record(stream)
+        a.prepare()
+        ev[i][1].record(stream)
+        a.verify()
+        ev[i][2].record(stream)
+        b.commit()
+        ev[i][3].record(stream)
+    torch.cuda.synchronize(dev)
+    kt = [sum(e[j].elapsed_time(e[j + 1]) for e in ev) / kb for j in range(3)]   # ms
+    assert not any(int(s.status.max()) for s in sets), "a sequence was flagged"
+
+    hbm, tf, which = measured_peaks()
+    verify_gbs = pb.verify / (kt[1] * 1e-3) / 1e9
+    roof_ms = max(pb.total / (hbm * 1e9), pb.tensor_flops / (tf * 1e12)) * 1e3
+    roofline = {"bound": "hbm", "kernel": "treewy_verify", "achieved": verify_gbs, "peak": hbm,
+                "unit": "GB/s", "frac": verify_gbs / hbm, "peak_source": f"of {which}",
+                "traffic": VERIFY_DRAM_TRAFFIC_BYTES.get(args.config),
+                "algorithmic_bytes_per_launch": pb.verify}
+
+    # end to end through the user-level API: pinned host inputs in, outputs back, every step
+    ke = max(3, min(args.steps, 20))
+    layer = tw.VerifyCommitLayer(sets[0].S0, w.H_qk, w.T, w.max_nodes)
+    host = {n: getattr(w, n).contiguous().pin_memory()
+            for n in ("q", "k", "v", "alpha", "beta", "parent", "node_offsets", "accepted")}
+    O_host = torch.empty((w.T, w.H_v, 128), dtype=w.io_dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = O_host.numel() * O_host.element_size()
+    for _ in range(3):
+        layer.step(host, O_host)
+    torch.cuda.synchronize(dev)
+    replicas.barrier(dev)
+    e0.record(stream)
+    for _ in range(ke):
+        layer.step(host, O_host)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
+    e2e = {"value": size * units * ke / (e2e_ms * 1e-3), "unit": UNIT, "steps": ke,
+           "ms_per_step": e2e_ms / ke, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.io_dtype == torch.bfloat16 else "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H_v": w.H_v, "H_qk": w.H_qk, "T": w.T,
+                   "max_nodes": w.max_nodes, "seed": w.seed,
+                   "l2": "inputs larger than L2: two layer sets (~0.6 GB each) rotated, commit "
+                         "runs one step after its verify",
+                   "parallelism": f"replicas x{size}, no collective"},
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 3 * args.steps,
+        "roofline": roofline,
+        "step_roofline": {"bytes": pb.total, "tensor_flops": pb.tensor_flops, "roof_ms": roof_ms,
+                          "frac": roof_ms / ms_per_step, "peak_source": f"of {which}"},
+        "kernel_ms": {"prepare": kt[0], "verify": kt[1], "commit": kt[2]},
+        "kernel_gbs": {"prepare": pb.prepare / kt[0] / 1e6, "verify": verify_gbs,
+                       "commit": pb.commit / kt[2] / 1e6},
+        "footprint": footprint.footprint_report(w.max_nodes, w.H_v, w.H_qk),
+    }
+    if rank == 0 and size == 1 and not args.no_cpu_baseline:
+        v, dt, passes, sub, cores = time_oracle(w, args.cpu_seqs)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "seconds": dt,
+                               "sample": f"first {sub.B} of {w.B} sequences, all heads, {passes} passes"}
+    if rank == 0:
+        print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=2, help="workload id (2 = the metric's)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seqs", type=int, default=256, help="sequences the CPU baseline times")
+    ap.add_argument("--ref-seqs", type=int, default=16, help="sequences per reference-arm step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank, size, local = replicas.world()
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    rank, size, local = replicas.init()
+    try:
+        run_ours(args, rank, size, local)
+    finally:
+        replicas.shutdown()
+
+
+if __name__ == "__main__":
+    main()
