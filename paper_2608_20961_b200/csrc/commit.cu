@@ -168,7 +168,7 @@ cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t s
 {
     if (a.B == 0 || a.H_v == 0) return cudaSuccess;
     if (io == TREEWY_F32) return launch_cm<float, 4>(a, stream);
-    return launch_cm<__nv_bfloat16, 4>(a, stream);
+    return launch_commit_pipe(a, stream);
 }
 
 }  // namespace treewy

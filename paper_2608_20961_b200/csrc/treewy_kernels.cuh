@@ -38,5 +38,6 @@ cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *a
 cudaError_t launch_verify_generic(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od,
                                   cudaStream_t stream);
 cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
+cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream);  // bf16 state
 
 }  // namespace treewy
