@@ -51,8 +51,10 @@ treewy_status_t verify_common(bool force_generic, const void *S0, const void *q,
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
-    (void)force_generic;
-    e = launch_verify_generic(a, io_dtype, o_dtype, stream);
+    if (io_dtype == TREEWY_BF16 && !force_generic)
+        e = launch_verify_sm100(a, tree->T, o_dtype, stream);
+    else
+        e = launch_verify_generic(a, io_dtype, o_dtype, stream);
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 
