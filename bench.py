@@ -228,7 +228,7 @@ def run_ours(args, rank: int, size: int, local: int):
     from paper_2608_20961_b200 import binding as tw
     tw.load_library()
 
-    w = wl.make_workload(args.config, prefix_device=str(dev))
+    w = wl.make_workload(args.config, B=args.batch, prefix_device=str(dev))
     units = w.T * w.H_v
     pb = pass_bytes(w)
     sets = [LayerSet(w, dev) for _ in range(2)]
@@ -338,6 +338,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=2, help="workload id (2 = the metric's)")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the workload's batch size (profiling captures on a small case)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seqs", type=int, default=256, help="sequences the CPU baseline times")
     ap.add_argument("--ref-seqs", type=int, default=16, help="sequences per reference-arm step")

@@ -84,13 +84,16 @@ typedef struct {
                                     ancestor of the node or the node itself */
     float *cum_log_gate;         /* [T,H_v] device, out: L[i,h] = sum over the root path of i,
                                     i included, of log(alpha[.,h])  (log of g_i in Eq. 2) */
+    uint8_t *level_order;        /* [T]   device, out: each sequence's local node indices sorted by
+                                    (depth, index).  Nodes of equal depth never depend on each
+                                    other, so verify solves them side by side in this order */
 } treewy_tree_t;
 
 /*
  * Tree indexing (Section 3, "Verifying a draft"; g_t of Eq. 2).
  * Reads tree->node_offsets, tree->parent and alpha [T,H_v] (fp32, linear gates in (0,1]);
- * writes tree->depth, tree->anc_mask (bit-exact, one correct value each) and
- * tree->cum_log_gate (fp32 sums of logf).  One small kernel on `cuda_stream`.
+ * writes tree->depth, tree->anc_mask, tree->level_order (bit-exact, one correct value each)
+ * and tree->cum_log_gate (fp32 sums of logf).  One small kernel on `cuda_stream`.
  * Malformed sequences get TREEWY_SEQ_BAD_PARENT / TREEWY_SEQ_TOO_MANY_NODES.
  * Topology is per decoding step, the log-gates per layer: call it once per layer, or reuse
  * depth / anc_mask across layers and let it rewrite only what changed.

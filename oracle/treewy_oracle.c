@@ -26,6 +26,7 @@
  *        anc_mask[t] = bit t  |  anc_mask[parent]            (ancestor-or-self)
  *        L[t,h]      = log(alpha[t,h]) + L[parent,h]          (log of the cumulative
  *                      decay g_t of Eq. 2, which includes node t's own alpha)
+ *        level_order = the sequence's nodes sorted by (depth, index)
  *
  * Matrix products are written as the triple loops of their definition.  The only
  * algebra applied to Eq. 1 is associativity of  S (k k^T) = (S k) k^T.
@@ -75,12 +76,13 @@ static int check_sequence(const int32_t *node_offsets, const int32_t *parent, in
 
 /*
  * Tree indexing.  alpha is [T, H_v] (already widened to fp64 by the caller).
- * depth [T], anc_mask [T], L [T, H_v] are written for well-formed sequences and
+ * depth [T], anc_mask [T], L [T, H_v], level_order [T] are written for well-formed sequences and
  * left untouched for malformed ones, whose seq_status[b] gets the reason OR-ed in.
  */
 int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
                           const int32_t *parent, const double *alpha, int32_t *depth,
-                          uint64_t *anc_mask, double *L, int32_t *seq_status)
+                          uint64_t *anc_mask, double *L, uint8_t *level_order,
+                          int32_t *seq_status)
 {
     for (int32_t b = 0; b < B; ++b) {
         const int bad = check_sequence(node_offsets, parent, b);
@@ -98,6 +100,14 @@ int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
                 const double up = (p < 0) ? 0.0 : L[(size_t)(lo + p) * H_v + h];
                 L[(size_t)(lo + i) * H_v + h] = up + log(alpha[(size_t)(lo + i) * H_v + h]);
             }
+        }
+        /* nodes sorted by (depth, index): one pass per depth value, in index order */
+        if (level_order) {
+            int32_t out = 0;
+            for (int32_t d = 0; out < n; ++d)
+                for (int32_t i = 0; i < n; ++i)
+                    if (depth[lo + i] == d)
+                        level_order[lo + out++] = (uint8_t)i;
         }
     }
     return 0;

@@ -69,6 +69,7 @@ class OracleTree:
     depth: np.ndarray        # int32 [T]
     anc_mask: np.ndarray     # uint64 [T], bit j = local node j is ancestor-or-self
     cum_log_gate: np.ndarray  # float64 [T, H_v]
+    level_order: np.ndarray  # uint8 [T], each sequence's nodes sorted by (depth, index)
     seq_status: np.ndarray   # int32 [B]
 
 
@@ -93,11 +94,13 @@ def prepare(node_offsets, parent, alpha) -> OracleTree:
     depth = np.full(T, -1, np.int32)
     mask = np.zeros(T, np.uint64)
     L = np.zeros((T, H_v), np.float64)
+    order = np.zeros(T, np.uint8)
     status = np.zeros(B, np.int32)
     rc = lib.treewy_oracle_prepare(ctypes.c_int32(B), ctypes.c_int32(H_v), _ptr(off), _ptr(par),
-                                   _ptr(al), _ptr(depth), _ptr(mask), _ptr(L), _ptr(status))
+                                   _ptr(al), _ptr(depth), _ptr(mask), _ptr(L), _ptr(order),
+                                   _ptr(status))
     assert rc == 0
-    return OracleTree(depth, mask, L, status)
+    return OracleTree(depth, mask, L, order, status)
 
 
 def verify_commit(node_offsets, parent, S0, q, k, v, alpha, beta, accepted,

@@ -32,7 +32,7 @@ class TreeStruct(ctypes.Structure):
         ("max_nodes", ctypes.c_int32),
         ("node_offsets", ctypes.c_void_p), ("parent", ctypes.c_void_p),
         ("depth", ctypes.c_void_p), ("anc_mask", ctypes.c_void_p),
-        ("cum_log_gate", ctypes.c_void_p),
+        ("cum_log_gate", ctypes.c_void_p), ("level_order", ctypes.c_void_p),
     ]
 
 
@@ -110,6 +110,7 @@ class Tree:
     depth: torch.Tensor          # int32 [T]
     anc_mask: torch.Tensor       # int64 storage of the uint64 masks [T]
     cum_log_gate: torch.Tensor   # fp32 [T, H_v]
+    level_order: torch.Tensor    # uint8 [T]
 
     @classmethod
     def empty(cls, node_offsets: torch.Tensor, parent: torch.Tensor, H_v: int,
@@ -120,13 +121,14 @@ class Tree:
                    node_offsets=node_offsets, parent=parent,
                    depth=torch.full((max(T, 1),), -1, dtype=torch.int32, device=dev),
                    anc_mask=torch.zeros((max(T, 1),), dtype=torch.int64, device=dev),
-                   cum_log_gate=torch.zeros((max(T, 1), H_v), dtype=torch.float32, device=dev))
+                   cum_log_gate=torch.zeros((max(T, 1), H_v), dtype=torch.float32, device=dev),
+                   level_order=torch.zeros((max(T, 1),), dtype=torch.uint8, device=dev))
 
     def struct(self) -> TreeStruct:
         return TreeStruct(self.B, self.T, self.H_v, self.max_nodes,
                           self.node_offsets.data_ptr(), self.parent.data_ptr(),
                           self.depth.data_ptr(), self.anc_mask.data_ptr(),
-                          self.cum_log_gate.data_ptr())
+                          self.cum_log_gate.data_ptr(), self.level_order.data_ptr())
 
 
 def treewy_tree_prepare(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tensor | None = None,
@@ -187,10 +189,11 @@ class VerifyCommitLayer:
         self.depth = z((max_T,), torch.int32)
         self.anc_mask = z((max_T,), torch.int64)
         self.cum_log_gate = z((max_T, self.H_v), torch.float32)
+        self.level_order = z((max_T,), torch.uint8)
 
     def tree(self, T: int) -> Tree:
         return Tree(self.B, T, self.H_v, self.max_nodes, self.node_offsets, self.parent,
-                    self.depth, self.anc_mask, self.cum_log_gate)
+                    self.depth, self.anc_mask, self.cum_log_gate, self.level_order)
 
     def upload(self, host: dict) -> int:
         """Host (pinned) tensors -> device buffers on the current stream; returns T."""

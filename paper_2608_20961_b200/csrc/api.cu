@@ -22,7 +22,8 @@ treewy_status_t check_tree(const treewy_tree_t *t, bool need_outputs, int *max_n
     if (bad_ptr(t->node_offsets)) return TREEWY_ERR_INVALID_ARG;
     if (t->T > 0 && bad_ptr(t->parent)) return TREEWY_ERR_INVALID_ARG;
     if (need_outputs && t->T > 0 &&
-        (bad_ptr(t->depth) || bad_ptr(t->anc_mask) || bad_ptr(t->cum_log_gate)))
+        (bad_ptr(t->depth) || bad_ptr(t->anc_mask) || bad_ptr(t->cum_log_gate) ||
+         bad_ptr(t->level_order)))
         return TREEWY_ERR_INVALID_ARG;
     return TREEWY_OK;
 }
@@ -47,6 +48,7 @@ treewy_status_t verify_common(bool force_generic, const void *S0, const void *q,
     a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -1,4 +1,4 @@
-// treewy_tree_prepare: parent array -> depth, ancestor-or-self bitmask, cumulative log-gate
+// treewy_tree_prepare: parent array -> depth, ancestor-or-self bitmask, level order, cumulative log-gate
 // (Section 3, "Verifying a draft"; g_t of Eq. 2 as a running sum of log alpha).
 //
 // One CTA per sequence.  Thread 0 walks the <= 64 nodes once for depth / mask (each node
@@ -18,7 +18,8 @@ __global__ void __launch_bounds__(PREP_THREADS)
 prepare_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_offsets,
                const int32_t *__restrict__ parent, const float *__restrict__ alpha,
                int32_t *__restrict__ depth, uint64_t *__restrict__ anc_mask,
-               float *__restrict__ cum_log_gate, int32_t *__restrict__ seq_status)
+               float *__restrict__ cum_log_gate, uint8_t *__restrict__ level_order,
+               int32_t *__restrict__ seq_status)
 {
     __shared__ int s_bad;
     __shared__ int32_t s_depth[MAXN];
@@ -65,8 +66,16 @@ prepare_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_o
         }
     }
     for (int i = threadIdx.x; i < n; i += PREP_THREADS) {
-        depth[lo + i] = s_depth[i];
+        const int di = s_depth[i];
+        depth[lo + i] = di;
         anc_mask[lo + i] = s_mask[i];
+        // position of node i when the nodes are sorted by (depth, index)
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const int dj = s_depth[j];
+            rank += (dj < di) || (dj == di && j < i);
+        }
+        level_order[lo + rank] = (uint8_t)i;
     }
 }
 
@@ -76,7 +85,7 @@ cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *a
     if (t.B == 0) return cudaSuccess;
     prepare_kernel<<<t.B, PREP_THREADS, 0, stream>>>(t.B, t.H_v, max_nodes, t.node_offsets,
                                                      t.parent, alpha, t.depth, t.anc_mask,
-                                                     t.cum_log_gate, seq_status);
+                                                     t.cum_log_gate, t.level_order, seq_status);
     return cudaGetLastError();
 }
 

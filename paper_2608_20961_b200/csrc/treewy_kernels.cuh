@@ -14,6 +14,8 @@ struct VerifyArgs {
     const int32_t *node_offsets, *parent;
     const uint64_t *anc_mask;
     const float *cum_log_gate;
+    const int32_t *depth;
+    const uint8_t *level_order;
     void *O;
     float *U;
     int32_t *seq_status;

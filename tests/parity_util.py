@@ -58,6 +58,7 @@ def run_gpu(w, o_dtype=torch.float32, generic=False, device="cuda:0", max_nodes=
     return dict(depth=tree.depth.cpu().numpy()[:T],
                 anc_mask=tree.anc_mask.cpu().numpy().view(np.uint64)[:T],
                 cum_log_gate=tree.cum_log_gate.cpu().numpy()[:T],
+                level_order=tree.level_order.cpu().numpy()[:T],
                 O=O.cpu()[:T], U=U.cpu()[:T], S=S.cpu(), S32=None if S32 is None else S32.cpu(),
                 status=status.cpu().numpy()[:w.B], canary=canary)
 
@@ -101,6 +102,7 @@ def assert_parity(w, gpu, tree_ref, ref, arith=True, skip_seqs=()):
     # integer outputs: bit-exact
     np.testing.assert_array_equal(gpu["depth"][rows], tree_ref.depth[rows])
     np.testing.assert_array_equal(gpu["anc_mask"][rows], tree_ref.anc_mask[rows])
+    np.testing.assert_array_equal(gpu["level_order"][rows], tree_ref.level_order[rows])
     np.testing.assert_allclose(gpu["cum_log_gate"][rows], tree_ref.cum_log_gate[rows], rtol=0,
                                atol=1e-5)
     sub_off = np.concatenate([[0], np.cumsum([off[b + 1] - off[b] for b in keep])])

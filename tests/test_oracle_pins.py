@@ -296,6 +296,9 @@ def test_prepare_against_parent_walk(oracle, seed):
     tr = oracle.prepare(off, parent, alpha)
     assert not tr.seq_status.any()
     for b, tree in enumerate(trees):
+        depths = [len(path_to(tree, i)) - 1 for i in range(len(tree))]
+        want = sorted(range(len(tree)), key=lambda i: (depths[i], i))
+        assert list(tr.level_order[off[b]:off[b + 1]]) == want
         for i in range(len(tree)):
             path = path_to(tree, i)
             t = off[b] + i
