@@ -140,3 +140,39 @@ def assert_bf16_outputs(w, gpu_bf16, gpu_f32, ref):
     assert f <= FROB_GATE, (m, f)
     assert m <= 2.0 * m0 + 1e-3, (m, m0)      # no worse than storage rounding explains
     return (m, f), (m0, f0)
+
+
+def assert_parity_sampled(oracle, w, gpu, seqs):
+    """Full-size run: compare the listed sequences (all heads, every output) against the oracle
+    run on exactly those sequences; returns the worst errors."""
+    sub = w.select_sequences(seqs)
+    tree_ref, ref = run_oracle(oracle, sub)
+    off = w.node_offsets.numpy()
+    rows = np.array([i for b in seqs for i in range(off[b], off[b + 1])], dtype=np.int64)
+    pick = {"depth": gpu["depth"][rows], "anc_mask": gpu["anc_mask"][rows],
+            "cum_log_gate": gpu["cum_log_gate"][rows], "level_order": gpu["level_order"][rows],
+            "O": gpu["O"][rows], "U": gpu["U"][rows], "S": gpu["S"][list(seqs)],
+            "S32": gpu["S32"][list(seqs)], "status": gpu["status"][list(seqs)]}
+    return assert_parity(sub, pick, tree_ref, ref)
+
+
+def assert_tree_invariants(w, gpu):
+    """Properties that hold for every node at any size (no oracle needed)."""
+    off = w.node_offsets.numpy()
+    par = w.parent.numpy()
+    depth, mask, order = gpu["depth"], gpu["anc_mask"], gpu["level_order"]
+    pop = np.array([bin(int(m)).count("1") for m in mask])
+    assert np.array_equal(pop, depth + 1)
+    local = np.concatenate([np.arange(off[b + 1] - off[b]) for b in range(w.B)])
+    assert np.all((mask >> local.astype(np.uint64)) & np.uint64(1) == 1)          # self bit
+    has_parent = par >= 0
+    seq_start = np.repeat(off[:-1], off[1:] - off[:-1])
+    pmask = mask[(seq_start + np.maximum(par, 0))]
+    low = mask & ((np.uint64(1) << local.astype(np.uint64)) - np.uint64(1))
+    assert np.array_equal(low[has_parent], pmask[has_parent]) and not low[~has_parent].any()
+    for b in range(w.B):
+        sl = slice(off[b], off[b + 1])
+        o = order[sl].astype(np.int64)
+        assert sorted(o.tolist()) == list(range(off[b + 1] - off[b]))
+        d = depth[sl][o]
+        assert np.all(np.diff(d) >= 0)
