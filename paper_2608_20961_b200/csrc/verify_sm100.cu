@@ -40,6 +40,7 @@
 #include <cuda.h>
 
 #include "ptx_sm100.cuh"
+#include "tma_host.cuh"
 #include "treewy_common.cuh"
 #include "treewy_kernels.cuh"
 
@@ -426,50 +427,13 @@ verify_sm100_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorM
 // ------------------------------------------------------------------------------ host side
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-        return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(fn);
-}
-
-// bf16 matrix [rows, cols] with `row_bytes` between rows; box = box_cols x box_rows
-bool make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows,
-              uint64_t row_bytes, uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle sw)
-{
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {row_bytes};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int NP, typename TOut>
 cudaError_t launch_vs(const VerifyArgs &a, int T, cudaStream_t stream)
 {
     using C = VsCfg<NP>;
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return cudaErrorNotSupported;
     const long long n_items = (long long)a.B * a.H_v;
-    CUtensorMap tmS0, tmQ, tmK, tmV;
-    bool ok = make_map(enc, &tmS0, a.S0, D, (uint64_t)n_items * D, D * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map(enc, &tmQ, a.q, (uint64_t)a.H_qk * D, T, (uint64_t)a.H_qk * D * 2, 64, NP,
-                        CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map(enc, &tmK, a.k, (uint64_t)a.H_qk * D, T, (uint64_t)a.H_qk * D * 2, 64, NP,
-                        CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map(enc, &tmV, a.v, (uint64_t)a.H_v * D, T, (uint64_t)a.H_v * D * 2, 128, NP,
-                        CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (!ok) return cudaErrorInvalidValue;
+    VerifyMaps m;
+    if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_items, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -479,25 +443,22 @@ cudaError_t launch_vs(const VerifyArgs &a, int T, cudaStream_t stream)
                              C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int grid = (int)(n_items < sms ? n_items : sms);
-    verify_sm100_kernel<NP, TOut><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, (int)n_items, tmS0, tmQ,
-                                                                                tmK, tmV);
+    verify_sm100_kernel<NP, TOut><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, (int)n_items, m.S0, m.Q,
+                                                                                m.K, m.V);
     return cudaGetLastError();
-}
-
-template <typename TOut> cudaError_t launch_vs_np(const VerifyArgs &a, int T, cudaStream_t stream)
-{
-    if (a.max_nodes <= 16) return launch_vs<16, TOut>(a, T, stream);
-    if (a.max_nodes <= 32) return launch_vs<32, TOut>(a, T, stream);
-    return launch_vs<64, TOut>(a, T, stream);
 }
 
 }  // namespace
 
-cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
+// general variant: any tree of up to 64 nodes; the solve runs on the CUDA cores
+cudaError_t launch_verify_sm100_simt(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
 {
-    if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
-    if (od == TREEWY_F32) return launch_vs_np<float>(a, T, stream);
-    return launch_vs_np<__nv_bfloat16>(a, T, stream);
+    if (a.max_nodes <= 32) {
+        if (od == TREEWY_F32) return launch_vs<32, float>(a, T, stream);
+        return launch_vs<32, __nv_bfloat16>(a, T, stream);
+    }
+    if (od == TREEWY_F32) return launch_vs<64, float>(a, T, stream);
+    return launch_vs<64, __nv_bfloat16>(a, T, stream);
 }
 
 }  // namespace treewy

@@ -1,0 +1,599 @@
+// treewy_verify, bf16 production kernel for trees of up to 32 nodes (Section 3: Eq. 2 and the
+// read-out), with BOTH contractions of the method on the tcgen05 tensor cores:
+//
+//   stage 1 (bf16 x bf16 -> fp32):   D1 = S0 [Q;K]^T  (S0 q_i, S0 k_i),   D2 = [Q;K] K^T  (Gram)
+//   stage 2 (tf32 split, ~fp32):     U^T = R^T T^T ,   (O - g.S0q)^T = R^T W^T
+//
+// where R[j] = beta_j (v_j - g_j S0 k_j) is the right-hand side of Eq. 2, T = (I + A)^{-1} and
+// W = P T.  The triangular system is not solved column by column: because A only couples a
+// node with its ancestors, row i of T (and of W) lives on node i's root path and is the last
+// row of the inverse of the small path matrix I + A_path, which one thread obtains by a
+// back-substitution of depth(i) steps.  All rows are independent, so the sequential part of
+// the solve shrinks from N steps per column to depth steps per node, done once per item, and
+// the N x N x 128 products go to the tensor pipe.
+//
+// fp32 accuracy on the tf32 pipe: every operand x is split as hi = x with the low 13 mantissa
+// bits cleared (exactly representable in tf32) and lo = x - hi; the kernel accumulates
+// hi.hi + lo.hi + hi.lo in fp32, dropping only lo.lo (relative 2^-22).
+//
+// Roles (persistent CTA, one per SM; item = one (sequence, value head)):
+//   producer warps   TMA tensor-map loads of S0 / [Q;K] / V into a stage ring, node scalars
+//   MMA-1 warp       stage-1 MMAs into a TMEM buffer           -> mma1_done
+//   consumer groups  (2 x 128 threads, alternate items; thread c = TMEM lane c = row c of d_v)
+//       G: Gram rows -> scaled ancestor lists (A, P, indices), branch-free column scan
+//       T: per-node back-substitution -> rows of T and W, scattered (hi, lo) into the swizzled
+//          operand tiles that overlay the stage's dead [Q;K] tile
+//       R: R^T rows (hi, lo) into the tiles that overlay the dead S0 tile    -> ops_ready
+//   MMA-2 warp       stage-2 MMAs (3 passes each for U and O)   -> mma2_done, stage released
+//   consumer groups  epilogue: u_i = DU[i], o_i = g_i (S0 q_i) + DO[i]; coalesced stores
+//
+// Every mbarrier wait is bounded; on give-up the role leaves its loop, TREEWY_SEQ_TIMEOUT is
+// raised, and the CTA still reaches the common exit where tensor memory is freed.
+#include <cuda.h>
+
+#include "ptx_sm100.cuh"
+#include "tma_host.cuh"
+#include "treewy_common.cuh"
+#include "treewy_kernels.cuh"
+
+namespace treewy {
+
+constexpr int VT_GROUP = 128;
+constexpr uint32_t VT_TMEM_COLS = 512;
+
+template <int NP> struct VtCfg {
+    static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
+    static constexpr int GROUPS = 2;
+    static constexpr int STAGES = NP <= 16 ? 4 : 3;
+    static constexpr int TBUF = 5;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
+    static constexpr int CONSUMERS = VT_GROUP * GROUPS;
+    static constexpr int MMA1_WARP = CONSUMERS / 32;
+    static constexpr int MMA2_WARP = MMA1_WARP + 1;
+    static constexpr int PROD_WARP0 = MMA2_WARP + 1;
+    static constexpr int THREADS = CONSUMERS + 64 + 32 * STAGES;
+    // stage: [Q;K] tile | S0 tile | V rows | meta
+    static constexpr int QK_HALF = 2 * NP * 128;
+    static constexpr int QK_BYTES = 2 * QK_HALF;
+    static constexpr int S0_HALF = D * 128;
+    static constexpr int S0_BYTES = 2 * S0_HALF;
+    static constexpr int V_BYTES = NP * D * 2;
+    static constexpr int OFF_S0 = QK_BYTES;
+    static constexpr int OFF_V = OFF_S0 + S0_BYTES;
+    static constexpr int OFF_META = OFF_V + V_BYTES;
+    static constexpr int META_BYTES = NP * 16 + 16;  // mask u64, L f32, beta f32 per node; n, lo
+    static constexpr int STAGE_BYTES = (OFF_META + META_BYTES + 1023) / 1024 * 1024;
+    // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
+    static constexpr int OFF_T_HI = 0, OFF_T_LO = NP * 128, OFF_W_HI = 2 * NP * 128, OFF_W_LO = 3 * NP * 128;
+    static constexpr int OFF_RT_HI = OFF_S0, OFF_RT_LO = OFF_S0 + D * 128;
+    static_assert(4 * NP * 128 <= QK_BYTES && 2 * D * 128 <= S0_BYTES, "operand overlays fit");
+    // group-private: path lists, per-node scalars, back-substitution rows
+    static constexpr int XLD = NP + 1;
+    static constexpr int GP_AP = 0, GP_PP = NP * NP * 4, GP_SCAL = 2 * NP * NP * 4;
+    static constexpr int GP_XR = GP_SCAL + 2 * NP * 16;  // per-node scalars are double-buffered
+    static constexpr int GP_IDX = GP_XR + 2 * NP * XLD * 4;
+    static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
+    static constexpr int GP_RAW = (GP_IDX + NP * NP + 15) / 16 * 16;
+    static constexpr int GP_BYTES = GP_RAW + 2 * NP * RLD * 4;
+    static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
+    static constexpr int OFF_GP = STAGES * STAGE_BYTES;
+    static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
+    static constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 4 * TBUF) * 8 + 16 + 1024;
+    static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES + V_BYTES;
+    // per TMEM buffer: SQ | SK | D2; stage 2 writes DO over SK and DU over D2 (both dead by then)
+    static constexpr int TM_COLS = 3 * NP;
+    static constexpr int TM_DO = NP, TM_DU = 2 * NP;
+    static_assert(TBUF * TM_COLS <= 512, "tensor memory");
+};
+
+// instruction descriptor, kind::tf32: tf32 x tf32 -> fp32, both operands K-major, dense
+__host__ __device__ constexpr uint32_t umma_idesc_tf32_f32(int M, int N)
+{
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// stores that are predicated instead of branched around (keeps the epilogue one straight line)
+__device__ __forceinline__ void st_global_if(float *p, float v, bool on)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v),
+                 "r"((int)on));
+}
+__device__ __forceinline__ void st_global_if(__nv_bfloat16 *p, float v, bool on)
+{
+    const unsigned short b = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.b16 [%0], %1;\n\t}" ::"l"(p), "h"(b),
+                 "r"((int)on));
+}
+
+__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
+
+template <int NP, typename TOut>
+__global__ void __launch_bounds__(VtCfg<NP>::THREADS, 1)
+verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorMap tmS0,
+                       const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                       const __grid_constant__ CUtensorMap tmV)
+{
+    using C = VtCfg<NP>;
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char *smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
+    uint64_t *empty = full + C::STAGES;
+    uint64_t *mma1_done = empty + C::STAGES;
+    uint64_t *ops_ready = mma1_done + C::TBUF;
+    uint64_t *mma2_done = ops_ready + C::TBUF;
+    uint64_t *tmem_free = mma2_done + C::TBUF;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tmem_free + C::TBUF);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        for (int i = 0; i < C::TBUF; ++i) {
+            ptx::mbar_init(&mma1_done[i], 1);
+            ptx::mbar_init(&ops_ready[i], VT_GROUP);
+            ptx::mbar_init(&mma2_done[i], 1);
+            ptx::mbar_init(&tmem_free[i], VT_GROUP);
+        }
+        ptx::fence_barrier_init();
+    }
+    if (warp == C::MMA1_WARP) {
+        ptx::tmem_alloc(tmem_slot, VT_TMEM_COLS);
+        ptx::tmem_relinquish();
+        ptx::tc_fence_before_sync();
+    }
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto meta_mask = [&](unsigned char *stage) { return reinterpret_cast<unsigned long long *>(stage + C::OFF_META); };
+    auto meta_L = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 8); };
+    auto meta_beta = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 12); };
+    auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
+
+    if (warp >= C::PROD_WARP0) {
+        // ------------------------------------------------------------------ producer warp
+        const int s = warp - C::PROD_WARP0;
+        unsigned char *stage = smem + s * C::STAGE_BYTES;
+        if (lane == 0) {
+            ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ);
+            ptx::prefetch_tmap(&tmK), ptx::prefetch_tmap(&tmV);
+        }
+        const int group = a.H_v / a.H_qk;
+        // Node scalars of an item: validated and loaded one round ahead (software pipeline), so the
+        // dependent chain  node_offsets -> parent / mask / log-gate / beta  never delays a TMA issue.
+        struct Pre {
+            int item, b, h, lo, n, bad;
+            unsigned long long mk;
+            float Lv, bv;
+        };
+        auto fetch = [&](int kk) {
+            Pre p;
+            p.item = blockIdx.x + kk * gridDim.x;
+            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
+            if (p.item >= n_items) return p;
+            p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
+            p.lo = a.node_offsets[p.b];
+            p.n = a.node_offsets[p.b + 1] - p.lo;
+            if (p.n < 1 || p.n > a.max_nodes || p.n > NP) {
+                p.bad = TREEWY_SEQ_TOO_MANY_NODES;
+            } else {
+                const int par = lane < p.n ? a.parent[p.lo + lane] : -1;
+                if (__any_sync(0xffffffffu, lane < p.n && (par < -1 || par >= lane))) p.bad = TREEWY_SEQ_BAD_PARENT;
+            }
+            const bool on = !p.bad && lane < p.n;  // NP <= 32: one node per lane
+            p.mk = on ? a.anc_mask[p.lo + lane] : 0ull;
+            p.Lv = on ? a.cum_log_gate[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
+            p.bv = on ? a.beta[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
+            return p;
+        };
+        Pre cur = fetch(s);
+        for (int kk = s;; kk += C::STAGES) {
+            if (cur.item >= n_items) break;
+            const Pre p = cur;
+            if (p.bad && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
+            if (!ptx::mbar_wait(&empty[s], ((kk / C::STAGES) & 1) ^ 1)) {
+                if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], TREEWY_SEQ_TIMEOUT);
+                break;
+            }
+            if (lane < NP) meta_mask(stage)[lane] = p.mk, meta_L(stage)[lane] = p.Lv, meta_beta(stage)[lane] = p.bv;
+            if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo;
+            __syncwarp();
+            if (lane == 0) {
+                if (p.bad) {
+                    ptx::mbar_arrive(&full[s]);
+                } else {
+                    ptx::mbar_arrive_expect_tx(&full[s], C::TX_BYTES);
+                    const int hq = p.h / group;
+                    ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.item * D, &full[s]);
+                    ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.item * D, &full[s]);
+                    ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
+                    ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
+                    ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
+                    ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
+                    ptx::tma_load_2d(stage + C::OFF_V, &tmV, p.h * D, p.lo, &full[s]);
+                }
+            }
+            cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
+        }
+    } else if (warp == C::MMA1_WARP) {
+        // ------------------------------------------------------------------ stage-1 MMAs
+        constexpr uint32_t idesc1 = ptx::umma_idesc_bf16_f32(128, 2 * NP);
+        constexpr uint32_t idesc2 = ptx::umma_idesc_bf16_f32(128, NP);
+        for (int kk = 0;; ++kk) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            if (item >= n_items) break;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) break;
+            const int n = meta_nlo(stage)[0];
+            if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
+            ptx::tc_fence_after_sync();
+            if (lane == 0) {
+                if (n > 0) {
+                    const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
+                    const uint32_t d1 = tmem_base + buf * C::TM_COLS, d2 = d1 + 2 * NP;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t ko = (ks & 3) * 32;
+                        const uint64_t da = ptx::umma_desc_k_sw128(s0 + (ks >> 2) * C::S0_HALF + ko);
+                        const uint64_t db = ptx::umma_desc_k_sw128(qk + (ks >> 2) * C::QK_HALF + ko);
+                        ptx::umma_bf16(d1, da, db, idesc1, ks > 0);
+                    }
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t ko = (ks & 3) * 32;
+                        const uint32_t base = qk + (ks >> 2) * C::QK_HALF + ko;
+                        ptx::umma_bf16(d2, ptx::umma_desc_k_sw128(base), ptx::umma_desc_k_sw128(base + NP * 128),
+                                       idesc2, ks > 0);
+                    }
+                    ptx::umma_commit(&mma1_done[buf]);
+                } else {
+                    ptx::mbar_arrive(&mma1_done[buf]);
+                }
+            }
+            __syncwarp();
+        }
+    } else if (warp == C::MMA2_WARP) {
+        // ------------------------------------------------------------------ stage-2 MMAs
+        constexpr uint32_t idesc = umma_idesc_tf32_f32(128, NP);
+        for (int kk = 0;; ++kk) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            if (item >= n_items) break;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            if (!ptx::mbar_wait(&ops_ready[buf], (kk / C::TBUF) & 1)) break;
+            ptx::tc_fence_after_sync();
+            const int n = meta_nlo(stage)[0];
+            if (lane == 0) {
+                if (n > 0) {
+                    const uint32_t base = ptx::smem_u32(stage);
+                    const uint32_t dU = tmem_base + buf * C::TM_COLS + C::TM_DU;
+                    const uint32_t dO = tmem_base + buf * C::TM_COLS + C::TM_DO;
+                    const uint32_t rt[3] = {base + C::OFF_RT_HI, base + C::OFF_RT_LO, base + C::OFF_RT_HI};
+                    const uint32_t tt[3] = {base + C::OFF_T_HI, base + C::OFF_T_HI, base + C::OFF_T_LO};
+                    const uint32_t ww[3] = {base + C::OFF_W_HI, base + C::OFF_W_HI, base + C::OFF_W_LO};
+#pragma unroll
+                    for (int p = 0; p < 3; ++p)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_tf32(dU, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
+                                      ptx::umma_desc_k_sw128(tt[p] + ks * 32), idesc, (p | ks) != 0);
+#pragma unroll
+                    for (int p = 0; p < 3; ++p)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_tf32(dO, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
+                                      ptx::umma_desc_k_sw128(ww[p] + ks * 32), idesc, (p | ks) != 0);
+                    ptx::umma_commit(&mma2_done[buf]);
+                    ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
+                } else {
+                    ptx::mbar_arrive(&mma2_done[buf]);
+                    ptx::mbar_arrive(&empty[s]);
+                }
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer groups
+        const int grp = warp >> 2, t = tid & (VT_GROUP - 1);
+        unsigned char *gp = smem + C::OFF_GP + grp * C::GP_BYTES;
+        float *Ap = reinterpret_cast<float *>(gp + C::GP_AP);
+        float *Pp = reinterpret_cast<float *>(gp + C::GP_PP);
+        float4 *scal2 = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
+        float *xr = reinterpret_cast<float *>(gp + C::GP_XR);
+        unsigned char *idx = gp + C::GP_IDX;
+        float *raw = reinterpret_cast<float *>(gp + C::GP_RAW);
+        TOut *Og = static_cast<TOut *>(a.O);
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
+
+        // Software pipeline: the front half of an item (lists, T / W rows, R^T -> ops_ready) is done
+        // before the back half (epilogue) of the group's previous item, so the stage-2 MMAs of
+        // one item run under the front half of the next.
+        int b_kk = -1, b_n = 0, b_lo = 0;  // the item whose back half is pending
+        bool dead = false;
+        for (int kk = grp; !dead; kk += C::GROUPS) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            const bool have = item < n_items;
+            int f_n = 0, f_lo = 0;
+            if (have) {
+            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+            float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            if (!ptx::mbar_wait(&mma1_done[buf], (kk / C::TBUF) & 1)) {
+                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                dead = true;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
+            const int n = meta_nlo(stage)[0];
+            const int lo = meta_nlo(stage)[1];
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK | D2 | DU | DO
+            if (n > 0) {
+                const unsigned long long *mask = meta_mask(stage);
+                const float *Lm = meta_L(stage);
+                const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_V);
+
+                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
+                for (int q = t; q < 4 * NP * 128 / 16; q += VT_GROUP)
+                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
+
+                // ---- phase G1: the rows of the Gram matrix leave tensor memory (row owner = lane)
+                if ((warp & 3) * 32 < 2 * NP) {  // warps whose lanes hold [Q;K] rows
+#pragma unroll
+                    for (int c0 = 0; c0 < NP; c0 += 16) {
+                        if (c0 < n) {
+                            uint32_t g[16];
+                            ptx::tmem_ld16(tm + 2 * NP + c0, g);
+                            ptx::tmem_wait_ld();
+                            if (t < 2 * NP) {
+                                float4 *dst = reinterpret_cast<float4 *>(raw + t * C::RLD + c0);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
+                                                         __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
+                            }
+                        }
+                    }
+                }
+                ptx::named_sync(1 + grp, VT_GROUP);
+
+                // ---- phase G2: scaled ancestor lists, PARTS threads per node, a few entries each
+                //   P[i][d] = e^{L_i-L_j} q_i.k_j ,  A[i][d] = beta_i e^{L_i-L_j} k_i.k_j ,  idx[i][d] = j
+                //   for j the d-th ancestor of i; lists are stored [d / 4][node][d % 4]
+                constexpr int HALF = C::PARTS / 2;
+                const int i = t & (NP - 1), part = t / NP;
+                const bool valid = i < n;
+                const bool a_kind = part >= HALF;
+                const int sub = a_kind ? part - HALF : part;
+                const uint32_t mi = valid ? (uint32_t)mask[i] : 0u;
+                const int dp = valid ? __popc(mi) - 1 : 0;  // ancestors of node i
+                const float Li = Lm[i];
+                const float bi = meta_beta(stage)[i];
+                {
+                    const float scale = a_kind ? bi : 1.f;
+                    const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
+                    uint32_t m = mi & ~(1u << i);
+                    for (int q = 0; q < sub; ++q) m &= m - 1;
+                    for (int d = sub; d < dp; d += HALF) {
+                        const int j = __ffs(m) - 1;
+                        const float val = scale * __expf(Li - Lm[j]) * row[j];
+                        const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
+                        if (a_kind) Ap[at] = val;
+                        else Pp[at] = val, idx[at] = (unsigned char)j;
+#pragma unroll
+                        for (int q = 0; q < HALF; ++q) m &= m - 1;
+                    }
+                    if (part == 0 && valid) {
+                        const float gi = __expf(Li);
+                        scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
+                    }
+                }
+                ptx::named_sync(1 + grp, VT_GROUP);  // lists, scalars and the zero fill are in place
+
+                // ---- phase T: rows of T = (I + A)^-1 (one thread) and W = P T (another) by
+                // back-substitution along node i's root path j_0 .. j_{dp-1}, j_dp = i:
+                //   x_dp = 1 (T) or P[i][i] (W);  x_e = p_e - sum_{f > e} x_f A[j_f][j_e]
+                if (valid && sub == 0) {
+                    const bool wrow = !a_kind;
+                    const float top = wrow ? scal[i].w : 1.f;
+                    unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
+                    unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
+                    if (dp <= 8) {  // registers only, every load issued up front
+                        int jf[9];
+                        float x[9], pe[8], co[9][8];
+#pragma unroll
+                        for (int e = 0; e < 9; ++e) {
+                            jf[e] = e < dp ? idx[((e >> 2) * NP + i) * 4 + (e & 3)] : i;
+                            x[e] = e == dp ? top : 0.f;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            pe[e] = (wrow && e < dp) ? Pp[((e >> 2) * NP + i) * 4 + (e & 3)] : 0.f;
+#pragma unroll
+                            for (int f = e + 1; f < 9; ++f)
+                                co[f][e] = f <= dp ? Ap[((e >> 2) * NP + jf[f]) * 4 + (e & 3)] : 0.f;
+                        }
+#pragma unroll
+                        for (int e = 7; e >= 0; --e) {
+                            float acc = pe[e];
+#pragma unroll
+                            for (int f = e + 1; f < 9; ++f) acc = fmaf(-x[f], co[f][e], acc);
+                            x[e] = e < dp ? acc : x[e];
+                        }
+#pragma unroll
+                        for (int e = 0; e < 9; ++e) {
+                            if (e <= dp) {
+                                const int col = jf[e];
+                                const float hi = tf32_hi(x[e]);
+                                const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
+                                *reinterpret_cast<float *>(Mhi + off) = hi;
+                                *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
+                            }
+                        }
+                    } else {  // deep paths: the same recurrence through shared memory
+                        float *x = xr + (wrow ? i : NP + i) * C::XLD;
+                        x[dp] = top;
+                        for (int e = dp - 1; e >= 0; --e) {
+                            const int col_e = ((e >> 2) * NP) * 4 + (e & 3);
+                            float acc = wrow ? Pp[col_e + i * 4] : 0.f;
+                            for (int f = e + 1; f <= dp; ++f) {
+                                const int jf = (f == dp) ? i : idx[((f >> 2) * NP + i) * 4 + (f & 3)];
+                                acc = fmaf(-x[f], Ap[col_e + jf * 4], acc);
+                            }
+                            x[e] = acc;
+                        }
+                        for (int e = 0; e <= dp; ++e) {
+                            const int col = (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)];
+                            const float val = x[e], hi = tf32_hi(val);
+                            const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
+                            *reinterpret_cast<float *>(Mhi + off) = hi;
+                            *reinterpret_cast<float *>(Mlo + off) = val - hi;
+                        }
+                    }
+                }
+
+                // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo
+                float r[32];
+#pragma unroll
+                for (int c0 = 0; c0 < 32; c0 += 16) {
+                    if (c0 < NP && c0 < n) {
+                        uint32_t sk[16];
+                        ptx::tmem_ld16(tm + NP + c0, sk);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const int j = c0 + jj;
+                            const float4 sc = scal[j < NP ? j : 0];
+                            const float v = __bfloat162float(vs[(j < NP ? j : 0) * D + t]);
+                            const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v);
+                            r[j] = j < n ? val : 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) r[c0 + jj] = 0.f;
+                    }
+                }
+                {
+                    unsigned char *row_hi = stage + C::OFF_RT_HI + t * 128;
+                    unsigned char *row_lo = stage + C::OFF_RT_LO + t * 128;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float4 hi, lo;
+                        hi.x = tf32_hi(r[4 * q]), hi.y = tf32_hi(r[4 * q + 1]);
+                        hi.z = tf32_hi(r[4 * q + 2]), hi.w = tf32_hi(r[4 * q + 3]);
+                        lo.x = r[4 * q] - hi.x, lo.y = r[4 * q + 1] - hi.y;
+                        lo.z = r[4 * q + 2] - hi.z, lo.w = r[4 * q + 3] - hi.w;
+                        const int off = ((q ^ (t & 7)) << 4);
+                        *reinterpret_cast<float4 *>(row_hi + off) = hi;
+                        *reinterpret_cast<float4 *>(row_lo + off) = lo;
+                    }
+                }
+                ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
+            }
+            ptx::mbar_arrive(&ops_ready[buf]);
+            f_n = n, f_lo = lo;
+            }
+
+            if (b_kk >= 0) {
+            const int kk = b_kk, n = b_n, lo = b_lo;
+            const int item = blockIdx.x + kk * gridDim.x, h = item % a.H_v;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+            const float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;
+            if (!ptx::mbar_wait(&mma2_done[buf], (kk / C::TBUF) & 1)) {
+                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            if (n > 0) {
+                // ---- epilogue: u_i = DU[i], o_i = g_i (S0 q_i) + DO[i]
+                float *Ub = a.U + ((size_t)lo * a.H_v + h) * D + t;
+                TOut *Ob = Og + ((size_t)lo * a.H_v + h) * D + t;
+#pragma unroll
+                for (int c0 = 0; c0 < NP; c0 += 16) {
+                    if (c0 < n) {
+                        uint32_t du[16], dout[16], sq[16];
+                        ptx::tmem_ld16(tm + C::TM_DU + c0, du);
+                        ptx::tmem_ld16(tm + C::TM_DO + c0, dout);
+                        ptx::tmem_ld16(tm + c0, sq);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const int node = c0 + jj;
+                            const float o = fmaf(scal[node].z, __uint_as_float(sq[jj]), __uint_as_float(dout[jj]));
+                            st_global_if(Ub + node * rs, __uint_as_float(du[jj]), node < n);
+                            st_global_if(Ob + node * rs, o, node < n);
+                        }
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(&tmem_free[buf]);
+            }
+            if (!have) break;
+            b_kk = kk, b_n = f_n, b_lo = f_lo;
+        }
+    }
+
+    // common exit: tensor memory goes back once every role is done with it
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == C::MMA1_WARP) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, VT_TMEM_COLS);
+    }
+}
+
+namespace {
+
+template <int NP, typename TOut>
+cudaError_t launch_vt(const VerifyArgs &a, int T, cudaStream_t stream)
+{
+    using C = VtCfg<NP>;
+    const long long n_items = (long long)a.B * a.H_v;
+    VerifyMaps m;
+    if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_items, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(verify_sm100_tc_kernel<NP, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const int grid = (int)(n_items < sms ? n_items : sms);
+    verify_sm100_tc_kernel<NP, TOut><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, (int)n_items, m.S0, m.Q,
+                                                                                   m.K, m.V);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// bf16 inputs.  Trees of up to 32 nodes take the kernel above; larger ones the general variant.
+cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
+{
+    if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
+    if (a.max_nodes > 32) return launch_verify_sm100_simt(a, T, od, stream);
+    if (a.max_nodes <= 16) {
+        if (od == TREEWY_F32) return launch_vt<16, float>(a, T, stream);
+        return launch_vt<16, __nv_bfloat16>(a, T, stream);
+    }
+    if (od == TREEWY_F32) return launch_vt<32, float>(a, T, stream);
+    return launch_vt<32, __nv_bfloat16>(a, T, stream);
+}
+
+}  // namespace treewy
