@@ -44,41 +44,43 @@ constexpr uint32_t VT_TMEM_COLS = 512;
 template <int NP> struct VtCfg {
     static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
     static constexpr int GROUPS = 2;
-    static constexpr int STAGES = NP <= 16 ? 4 : 3;
+    static constexpr int STAGES = 4;
     static constexpr int TBUF = 5;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
     static constexpr int CONSUMERS = VT_GROUP * GROUPS;
     static constexpr int MMA1_WARP = CONSUMERS / 32;
     static constexpr int MMA2_WARP = MMA1_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
     static constexpr int THREADS = CONSUMERS + 64 + 32 * STAGES;
-    // stage: [Q;K] tile | S0 tile | V rows | meta
+    // stage: [Q;K] tile | S0 tile | meta   (the v rows arrive later, into the dead S0 tile)
     static constexpr int QK_HALF = 2 * NP * 128;
     static constexpr int QK_BYTES = 2 * QK_HALF;
     static constexpr int S0_HALF = D * 128;
     static constexpr int S0_BYTES = 2 * S0_HALF;
-    static constexpr int V_BYTES = NP * D * 2;
     static constexpr int OFF_S0 = QK_BYTES;
-    static constexpr int OFF_V = OFF_S0 + S0_BYTES;
-    static constexpr int OFF_META = OFF_V + V_BYTES;
+    static constexpr int OFF_META = OFF_S0 + S0_BYTES;
     static constexpr int META_BYTES = NP * 16 + 16;  // mask u64, L f32, beta f32 per node; n, lo
     static constexpr int STAGE_BYTES = (OFF_META + META_BYTES + 1023) / 1024 * 1024;
     // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
     static constexpr int OFF_T_HI = 0, OFF_T_LO = NP * 128, OFF_W_HI = 2 * NP * 128, OFF_W_LO = 3 * NP * 128;
     static constexpr int OFF_RT_HI = OFF_S0, OFF_RT_LO = OFF_S0 + D * 128;
     static_assert(4 * NP * 128 <= QK_BYTES && 2 * D * 128 <= S0_BYTES, "operand overlays fit");
-    // group-private: path lists, per-node scalars, back-substitution rows
-    static constexpr int XLD = NP + 1;
-    static constexpr int GP_AP = 0, GP_PP = NP * NP * 4, GP_SCAL = 2 * NP * NP * 4;
-    static constexpr int GP_XR = GP_SCAL + 2 * NP * 16;  // per-node scalars are double-buffered
-    static constexpr int GP_IDX = GP_XR + 2 * NP * XLD * 4;
+    // scratch over the dead S0 tile, used before R^T is written there: the raw Gram rows and the
+    // back-substitution rows of deep paths
     static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
-    static constexpr int GP_RAW = (GP_IDX + NP * NP + 15) / 16 * 16;
-    static constexpr int GP_BYTES = GP_RAW + 2 * NP * RLD * 4;
+    static constexpr int XLD = NP + 1;
+    static constexpr int OFF_RAW = OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;
+    static constexpr int OFF_VS = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 127) / 128 * 128;  // v rows [NP][128] bf16
+    static constexpr int V_BYTES = NP * D * 2;
+    static_assert(OFF_VS + V_BYTES <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
+    // group-private: path lists, per-node scalars (double-buffered), ancestor indices
+    static constexpr int GP_AP = 0, GP_PP = NP * NP * 4, GP_SCAL = 2 * NP * NP * 4;
+    static constexpr int GP_IDX = GP_SCAL + 2 * NP * 16;
+    static constexpr int GP_BYTES = (GP_IDX + NP * NP + 15) / 16 * 16;
     static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 4 * TBUF) * 8 + 16 + 1024;
-    static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES + V_BYTES;
+    static constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 4 * TBUF + GROUPS) * 8 + 16 + 1024;
+    static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // per TMEM buffer: SQ | SK | D2; stage 2 writes DO over SK and DU over D2 (both dead by then)
     static constexpr int TM_COLS = 3 * NP;
     static constexpr int TM_DO = NP, TM_DU = 2 * NP;
@@ -131,7 +133,8 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
     uint64_t *ops_ready = mma1_done + C::TBUF;
     uint64_t *mma2_done = ops_ready + C::TBUF;
     uint64_t *tmem_free = mma2_done + C::TBUF;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tmem_free + C::TBUF);
+    uint64_t *v_ready = tmem_free + C::TBUF;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(v_ready + C::GROUPS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -146,6 +149,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             ptx::mbar_init(&mma2_done[i], 1);
             ptx::mbar_init(&tmem_free[i], VT_GROUP);
         }
+        for (int g = 0; g < C::GROUPS; ++g) ptx::mbar_init(&v_ready[g], 1);
         ptx::fence_barrier_init();
     }
     if (warp == C::MMA1_WARP) {
@@ -168,7 +172,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
         unsigned char *stage = smem + s * C::STAGE_BYTES;
         if (lane == 0) {
             ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ);
-            ptx::prefetch_tmap(&tmK), ptx::prefetch_tmap(&tmV);
+            ptx::prefetch_tmap(&tmK);
         }
         const int group = a.H_v / a.H_qk;
         // Node scalars of an item: validated and loaded one round ahead (software pipeline), so the
@@ -222,7 +226,6 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                     ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
                     ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
                     ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
-                    ptx::tma_load_2d(stage + C::OFF_V, &tmV, p.h * D, p.lo, &full[s]);
                 }
             }
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
@@ -312,9 +315,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
         float *Ap = reinterpret_cast<float *>(gp + C::GP_AP);
         float *Pp = reinterpret_cast<float *>(gp + C::GP_PP);
         float4 *scal2 = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
-        float *xr = reinterpret_cast<float *>(gp + C::GP_XR);
         unsigned char *idx = gp + C::GP_IDX;
-        float *raw = reinterpret_cast<float *>(gp + C::GP_RAW);
         TOut *Og = static_cast<TOut *>(a.O);
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
@@ -341,11 +342,21 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
             const int n = meta_nlo(stage)[0];
             const int lo = meta_nlo(stage)[1];
-            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK | D2 | DU | DO
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK | D2 (DO over SK, DU over D2)
+            if (t == 0) {  // the v rows of this item go to a free corner of the dead S0 tile
+                if (n > 0) {
+                    ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
+                    ptx::tma_load_2d(stage + C::OFF_VS, &tmV, (item % a.H_v) * D, lo, &v_ready[grp]);
+                } else {
+                    ptx::mbar_arrive(&v_ready[grp]);
+                }
+            }
             if (n > 0) {
                 const unsigned long long *mask = meta_mask(stage);
                 const float *Lm = meta_L(stage);
-                const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_V);
+                float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
+                float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
+                const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_VS);
 
                 // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
                 for (int q = t; q < 4 * NP * 128 / 16; q += VT_GROUP)
@@ -402,7 +413,8 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                         scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
                     }
                 }
-                ptx::named_sync(1 + grp, VT_GROUP);  // lists, scalars and the zero fill are in place
+                // lists, scalars and the zero fill are in place; learn whether any path is deep
+                const bool deep = ptx::named_sync_or(1 + grp, VT_GROUP, dp > 8);
 
                 // ---- phase T: rows of T = (I + A)^-1 (one thread) and W = P T (another) by
                 // back-substitution along node i's root path j_0 .. j_{dp-1}, j_dp = i:
@@ -412,7 +424,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
-                    if (dp <= 8) {  // registers only, every load issued up front
+                    if (!deep) {  // registers only, every load issued up front
                         int jf[9];
                         float x[9], pe[8], co[9][8];
 #pragma unroll
@@ -466,6 +478,13 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                     }
                 }
 
+                // this thread's column of the v rows leaves the S0 tile before R^T lands on it
+                ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);
+                __nv_bfloat16 vreg[NP];
+#pragma unroll
+                for (int j = 0; j < NP; ++j) vreg[j] = vs[j * D + t];
+                ptx::named_sync(1 + grp, VT_GROUP);
+
                 // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo
                 float r[32];
 #pragma unroll
@@ -478,7 +497,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                         for (int jj = 0; jj < 16; ++jj) {
                             const int j = c0 + jj;
                             const float4 sc = scal[j < NP ? j : 0];
-                            const float v = __bfloat162float(vs[(j < NP ? j : 0) * D + t]);
+                            const float v = __bfloat162float(vreg[j < NP ? j : 0]);
                             const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v);
                             r[j] = j < n ? val : 0.f;
                         }
