@@ -163,10 +163,38 @@ def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Te
 
 # --------------------------------------------------------------------------- user-level step
 
+class _StepBuffers:
+    """Device-side inputs and outputs of one in-flight step."""
+
+    def __init__(self, B, H_v, H_qk, max_T, io, o_dtype, dev):
+        z = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        self.q, self.k = z((max_T, H_qk, D), io), z((max_T, H_qk, D), io)
+        self.v = z((max_T, H_v, D), io)
+        self.alpha, self.beta = z((max_T, H_v), torch.float32), z((max_T, H_v), torch.float32)
+        self.node_offsets = z((B + 1,), torch.int32)
+        self.parent = z((max_T,), torch.int32)
+        self.accepted = z((B,), torch.int32)
+        self.O = z((max_T, H_v, D), o_dtype)
+        self.U = z((max_T, H_v, D), torch.float32)
+        self.depth = z((max_T,), torch.int32)
+        self.anc_mask = z((max_T,), torch.int64)
+        self.cum_log_gate = z((max_T, H_v), torch.float32)
+        self.level_order = z((max_T,), torch.uint8)
+        self.uploaded = torch.cuda.Event()
+        self.verified = torch.cuda.Event()
+        self.computed = torch.cuda.Event()
+        self.downloaded = torch.cuda.Event()
+
+
 class VerifyCommitLayer:
     """One GDN layer's speculative state on a device: the committed state lives in HBM across
     steps; each step uploads the draft window's inputs, verifies, returns the outputs to the
-    host, and commits the accepted node.  This is the call a serving loop makes."""
+    host, and commits the accepted node.  This is the call a serving loop makes.
+
+    ``step`` runs everything on the current stream.  ``step_async`` pipelines consecutive steps
+    over three streams (upload / compute / download) with double-buffered inputs and outputs:
+    the upload of step i+1 and the download of step i overlap the kernels, which stay in order
+    because every step reads and writes the same committed state."""
 
     def __init__(self, S0: torch.Tensor, H_qk: int, max_T: int, max_nodes: int = 0,
                  o_dtype: torch.dtype | None = None):
@@ -174,50 +202,63 @@ class VerifyCommitLayer:
         self.S0 = S0
         self.B, self.H_v = int(S0.shape[0]), int(S0.shape[1])
         self.H_qk, self.max_nodes = H_qk, max_nodes
-        io = S0.dtype
-        o_dtype = o_dtype or io
-        z = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
-        self.q, self.k = z((max_T, H_qk, D), io), z((max_T, H_qk, D), io)
-        self.v = z((max_T, self.H_v, D), io)
-        self.alpha, self.beta = z((max_T, self.H_v), torch.float32), z((max_T, self.H_v), torch.float32)
-        self.node_offsets = z((self.B + 1,), torch.int32)
-        self.parent = z((max_T,), torch.int32)
-        self.accepted = z((self.B,), torch.int32)
-        self.O = z((max_T, self.H_v, D), o_dtype)
-        self.U = z((max_T, self.H_v, D), torch.float32)
+        o_dtype = o_dtype or S0.dtype
+        self.bufs = [_StepBuffers(self.B, self.H_v, H_qk, max_T, S0.dtype, o_dtype, dev)
+                     for _ in range(2)]
         self.status = torch.zeros((self.B,), dtype=torch.int32, device=dev)
-        self.depth = z((max_T,), torch.int32)
-        self.anc_mask = z((max_T,), torch.int64)
-        self.cum_log_gate = z((max_T, self.H_v), torch.float32)
-        self.level_order = z((max_T,), torch.uint8)
+        self.s_up, self.s_run, self.s_down = (torch.cuda.Stream(dev) for _ in range(3))
+        self._n = 0
 
-    def tree(self, T: int) -> Tree:
-        return Tree(self.B, T, self.H_v, self.max_nodes, self.node_offsets, self.parent,
-                    self.depth, self.anc_mask, self.cum_log_gate, self.level_order)
+    @property
+    def O(self) -> torch.Tensor:
+        return self.bufs[0].O
 
-    def upload(self, host: dict) -> int:
-        """Host (pinned) tensors -> device buffers on the current stream; returns T."""
+    def _tree(self, b: _StepBuffers, T: int) -> Tree:
+        return Tree(self.B, T, self.H_v, self.max_nodes, b.node_offsets, b.parent, b.depth,
+                    b.anc_mask, b.cum_log_gate, b.level_order)
+
+    @staticmethod
+    def _upload(b: _StepBuffers, host: dict) -> int:
         T = int(host["parent"].numel())
         for name in ("q", "k", "v", "alpha", "beta", "parent"):
-            getattr(self, name)[:T].copy_(host[name], non_blocking=True)
-        self.node_offsets.copy_(host["node_offsets"], non_blocking=True)
+            getattr(b, name)[:T].copy_(host[name], non_blocking=True)
+        b.node_offsets.copy_(host["node_offsets"], non_blocking=True)
+        b.accepted.copy_(host["accepted"], non_blocking=True)
         return T
 
-    def verify(self, T: int) -> None:
-        tree = self.tree(T)
-        treewy_tree_prepare(tree, self.alpha, self.status)
-        treewy_verify(self.S0, self.q, self.k, self.v, self.beta, tree, self.H_qk, self.O, self.U,
-                      self.status)
-
-    def commit(self, T: int, accepted_host: torch.Tensor | None = None) -> None:
-        if accepted_host is not None:
-            self.accepted.copy_(accepted_host, non_blocking=True)
-        treewy_commit(self.S0, self.U, self.k, self.tree(T), self.H_qk, self.accepted, None,
-                      self.status)
+    def _run(self, b: _StepBuffers, T: int, stream=None) -> None:
+        tree = self._tree(b, T)
+        treewy_tree_prepare(tree, b.alpha, self.status, stream)
+        treewy_verify(self.S0, b.q, b.k, b.v, b.beta, tree, self.H_qk, b.O, b.U, self.status, stream)
+        b.verified.record(stream)
+        treewy_commit(self.S0, b.U, b.k, tree, self.H_qk, b.accepted, None, self.status, stream)
 
     def step(self, host: dict, O_host: torch.Tensor) -> None:
         """upload -> prepare -> verify -> outputs to host -> commit, all on the current stream."""
-        T = self.upload(host)
-        self.verify(T)
-        O_host[:T].copy_(self.O[:T], non_blocking=True)
-        self.commit(T, host["accepted"])
+        b = self.bufs[0]
+        T = self._upload(b, host)
+        self._run(b, T, torch.cuda.current_stream())
+        O_host[:T].copy_(b.O[:T], non_blocking=True)
+
+    def step_async(self, host: dict, O_host: torch.Tensor) -> None:
+        """Enqueue one step; returns at once.  ``host`` and ``O_host`` must be pinned and must not
+        be reused before the second-next ``step_async`` (or ``synchronize``)."""
+        b = self.bufs[self._n & 1]
+        self._n += 1
+        with torch.cuda.stream(self.s_up):
+            self.s_up.wait_event(b.computed)     # the kernels that last read this buffer set
+            T = self._upload(b, host)
+            b.uploaded.record(self.s_up)
+        with torch.cuda.stream(self.s_run):
+            self.s_run.wait_event(b.uploaded)
+            self.s_run.wait_event(b.downloaded)  # O of this buffer set has left for the host
+            self._run(b, T, self.s_run)
+            b.computed.record(self.s_run)
+        with torch.cuda.stream(self.s_down):
+            self.s_down.wait_event(b.verified)
+            O_host[:T].copy_(b.O[:T], non_blocking=True)
+            b.downloaded.record(self.s_down)
+
+    def synchronize(self) -> None:
+        for s in (self.s_up, self.s_run, self.s_down):
+            s.synchronize()
