@@ -21,17 +21,21 @@ SMALL = {  # config id -> overrides that keep the structure but shrink the batch
 }
 
 
-@pytest.mark.parametrize("generic", [True, False])
+# "generic": fp32 SIMT kernel; "general": tensor-core kernel for up to 64 nodes (no size hint);
+# "hinted": the caller states max_nodes, so trees of up to 32 nodes take the tensor-core solve
+@pytest.mark.parametrize("path", ["generic", "general", "hinted"])
 @pytest.mark.parametrize("cid", sorted(SMALL))
-def test_configs_match_oracle(oracle, cid, generic):
+def test_configs_match_oracle(oracle, cid, path):
     w = wl.make_workload(cid, **SMALL[cid])
+    generic = path == "generic"
+    hint = w.max_nodes if path == "hinted" else 0
     tree_ref, ref = pu.run_oracle(oracle, w)
-    gpu = pu.run_gpu(w, torch.float32, generic=generic)
+    gpu = pu.run_gpu(w, torch.float32, generic=generic, max_nodes=hint)
     assert not gpu["status"].any()
     errs = pu.assert_parity(w, gpu, tree_ref, ref)
-    print(f"config {cid} generic={generic}: worst (max-abs/rms, rel-fro) {errs}")
+    print(f"config {cid} path={path}: worst (max-abs/rms, rel-fro) {errs}")
     if w.io_dtype == torch.bfloat16:
-        gpu16 = pu.run_gpu(w, torch.bfloat16, generic=generic)
+        gpu16 = pu.run_gpu(w, torch.bfloat16, generic=generic, max_nodes=hint)
         got, floor = pu.assert_bf16_outputs(w, gpu16, gpu, ref)
         print(f"   bf16 O: {got} against rounding floor {floor}")
         assert torch.equal(gpu16["S"], gpu["S"])
@@ -151,3 +155,36 @@ def test_metamorphic_commit_then_verify_on_gpu(oracle):
     second = pu.run_gpu(w2, torch.float32)
     torch.testing.assert_close(second["O"], first["O"][idx], rtol=0, atol=2e-5)
     torch.testing.assert_close(second["U"], first["U"][idx], rtol=0, atol=2e-5)
+
+
+@pytest.mark.parametrize("hint", [16, 32])
+def test_small_trees_through_the_tensor_core_solve(oracle, hint):
+    """Shapes that stress the up-to-32-node kernel: full chains (paths deeper than the eight
+    ancestors its register path handles), stars, forests, single nodes, mixed in one batch."""
+    n = hint
+    chain = [i - 1 for i in range(n)]
+    star = [-1] + [0] * (n - 1)
+    forest = [-1, -1, 0, 1, -1, 4, 5]
+    comb = [-1] + [max(0, i - 2) for i in range(1, n)]          # depth ~ n/2
+    trees = [chain, star, forest, [-1], [-1, 0], comb, chain[:9], chain[:10]]
+    w = _custom(trees, H_v=4, H_qk=2, accepted=[n - 1, 3, 6, 0, -1, n - 1, 8, 9])
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    gpu = pu.run_gpu(w, torch.float32, max_nodes=hint)
+    assert not gpu["status"].any()
+    pu.assert_parity(w, gpu, tree_ref, ref)
+    gpu16 = pu.run_gpu(w, torch.bfloat16, max_nodes=hint)
+    assert torch.equal(gpu16["O"], gpu["O"].to(torch.bfloat16)) and torch.equal(gpu16["U"], gpu["U"])
+
+
+def test_malformed_sequences_in_the_tensor_core_solve(oracle):
+    from paper_2608_20961_b200 import binding as tw
+    good = [-1, 0, 0, 2]
+    trees = [good, [-1, 2, 0], good, [i - 1 for i in range(20)]]
+    w = _custom(trees, H_v=2, H_qk=2, accepted=[3, 1, 9, 1])
+    gpu = pu.run_gpu(w, torch.float32, max_nodes=16)
+    assert list(gpu["status"]) == [0, tw.SEQ_BAD_PARENT, tw.SEQ_BAD_ACCEPTED, tw.SEQ_TOO_MANY_NODES]
+    tree_ref, ref = pu.run_oracle(oracle, w.select_sequences([0]))
+    off = w.node_offsets.tolist()
+    np.testing.assert_allclose(gpu["O"][:4].double().numpy(), ref.O, atol=1e-4)
+    assert torch.all(gpu["O"][off[1]:off[2]] == gpu["canary"])
+    assert torch.all(gpu["U"][off[3]:off[4]] == gpu["canary"])
