@@ -51,6 +51,7 @@ treewy_status_t verify_common(bool force_generic, const void *S0, const void *q,
     a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.cls_lo = 0, a.cls_hi = max_nodes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
     if (io_dtype == TREEWY_BF16 && !force_generic)

@@ -20,6 +20,9 @@ struct VerifyArgs {
     float *U;
     int32_t *seq_status;
     int B, H_v, H_qk, max_nodes;
+    // size class of this launch: sequences with cls_lo < N_b <= cls_hi are processed, the others are
+    // left to the launch of their class (N_b outside 1..max_nodes is flagged where cls_lo == 0)
+    int cls_lo, cls_hi;
 };
 
 struct CommitArgs {

@@ -157,8 +157,13 @@ verify_sm100_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorM
             const int lo = a.node_offsets[b];
             const int n = a.node_offsets[b + 1] - lo;
             int bad = 0;
-            if (n < 1 || n > a.max_nodes || n > NP) {
+            bool other_class = false;  // handled by another launch: skipped here without a flag
+            if (n < 1 || n > a.max_nodes) {
                 bad = TREEWY_SEQ_TOO_MANY_NODES;
+                other_class = a.cls_lo != 0;
+            } else if (n <= a.cls_lo || n > a.cls_hi || n > NP) {
+                bad = TREEWY_SEQ_TOO_MANY_NODES;
+                other_class = true;
             } else {
                 int bp = 0;
                 for (int i = lane; i < n; i += 32) {
@@ -167,7 +172,7 @@ verify_sm100_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorM
                 }
                 if (__any_sync(0xffffffffu, bp)) bad = TREEWY_SEQ_BAD_PARENT;
             }
-            if (bad && h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
+            if (bad && !other_class && h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
             // node scalars: issued before the wait so their latency hides under it
             constexpr int R = (NP + 4 + 31) / 32;
             unsigned long long mk[R];
@@ -453,10 +458,6 @@ cudaError_t launch_vs(const VerifyArgs &a, int T, cudaStream_t stream)
 // general variant: any tree of up to 64 nodes; the solve runs on the CUDA cores
 cudaError_t launch_verify_sm100_simt(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
 {
-    if (a.max_nodes <= 32) {
-        if (od == TREEWY_F32) return launch_vs<32, float>(a, T, stream);
-        return launch_vs<32, __nv_bfloat16>(a, T, stream);
-    }
     if (od == TREEWY_F32) return launch_vs<64, float>(a, T, stream);
     return launch_vs<64, __nv_bfloat16>(a, T, stream);
 }

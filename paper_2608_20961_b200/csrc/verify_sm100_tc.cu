@@ -178,20 +178,24 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
         // Node scalars of an item: validated and loaded one round ahead (software pipeline), so the
         // dependent chain  node_offsets -> parent / mask / log-gate / beta  never delays a TMA issue.
         struct Pre {
-            int item, b, h, lo, n, bad;
+            int item, b, h, lo, n, bad, flag;
             unsigned long long mk;
             float Lv, bv;
         };
         auto fetch = [&](int kk) {
             Pre p;
             p.item = blockIdx.x + kk * gridDim.x;
-            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
+            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
             if (p.item >= n_items) return p;
             p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
             p.lo = a.node_offsets[p.b];
             p.n = a.node_offsets[p.b + 1] - p.lo;
-            if (p.n < 1 || p.n > a.max_nodes || p.n > NP) {
+            if (p.n < 1 || p.n > a.max_nodes) {
                 p.bad = TREEWY_SEQ_TOO_MANY_NODES;
+                p.flag = a.cls_lo == 0;
+            } else if (p.n <= a.cls_lo || p.n > a.cls_hi || p.n > NP) {
+                p.bad = TREEWY_SEQ_TOO_MANY_NODES;  // another launch's size class: skipped, not flagged
+                p.flag = 0;
             } else {
                 const int par = lane < p.n ? a.parent[p.lo + lane] : -1;
                 if (__any_sync(0xffffffffu, lane < p.n && (par < -1 || par >= lane))) p.bad = TREEWY_SEQ_BAD_PARENT;
@@ -206,7 +210,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
         for (int kk = s;; kk += C::STAGES) {
             if (cur.item >= n_items) break;
             const Pre p = cur;
-            if (p.bad && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
+            if (p.bad && p.flag && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
             if (!ptx::mbar_wait(&empty[s], ((kk / C::STAGES) & 1) ^ 1)) {
                 if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], TREEWY_SEQ_TIMEOUT);
                 break;
@@ -602,17 +606,22 @@ cudaError_t launch_vt(const VerifyArgs &a, int T, cudaStream_t stream)
 
 }  // namespace
 
-// bf16 inputs.  Trees of up to 32 nodes take the kernel above; larger ones the general variant.
+// bf16 inputs.  Sequences of up to 32 nodes take the kernel above, larger ones the general variant;
+// a batch that may hold both (max_nodes > 32) gets one launch per size class.
 cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
 {
     if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
-    if (a.max_nodes > 32) return launch_verify_sm100_simt(a, T, od, stream);
-    if (a.max_nodes <= 16) {
-        if (od == TREEWY_F32) return launch_vt<16, float>(a, T, stream);
-        return launch_vt<16, __nv_bfloat16>(a, T, stream);
-    }
-    if (od == TREEWY_F32) return launch_vt<32, float>(a, T, stream);
-    return launch_vt<32, __nv_bfloat16>(a, T, stream);
+    VerifyArgs small = a;
+    small.cls_lo = 0, small.cls_hi = a.max_nodes < 32 ? a.max_nodes : 32;
+    cudaError_t e;
+    if (a.max_nodes <= 16)
+        e = od == TREEWY_F32 ? launch_vt<16, float>(small, T, stream) : launch_vt<16, __nv_bfloat16>(small, T, stream);
+    else
+        e = od == TREEWY_F32 ? launch_vt<32, float>(small, T, stream) : launch_vt<32, __nv_bfloat16>(small, T, stream);
+    if (e != cudaSuccess || a.max_nodes <= 32) return e;
+    VerifyArgs large = a;
+    large.cls_lo = 32, large.cls_hi = a.max_nodes;
+    return launch_verify_sm100_simt(large, T, od, stream);
 }
 
 }  // namespace treewy
