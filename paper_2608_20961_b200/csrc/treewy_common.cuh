@@ -61,6 +61,19 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
+// stores that are predicated instead of branched around (keeps the epilogue one straight line)
+__device__ __forceinline__ void st_global_if(float *p, float v, bool on)
+{
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v),
+                 "r"((int)on));
+}
+__device__ __forceinline__ void st_global_if(__nv_bfloat16 *p, float v, bool on)
+{
+    const unsigned short b = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.b16 [%0], %1;\n\t}" ::"l"(p), "h"(b),
+                 "r"((int)on));
+}
+
 // Status bits of sequence [lo, lo+n): node count in 1..max_nodes, parent[i] in -1..i-1.
 // Called by every thread of a CTA with the same arguments; `scratch` is one shared int the
 // caller zeroed before a barrier.  Returns the same value in every thread.

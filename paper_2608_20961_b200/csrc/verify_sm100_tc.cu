@@ -87,37 +87,6 @@ template <int NP> struct VtCfg {
     static_assert(TBUF * TM_COLS <= 512, "tensor memory");
 };
 
-// instruction descriptor, kind::tf32: tf32 x tf32 -> fp32, both operands K-major, dense
-__host__ __device__ constexpr uint32_t umma_idesc_tf32_f32(int M, int N)
-{
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// stores that are predicated instead of branched around (keeps the epilogue one straight line)
-__device__ __forceinline__ void st_global_if(float *p, float v, bool on)
-{
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v),
-                 "r"((int)on));
-}
-__device__ __forceinline__ void st_global_if(__nv_bfloat16 *p, float v, bool on)
-{
-    const unsigned short b = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.b16 [%0], %1;\n\t}" ::"l"(p), "h"(b),
-                 "r"((int)on));
-}
-
-__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
-
 template <int NP, typename TOut>
 __global__ void __launch_bounds__(VtCfg<NP>::THREADS, 1)
 verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorMap tmS0,
@@ -274,7 +243,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
         }
     } else if (warp == C::MMA2_WARP) {
         // ------------------------------------------------------------------ stage-2 MMAs
-        constexpr uint32_t idesc = umma_idesc_tf32_f32(128, NP);
+        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, NP);
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -295,13 +264,13 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                     for (int p = 0; p < 3; ++p)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            umma_tf32(dU, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
+                            ptx::umma_tf32(dU, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
                                       ptx::umma_desc_k_sw128(tt[p] + ks * 32), idesc, (p | ks) != 0);
 #pragma unroll
                     for (int p = 0; p < 3; ++p)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            umma_tf32(dO, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
+                            ptx::umma_tf32(dO, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
                                       ptx::umma_desc_k_sw128(ww[p] + ks * 32), idesc, (p | ks) != 0);
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
@@ -454,7 +423,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                         for (int e = 0; e < 9; ++e) {
                             if (e <= dp) {
                                 const int col = jf[e];
-                                const float hi = tf32_hi(x[e]);
+                                const float hi = ptx::tf32_hi(x[e]);
                                 const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
                                 *reinterpret_cast<float *>(Mhi + off) = hi;
                                 *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
@@ -474,7 +443,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                         }
                         for (int e = 0; e <= dp; ++e) {
                             const int col = (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)];
-                            const float val = x[e], hi = tf32_hi(val);
+                            const float val = x[e], hi = ptx::tf32_hi(val);
                             const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
                             *reinterpret_cast<float *>(Mhi + off) = hi;
                             *reinterpret_cast<float *>(Mlo + off) = val - hi;
@@ -516,8 +485,8 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         float4 hi, lo;
-                        hi.x = tf32_hi(r[4 * q]), hi.y = tf32_hi(r[4 * q + 1]);
-                        hi.z = tf32_hi(r[4 * q + 2]), hi.w = tf32_hi(r[4 * q + 3]);
+                        hi.x = ptx::tf32_hi(r[4 * q]), hi.y = ptx::tf32_hi(r[4 * q + 1]);
+                        hi.z = ptx::tf32_hi(r[4 * q + 2]), hi.w = ptx::tf32_hi(r[4 * q + 3]);
                         lo.x = r[4 * q] - hi.x, lo.y = r[4 * q + 1] - hi.y;
                         lo.z = r[4 * q + 2] - hi.z, lo.w = r[4 * q + 3] - hi.w;
                         const int off = ((q ^ (t & 7)) << 4);
@@ -621,7 +590,7 @@ cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, c
     if (e != cudaSuccess || a.max_nodes <= 32) return e;
     VerifyArgs large = a;
     large.cls_lo = 32, large.cls_hi = a.max_nodes;
-    return launch_verify_sm100_simt(large, T, od, stream);
+    return launch_verify_sm100_tc64(large, T, od, stream);
 }
 
 }  // namespace treewy
