@@ -397,20 +397,26 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
-                    if (!deep) {  // registers only, every load issued up front
+                    if (!deep) {  // registers only; every load is unconditional (all addresses are valid)
+                                  // and masked by a select, so the phase has no branches
                         int jf[9];
                         float x[9], pe[8], co[9][8];
 #pragma unroll
                         for (int e = 0; e < 9; ++e) {
-                            jf[e] = e < dp ? idx[((e >> 2) * NP + i) * 4 + (e & 3)] : i;
+                            const int ee = e < 8 ? e : 7;
+                            const int j = idx[((ee >> 2) * NP + i) * 4 + (ee & 3)];
+                            jf[e] = e < dp ? j : i;
                             x[e] = e == dp ? top : 0.f;
                         }
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            pe[e] = (wrow && e < dp) ? Pp[((e >> 2) * NP + i) * 4 + (e & 3)] : 0.f;
+                            const float pv = Pp[((e >> 2) * NP + i) * 4 + (e & 3)];
+                            pe[e] = (wrow && e < dp) ? pv : 0.f;
 #pragma unroll
-                            for (int f = e + 1; f < 9; ++f)
-                                co[f][e] = f <= dp ? Ap[((e >> 2) * NP + jf[f]) * 4 + (e & 3)] : 0.f;
+                            for (int f = e + 1; f < 9; ++f) {
+                                const float cv = Ap[((e >> 2) * NP + jf[f]) * 4 + (e & 3)];
+                                co[f][e] = f <= dp ? cv : 0.f;
+                            }
                         }
 #pragma unroll
                         for (int e = 7; e >= 0; --e) {
@@ -419,15 +425,15 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
                             for (int f = e + 1; f < 9; ++f) acc = fmaf(-x[f], co[f][e], acc);
                             x[e] = e < dp ? acc : x[e];
                         }
+                        // entries beyond the path all aim at the diagonal and carry 0; going down from
+                        // e = 8 the real diagonal entry (e = dp) is written after them
 #pragma unroll
-                        for (int e = 0; e < 9; ++e) {
-                            if (e <= dp) {
-                                const int col = jf[e];
-                                const float hi = ptx::tf32_hi(x[e]);
-                                const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
-                                *reinterpret_cast<float *>(Mhi + off) = hi;
-                                *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
-                            }
+                        for (int e = 8; e >= 0; --e) {
+                            const int col = jf[e];
+                            const float hi = ptx::tf32_hi(x[e]);
+                            const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
+                            *reinterpret_cast<float *>(Mhi + off) = hi;
+                            *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
                         }
                     } else {  // deep paths: the same recurrence through shared memory
                         float *x = xr + (wrow ? i : NP + i) * C::XLD;

@@ -367,23 +367,29 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                         unsigned char *Mlo = stage + (wrow ? V6_OFF_W_LO : V6_OFF_T_LO);
 #pragma unroll
                         for (int q = 0; q < 16; ++q) {  // the row starts as zeros
-                            const int off = (q >> 3) * V6_ATOM + i * 128 + (q & 7) * 16;
+                            const int off = (q >> 3) * V6_ATOM + i * 128 + (((q & 7) ^ (i & 7)) << 4);  // bank-conflict free
                             *reinterpret_cast<uint4 *>(Mhi + off) = make_uint4(0u, 0u, 0u, 0u);
                             *reinterpret_cast<uint4 *>(Mlo + off) = make_uint4(0u, 0u, 0u, 0u);
                         }
-                        if (!deep) {  // registers only, every load issued up front
+                        if (!deep) {  // registers only; every load is unconditional (all addresses are
+                                      // valid) and masked by a select, so the phase has no branches
                             int jf[9];
                             float x[9], pe[8], co[9][8];
 #pragma unroll
                             for (int e = 0; e < 9; ++e) {
-                                jf[e] = e < dp ? idx[v6_at(i, e)] : i;
+                                const int j = idx[v6_at(i, e < 8 ? e : 7)];
+                                jf[e] = e < dp ? j : i;
                                 x[e] = e == dp ? top : 0.f;
                             }
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
-                                pe[e] = (wrow && e < dp) ? Pp[v6_at(i, e)] : 0.f;
+                                const float pv = Pp[v6_at(i, e)];
+                                pe[e] = (wrow && e < dp) ? pv : 0.f;
 #pragma unroll
-                                for (int f = e + 1; f < 9; ++f) co[f][e] = f <= dp ? Ap[v6_at(jf[f], e)] : 0.f;
+                                for (int f = e + 1; f < 9; ++f) {
+                                    const float cv = Ap[v6_at(jf[f], e)];
+                                    co[f][e] = f <= dp ? cv : 0.f;
+                                }
                             }
 #pragma unroll
                             for (int e = 7; e >= 0; --e) {
@@ -392,14 +398,14 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                                 for (int f = e + 1; f < 9; ++f) acc = fmaf(-x[f], co[f][e], acc);
                                 x[e] = e < dp ? acc : x[e];
                             }
+                            // entries beyond the path all aim at the diagonal and carry 0; going down
+                            // from e = 8 the real diagonal entry (e = dp) is written after them
 #pragma unroll
-                            for (int e = 0; e < 9; ++e) {
-                                if (e <= dp) {
-                                    const float hi = ptx::tf32_hi(x[e]);
-                                    const int off = v6_tile_off(i, jf[e]);
-                                    *reinterpret_cast<float *>(Mhi + off) = hi;
-                                    *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
-                                }
+                            for (int e = 8; e >= 0; --e) {
+                                const float hi = ptx::tf32_hi(x[e]);
+                                const int off = v6_tile_off(i, jf[e]);
+                                *reinterpret_cast<float *>(Mhi + off) = hi;
+                                *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
                             }
                         } else {  // deep paths: x_e is kept in the hi tile at its final column
                             *reinterpret_cast<float *>(Mhi + v6_tile_off(i, i)) = top;
