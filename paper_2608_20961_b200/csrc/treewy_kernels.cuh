@@ -45,7 +45,6 @@ cudaError_t launch_verify_generic(const VerifyArgs &a, treewy_dtype_t io, treewy
 // bf16 inputs: TMA + tcgen05 kernel; T = packed node count (bounds the q/k/v tensor maps)
 cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
 cudaError_t launch_verify_sm100_tc64(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
-cudaError_t launch_verify_sm100_simt(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
 cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
 cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream);  // bf16 state
 

@@ -342,12 +342,21 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                         const float scale = a_kind ? bi : 1.f;
                         const float *row = raw + t * V6_RLD;
                         unsigned long long m = mi & ~(1ull << i);
-                        for (int d = 0; d < dp; ++d) {
-                            const int j = __ffsll((long long)m) - 1;
+                        for (int d = 0; d < dp; d += 2) {  // two ancestors per round: independent chains
+                            const int j0 = __ffsll((long long)m) - 1;
                             m &= m - 1;
-                            const float val = scale * __expf(Li - Lm[j]) * row[j];
-                            if (a_kind) Ap[v6_at(i, d)] = val;
-                            else Pp[v6_at(i, d)] = val, idx[v6_at(i, d)] = (unsigned char)j;
+                            const bool two = d + 1 < dp;
+                            const int j1 = two ? __ffsll((long long)m) - 1 : j0;
+                            m &= m - 1;
+                            const float v0 = scale * __expf(Li - Lm[j0]) * row[j0];
+                            const float v1 = scale * __expf(Li - Lm[j1]) * row[j1];
+                            if (a_kind) {
+                                Ap[v6_at(i, d)] = v0;
+                                if (two) Ap[v6_at(i, d + 1)] = v1;
+                            } else {
+                                Pp[v6_at(i, d)] = v0, idx[v6_at(i, d)] = (unsigned char)j0;
+                                if (two) Pp[v6_at(i, d + 1)] = v1, idx[v6_at(i, d + 1)] = (unsigned char)j1;
+                            }
                         }
                         if (!a_kind && valid) {
                             const float gi = __expf(Li);
