@@ -144,6 +144,20 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
                               int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
                               float *S_out_f32, int32_t *seq_status, void *cuda_stream);
 
+/*
+ * Full-state snapshotting, the scheme the method replaces (Section 2, "Speculative verification:
+ * where GDN blows up" and "Existing approaches" (i)): materialise the state of EVERY draft node,
+ *   Snap[t,h] = g_t S0[b,h] + sum_{j ancestor-or-self of t} (g_t/g_j) u_j k_j^T      (Eq. 3 with a = t)
+ * for each packed node t of sequence b, out of place (S0 is not modified).  Provided as a measured
+ * comparator: it writes N states per sequence and head where commit writes one.
+ *   S0 [B,H_v,128,128], k [T,H_qk,128]: BF16 only (F32 returns TREEWY_ERR_UNSUPPORTED);
+ *   U [T,H_v,128] fp32 from treewy_verify;  Snap [T,H_v,128,128] bf16, out.
+ * Malformed sequences are flagged and their states left untouched, as in treewy_commit.
+ */
+treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *k, const treewy_tree_t *tree,
+                                    int32_t H_qk, treewy_dtype_t io_dtype, void *Snap, int32_t *seq_status,
+                                    void *cuda_stream);
+
 /* A short constant string for a status code. */
 const char *treewy_status_string(treewy_status_t status);
 

@@ -68,6 +68,8 @@ def load_library(path: str | None = None):
     lib.treewy_commit.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, vp, ctypes.c_int,
                                   vp, vp, vp]
     lib.treewy_commit.restype = ctypes.c_int
+    lib.treewy_snapshot_all.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, vp, vp, vp]
+    lib.treewy_snapshot_all.restype = ctypes.c_int
     lib.treewy_status_string.argtypes = [ctypes.c_int]
     lib.treewy_status_string.restype = ctypes.c_char_p
     lib.treewy_version.restype = ctypes.c_int
@@ -159,6 +161,16 @@ def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Te
     _check("treewy_commit",
            lib.treewy_commit(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
                              _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+
+
+def treewy_snapshot_all(S0, U, k, tree: Tree, H_qk: int, Snap: torch.Tensor,
+                        seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """Every node's state into Snap [T, H_v, 128, 128] (the snapshotting comparator); S0 is read only."""
+    lib = load_library()
+    ts = tree.struct()
+    _check("treewy_snapshot_all",
+           lib.treewy_snapshot_all(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
+                                   _p(Snap), _p(seq_status), _stream(stream)))
 
 
 # --------------------------------------------------------------------------- user-level step

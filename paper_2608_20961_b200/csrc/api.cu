@@ -118,7 +118,32 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.snap_out = nullptr, a.T = tree->T;
     cudaError_t e = launch_commit(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *k, const treewy_tree_t *tree,
+                                    int32_t H_qk, treewy_dtype_t io_dtype, void *Snap, int32_t *seq_status,
+                                    void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (io_dtype != TREEWY_BF16) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0 || tree->T == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(U) || bad_ptr(k) || bad_ptr(Snap)) return TREEWY_ERR_INVALID_ARG;
+
+    CommitArgs a;
+    a.S0 = const_cast<void *>(S0), a.U = U, a.k = k;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.accepted = nullptr, a.S_out_f32 = nullptr, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.snap_out = Snap, a.T = tree->T;
+    cudaError_t e = launch_commit_pipe(a, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 

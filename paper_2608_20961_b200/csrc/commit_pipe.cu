@@ -16,6 +16,10 @@
 //     of them sends it back with a bulk store; the stage is handed back to its producer once
 //     the store has drained the shared-memory buffer.
 //
+// Snapshot mode (the full-state-snapshotting comparator): the same pipeline with one item per
+// (packed node, value head), the node playing the accepted node and the result going to a
+// separate [T, H_v] array of states instead of back to S0.
+//
 // Paths longer than CP_PCH nodes (deep chains) take the staged rows first and fetch the rest
 // with ordinary loads.  All mbarrier waits are bounded (TREEWY_SEQ_TIMEOUT on give-up).
 #include "ptx_sm100.cuh"
@@ -38,7 +42,8 @@ struct __align__(128) CommitStage {
     unsigned long long mask;  // ancestor-or-self mask of the accepted node
     float La, ga;             // log-gate of the accepted node and e^{La}
     int plen;                 // path length; -1 = nothing to do for this item
-    int store_tile;           // 1: tile goes back to S0 (accepted >= 0)
+    int store_tile;           // 1: tile goes back to memory (accepted >= 0)
+    int b, h;                 // sequence and value head of the item
 };
 
 struct CommitPipeSmem {
@@ -85,10 +90,23 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         for (int kk = s;; kk += CP_STAGES) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
-            const int b = item / a.H_v, h = item - b * a.H_v;
+            int b, h;
+            if (a.snap_out) {  // snapshot mode: item = (packed node, head); find the node's sequence
+                const int t = item / a.H_v;
+                h = item - t * a.H_v;
+                int l = 0, r = a.B - 1;
+                while (l < r) {
+                    const int mid = (l + r + 1) >> 1;
+                    if (a.node_offsets[mid] <= t) l = mid;
+                    else r = mid - 1;
+                }
+                b = l;
+            } else {
+                b = item / a.H_v, h = item - b * a.H_v;
+            }
             const int lo = a.node_offsets[b];
             const int n = a.node_offsets[b + 1] - lo;
-            const int acc = a.accepted[b];
+            const int acc = a.snap_out ? item / a.H_v - lo : a.accepted[b];
 
             int bad = 0;
             if (n < 1 || n > a.max_nodes) {
@@ -102,7 +120,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 if (__any_sync(0xffffffffu, bp)) bad = TREEWY_SEQ_BAD_PARENT;
                 else if (acc < -1 || acc >= n) bad = TREEWY_SEQ_BAD_ACCEPTED;
             }
-            if (bad && h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
+            if (bad && h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);  // idempotent
 
             const bool work = !bad && (acc >= 0 || a.S_out_f32 != nullptr);
             unsigned long long mask = 0;
@@ -127,6 +145,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             if (lane == 0) {
                 g.mask = mask, g.La = La, g.ga = expf(La), g.plen = plen;
                 g.store_tile = (acc >= 0);
+                g.b = b, g.h = h;
             }
             __syncwarp();
             if (!work) {
@@ -135,7 +154,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             }
             if (lane == 0) {
                 ptx::mbar_arrive_expect_tx(&sm.full[s], CP_TILE_BYTES + cnt * (D * 2 + D * 4));
-                ptx::bulk_g2s(g.tile, S0 + (size_t)item * D * D, CP_TILE_BYTES, &sm.full[s]);
+                ptx::bulk_g2s(g.tile, S0 + ((size_t)b * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
             }
             __syncwarp();
             if (lane < cnt) {
@@ -157,13 +176,13 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         const int s = kk % CP_STAGES;
         CommitStage &g = sm.stage[s];
         if (!ptx::mbar_wait(&sm.full[s], (kk / CP_STAGES) & 1)) {
-            if (tid == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+            if (tid == 0 && a.seq_status && !a.snap_out) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
             break;
         }
         const int plen = g.plen;
         const int store_tile = g.store_tile;
         if (plen >= 0) {
-            const int b = item / a.H_v, h = item - b * a.H_v;
+            const int b = g.b, h = g.h;
             float acc[8][8];
             const float ga = g.ga;
 #pragma unroll
@@ -235,7 +254,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         ptx::named_sync(1, CP_CONSUMERS);  // every consumer is done with this stage
         if (tid == 0) {
             if (plen >= 0 && store_tile) {
-                ptx::bulk_s2g(S0 + (size_t)item * D * D, g.tile, CP_TILE_BYTES);
+                __nv_bfloat16 *dst = a.snap_out ? static_cast<__nv_bfloat16 *>(a.snap_out) : S0;
+                ptx::bulk_s2g(dst + (size_t)item * D * D, g.tile, CP_TILE_BYTES);
                 ptx::bulk_commit_group();
                 if (pending >= 0) {
                     ptx::bulk_wait_group_read<1>();  // the previous store has left its stage
@@ -257,7 +277,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
 
 cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream)
 {
-    const long long n_items = (long long)a.B * a.H_v;
+    const long long n_items = (long long)(a.snap_out ? a.T : a.B) * a.H_v;
     if (n_items == 0) return cudaSuccess;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);

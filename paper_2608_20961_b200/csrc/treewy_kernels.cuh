@@ -36,6 +36,8 @@ struct CommitArgs {
     float *S_out_f32;
     int32_t *seq_status;
     int B, H_v, H_qk, max_nodes;
+    void *snap_out;  // snapshot mode when not NULL: [T, H_v, 128, 128] states, one per node
+    int T;
 };
 
 cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha,
