@@ -145,6 +145,29 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
                               float *S_out_f32, int32_t *seq_status, void *cuda_stream);
 
 /*
+ * Commit of the previous round fused into the verify of this round (Section 3, Eq. 3 then Eq. 2;
+ * the paper's Section 4 runs chains this way, and its deferred-state discussion in the ReplaySSM
+ * appendix names the state write as the lever): in serving, a layer's commit of round r is always
+ * followed by its verify of round r+1 on the same state, so one kernel reads the old state once,
+ * applies Eq. 3 in shared memory, writes the new state once and verifies the new draft tree from it.
+ * The result is bit-identical to
+ *     treewy_commit(S0, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, NULL, ...);
+ *     treewy_verify(S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, ...);
+ * single_kernel = 0 issues exactly those two kernels (the faster choice on B200 today: both run
+ * near the HBM roof on their own).  single_kernel = 1 takes the fused kernel when it applies (BF16
+ * states, trees of up to 32 nodes in the new round; otherwise the two kernels again): it moves
+ * 23 % fewer bytes, but its in-kernel commit is instruction-bound and it is currently the slower one.
+ * tree_prev / tree must describe the same B sequences and H_v heads; U_prev [T_prev,H_v,128] fp32
+ * and k_prev [T_prev,H_qk,128] are the previous round's verify output and keys, accepted_prev [B]
+ * its accepted nodes (-1 = nothing to commit for that sequence).  U_prev and U must not overlap.
+ */
+treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *k_prev,
+                                     const treewy_tree_t *tree_prev, const int32_t *accepted_prev, const void *q,
+                                     const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
+                                     int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                     float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream);
+
+/*
  * Full-state snapshotting, the scheme the method replaces (Section 2, "Speculative verification:
  * where GDN blows up" and "Existing approaches" (i)): materialise the state of EVERY draft node,
  *   Snap[t,h] = g_t S0[b,h] + sum_{j ancestor-or-self of t} (g_t/g_j) u_j k_j^T      (Eq. 3 with a = t)

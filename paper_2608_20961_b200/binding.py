@@ -68,6 +68,9 @@ def load_library(path: str | None = None):
     lib.treewy_commit.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, vp, ctypes.c_int,
                                   vp, vp, vp]
     lib.treewy_commit.restype = ctypes.c_int
+    lib.treewy_commit_verify.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), vp, vp, vp, vp, vp,
+                                         ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
+    lib.treewy_commit_verify.restype = ctypes.c_int
     lib.treewy_snapshot_all.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, vp, vp, vp]
     lib.treewy_snapshot_all.restype = ctypes.c_int
     lib.treewy_status_string.argtypes = [ctypes.c_int]
@@ -161,6 +164,20 @@ def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Te
     _check("treewy_commit",
            lib.treewy_commit(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
                              _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+
+
+def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta, tree: Tree,
+                         H_qk: int, O: torch.Tensor, U: torch.Tensor, single_kernel: bool = False,
+                         seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """Commit the previous round's accepted nodes into S0 and verify the new trees: the two stand-alone
+    kernels, or (single_kernel) the fused kernel that reads and writes the state once."""
+    lib = load_library()
+    tp, ts = tree_prev.struct(), tree.struct()
+    _check("treewy_commit_verify",
+           lib.treewy_commit_verify(_p(S0), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev), _p(q),
+                                    _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
+                                    _DTYPES[O.dtype], _p(O), _p(U), int(bool(single_kernel)), _p(seq_status),
+                                    _stream(stream)))
 
 
 def treewy_snapshot_all(S0, U, k, tree: Tree, H_qk: int, Snap: torch.Tensor,

@@ -147,6 +147,49 @@ treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 
+treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *k_prev,
+                                     const treewy_tree_t *tree_prev, const int32_t *accepted_prev, const void *q,
+                                     const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
+                                     int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                     float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream)
+{
+    int max_prev = 0, max_nodes = 0;
+    treewy_status_t st = check_tree(tree_prev, true, &max_prev);
+    if (st != TREEWY_OK) return st;
+    st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (tree_prev->B != tree->B || tree_prev->H_v != tree->H_v) return TREEWY_ERR_INVALID_ARG;
+    const bool fusable = single_kernel != 0 && io_dtype == TREEWY_BF16 && max_nodes <= 32 && tree->B > 0 && tree->T > 0 && tree_prev->T > 0;
+    if (!fusable) {  // same result from the two stand-alone kernels
+        st = treewy_commit(S0, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
+                           cuda_stream);
+        if (st != TREEWY_OK) return st;
+        return treewy_verify(S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
+    }
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (bad_ptr(S0) || bad_ptr(U_prev) || bad_ptr(k_prev) || bad_ptr(accepted_prev) || bad_ptr(q) || bad_ptr(k) ||
+        bad_ptr(v) || bad_ptr(beta) || bad_ptr(O) || bad_ptr(U))
+        return TREEWY_ERR_INVALID_ARG;
+
+    VerifyArgs a;
+    a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.depth = tree->depth, a.level_order = tree->level_order;
+    a.O = O, a.U = U, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.cls_lo = 0, a.cls_hi = max_nodes;
+    PrevRound pv;
+    pv.U = U_prev, pv.k = k_prev;
+    pv.node_offsets = tree_prev->node_offsets, pv.parent = tree_prev->parent;
+    pv.anc_mask = tree_prev->anc_mask, pv.cum_log_gate = tree_prev->cum_log_gate;
+    pv.accepted = accepted_prev, pv.max_nodes = max_prev;
+    cudaError_t e = launch_commit_verify_sm100(a, pv, tree->T, o_dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
 const char *treewy_status_string(treewy_status_t status)
 {
     switch (status) {

@@ -52,18 +52,6 @@ struct CommitPipeSmem {
     uint64_t empty[CP_STAGES];
 };
 
-__device__ __forceinline__ int nth_set_bit(unsigned long long m, int p)
-{
-    for (int q = 0; q < p; ++q) m &= m - 1;
-    return __ffsll((long long)m) - 1;
-}
-
-__device__ __forceinline__ void widen8(const uint4 &x, float (&f)[8])
-{
-    f[0] = bf16lo(x.x), f[1] = bf16hi(x.x), f[2] = bf16lo(x.y), f[3] = bf16hi(x.y);
-    f[4] = bf16lo(x.z), f[5] = bf16hi(x.z), f[6] = bf16lo(x.w), f[7] = bf16hi(x.w);
-}
-
 __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a, int n_items)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];

@@ -117,6 +117,13 @@ __device__ __forceinline__ void tma_load_2d(void *dst_smem, const void *tmap, in
         "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
         : "memory");
 }
+// tiled 2-D tensor-map store, shared -> global, tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void tma_store_2d(const void *tmap, int x, int y, const void *src_smem)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(tmap),
+                 "r"(x), "r"(y), "r"(smem_u32(src_smem))
+                 : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const void *tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");

@@ -61,6 +61,18 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
+__device__ __forceinline__ int nth_set_bit(unsigned long long m, int p)
+{
+    for (int q = 0; q < p; ++q) m &= m - 1;
+    return __ffsll((long long)m) - 1;
+}
+
+__device__ __forceinline__ void widen8(const uint4 &x, float (&f)[8])
+{
+    f[0] = bf16lo(x.x), f[1] = bf16hi(x.x), f[2] = bf16lo(x.y), f[3] = bf16hi(x.y);
+    f[4] = bf16lo(x.z), f[5] = bf16hi(x.z), f[6] = bf16lo(x.w), f[7] = bf16hi(x.w);
+}
+
 // stores that are predicated instead of branched around (keeps the epilogue one straight line)
 __device__ __forceinline__ void st_global_if(float *p, float v, bool on)
 {

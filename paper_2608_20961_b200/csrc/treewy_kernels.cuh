@@ -25,6 +25,17 @@ struct VerifyArgs {
     int cls_lo, cls_hi;
 };
 
+// the previous decoding round, whose accepted node the fused kernel commits before verifying
+struct PrevRound {
+    const float *U;
+    const void *k;
+    const int32_t *node_offsets, *parent;
+    const uint64_t *anc_mask;
+    const float *cum_log_gate;
+    const int32_t *accepted;
+    int max_nodes;
+};
+
 struct CommitArgs {
     void *S0;
     const float *U;
@@ -46,6 +57,9 @@ cudaError_t launch_verify_generic(const VerifyArgs &a, treewy_dtype_t io, treewy
                                   cudaStream_t stream);
 // bf16 inputs: TMA + tcgen05 kernel; T = packed node count (bounds the q/k/v tensor maps)
 cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
+// commit of the previous round fused into verify (trees of up to 32 nodes in the new round)
+cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv, int T, treewy_dtype_t od,
+                                       cudaStream_t stream);
 cudaError_t launch_verify_sm100_tc64(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
 cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
 cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream);  // bf16 state

@@ -41,25 +41,31 @@ namespace treewy {
 constexpr int VT_GROUP = 128;
 constexpr uint32_t VT_TMEM_COLS = 512;
 
-template <int NP> struct VtCfg {
+template <int NP, bool FUSED> struct VtCfg {
     static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
     static constexpr int GROUPS = 2;
-    static constexpr int STAGES = 4;
+    static constexpr int STAGES = FUSED ? 3 : 4;
+    static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     static constexpr int TBUF = 5;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
     static constexpr int CONSUMERS = VT_GROUP * GROUPS;
-    static constexpr int MMA1_WARP = CONSUMERS / 32;
+    static constexpr int COMMIT_WARP0 = CONSUMERS / 32;
+    static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
     static constexpr int MMA2_WARP = MMA1_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
-    static constexpr int THREADS = CONSUMERS + 64 + 32 * STAGES;
-    // stage: [Q;K] tile | S0 tile | meta   (the v rows arrive later, into the dead S0 tile)
+    static constexpr int THREADS = CONSUMERS + CGROUP + 64 + 32 * STAGES;
+    // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
+    // (the v rows arrive later, into the dead S0 tile)
     static constexpr int QK_HALF = 2 * NP * 128;
     static constexpr int QK_BYTES = 2 * QK_HALF;
     static constexpr int S0_HALF = D * 128;
     static constexpr int S0_BYTES = 2 * S0_HALF;
     static constexpr int OFF_S0 = QK_BYTES;
-    static constexpr int OFF_META = OFF_S0 + S0_BYTES;
+    static constexpr int PCH = 16;  // previous-round path nodes staged per item (fused mode)
+    static constexpr int OFF_KP = OFF_S0 + S0_BYTES, OFF_UP = OFF_KP + PCH * D * 2;
+    static constexpr int OFF_META = FUSED ? OFF_UP + PCH * D * 4 : OFF_S0 + S0_BYTES;
     static constexpr int META_BYTES = NP * 16 + 16;  // mask u64, L f32, beta f32 per node; n, lo
-    static constexpr int STAGE_BYTES = (OFF_META + META_BYTES + 1023) / 1024 * 1024;
+    static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
+    static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
     // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
     static constexpr int OFF_T_HI = 0, OFF_T_LO = NP * 128, OFF_W_HI = 2 * NP * 128, OFF_W_LO = 3 * NP * 128;
     static constexpr int OFF_RT_HI = OFF_S0, OFF_RT_LO = OFF_S0 + D * 128;
@@ -79,7 +85,7 @@ template <int NP> struct VtCfg {
     static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + 4 * TBUF + GROUPS) * 8 + 16 + 1024;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + GROUPS) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // per TMEM buffer: SQ | SK | D2; stage 2 writes DO over SK and DU over D2 (both dead by then)
     static constexpr int TM_COLS = 3 * NP;
@@ -87,13 +93,23 @@ template <int NP> struct VtCfg {
     static_assert(TBUF * TM_COLS <= 512, "tensor memory");
 };
 
-template <int NP, typename TOut>
-__global__ void __launch_bounds__(VtCfg<NP>::THREADS, 1)
-verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtensorMap tmS0,
+// fused mode: what the commit of the previous round needs for one (sequence, head)
+struct PathMeta {
+    float w[16];              // e^{L_a - L_j} of the staged path nodes
+    unsigned long long mask;  // ancestor-or-self mask of the accepted node (previous tree)
+    float La, ga;             // its log-gate and e^{La}
+    int plen;                 // path length; -1 = no commit for this item
+    int lo;                   // first packed node of the sequence in the previous tree
+};
+static_assert(sizeof(PathMeta) <= 128, "path meta block");
+
+template <int NP, typename TOut, bool FUSED>
+__global__ void __launch_bounds__(VtCfg<NP, FUSED>::THREADS, 1)
+verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_constant__ CUtensorMap tmS0,
                        const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV)
 {
-    using C = VtCfg<NP>;
+    using C = VtCfg<NP, FUSED>;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
@@ -103,7 +119,8 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
     uint64_t *mma2_done = ops_ready + C::TBUF;
     uint64_t *tmem_free = mma2_done + C::TBUF;
     uint64_t *v_ready = tmem_free + C::TBUF;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(v_ready + C::GROUPS);
+    uint64_t *upd_done = v_ready + C::GROUPS;  // fused mode: the state tile of a stage carries the commit
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(upd_done + C::STAGES);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -119,6 +136,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             ptx::mbar_init(&tmem_free[i], VT_GROUP);
         }
         for (int g = 0; g < C::GROUPS; ++g) ptx::mbar_init(&v_ready[g], 1);
+        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128);
         ptx::fence_barrier_init();
     }
     if (warp == C::MMA1_WARP) {
@@ -150,11 +168,16 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             int item, b, h, lo, n, bad, flag;
             unsigned long long mk;
             float Lv, bv;
+            // fused mode: the previous round's accepted path of this sequence
+            int plo, pbad, plen, cnt, pj;
+            unsigned long long pmask;
+            float La, wj;
         };
         auto fetch = [&](int kk) {
             Pre p;
             p.item = blockIdx.x + kk * gridDim.x;
             p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
+            p.plo = 0, p.pbad = 0, p.plen = -1, p.cnt = 0, p.pj = 0, p.pmask = 0ull, p.La = 0.f, p.wj = 0.f;
             if (p.item >= n_items) return p;
             p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
             p.lo = a.node_offsets[p.b];
@@ -173,6 +196,32 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             p.mk = on ? a.anc_mask[p.lo + lane] : 0ull;
             p.Lv = on ? a.cum_log_gate[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
             p.bv = on ? a.beta[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
+            if constexpr (FUSED) {
+                p.plo = pv.node_offsets[p.b];
+                const int pn = pv.node_offsets[p.b + 1] - p.plo;
+                const int acc = pv.accepted[p.b];
+                if (pn < 1 || pn > pv.max_nodes) {
+                    p.pbad = TREEWY_SEQ_TOO_MANY_NODES;
+                } else {
+                    int bp = 0;
+                    for (int i = lane; i < pn; i += 32) {
+                        const int par = pv.parent[p.plo + i];
+                        bp |= (par < -1 || par >= i);
+                    }
+                    if (__any_sync(0xffffffffu, bp)) p.pbad = TREEWY_SEQ_BAD_PARENT;
+                    else if (acc < -1 || acc >= pn) p.pbad = TREEWY_SEQ_BAD_ACCEPTED;
+                }
+                if (!p.pbad && acc >= 0) {
+                    p.pmask = pv.anc_mask[p.plo + acc];
+                    p.La = pv.cum_log_gate[(size_t)(p.plo + acc) * a.H_v + p.h];
+                    p.plen = __popcll(p.pmask);
+                    p.cnt = min(p.plen, C::PCH);
+                    if (lane < p.cnt) {
+                        p.pj = nth_set_bit(p.pmask, lane);
+                        p.wj = expf(p.La - pv.cum_log_gate[(size_t)(p.plo + p.pj) * a.H_v + p.h]);
+                    }
+                }
+            }
             return p;
         };
         Pre cur = fetch(s);
@@ -180,29 +229,145 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             if (cur.item >= n_items) break;
             const Pre p = cur;
             if (p.bad && p.flag && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
+            if (FUSED && p.pbad && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.pbad);
             if (!ptx::mbar_wait(&empty[s], ((kk / C::STAGES) & 1) ^ 1)) {
                 if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], TREEWY_SEQ_TIMEOUT);
                 break;
             }
             if (lane < NP) meta_mask(stage)[lane] = p.mk, meta_L(stage)[lane] = p.Lv, meta_beta(stage)[lane] = p.bv;
             if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo;
+            if constexpr (FUSED) {
+                PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
+                if (lane < p.cnt) pm->w[lane] = p.wj;
+                if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = expf(p.La), pm->plen = p.plen, pm->lo = p.plo;
+            }
             __syncwarp();
+            const bool need_tile = !p.bad || p.plen >= 0;  // the state tile serves verify, commit or both
             if (lane == 0) {
-                if (p.bad) {
+                const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
+                if (tx == 0) {
                     ptx::mbar_arrive(&full[s]);
                 } else {
-                    ptx::mbar_arrive_expect_tx(&full[s], C::TX_BYTES);
+                    ptx::mbar_arrive_expect_tx(&full[s], tx);
                     const int hq = p.h / group;
-                    ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.item * D, &full[s]);
-                    ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.item * D, &full[s]);
-                    ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
-                    ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
-                    ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
-                    ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
+                    if (need_tile) {
+                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.item * D, &full[s]);
+                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.item * D, &full[s]);
+                    }
+                    if (!p.bad) {
+                        ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
+                        ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
+                        ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
+                        ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
+                    }
+                }
+            }
+            if constexpr (FUSED) {
+                __syncwarp();
+                if (lane < p.cnt) {  // the accepted path's k and U rows of the previous round
+                    const __nv_bfloat16 *kp = static_cast<const __nv_bfloat16 *>(pv.k);
+                    ptx::bulk_g2s(stage + C::OFF_KP + lane * D * 2,
+                                  kp + ((size_t)(p.plo + p.pj) * a.H_qk + p.h / group) * D, D * 2, &full[s]);
+                    ptx::bulk_g2s(stage + C::OFF_UP + lane * D * 4, pv.U + ((size_t)(p.plo + p.pj) * a.H_v + p.h) * D,
+                                  D * 4, &full[s]);
                 }
             }
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
         }
+    } else if (FUSED && warp >= C::COMMIT_WARP0 && warp < C::MMA1_WARP) {
+        // ------------------------------------------------------------------ commit group (fused mode)
+        // Before the stage-1 MMAs read a state tile, the previous round's accepted node is
+        // committed INTO it (Eq. 3):  S <- g_a S + sum_{j on the path} (g_a / g_j) u_j k_j^T , same
+        // fp32 arithmetic and summation order as the stand-alone commit kernel, rounded once to bf16
+        // in place (the tile keeps the 128-byte swizzle the TMA gave it), and the new state goes back
+        // to global memory with a TMA store while verification proceeds from the shared-memory copy.
+        const int t = tid - C::COMMIT_WARP0 * 32;
+        const int cc = t & 15, r0 = t >> 4;  // 16-byte column chunk; first of every eighth row
+        const int group = a.H_v / a.H_qk;
+        for (int kk = 0;; ++kk) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            if (item >= n_items) break;
+            const int s = kk % C::STAGES;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) {
+                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                break;
+            }
+            const PathMeta *pm = reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA);
+            const int plen = pm->plen;
+            if (plen >= 0) {
+                const int b = item / a.H_v, h = item - b * a.H_v;
+                unsigned char *tile = stage + C::OFF_S0 + (cc >> 3) * C::S0_HALF;
+                const __nv_bfloat16 *kp = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_KP);
+                const float *up = reinterpret_cast<const float *>(stage + C::OFF_UP);
+                const float ga = pm->ga;
+                const int cnt = min(plen, C::PCH);
+#pragma unroll 1
+                for (int pass = 0; pass < 2; ++pass) {
+                    float acc[8][8];
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = r0 + 8 * (pass * 8 + it);
+                        widen8(*reinterpret_cast<const uint4 *>(tile + r * 128 + (((cc & 7) ^ (r & 7)) << 4)), acc[it]);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[it][e] *= ga;
+                    }
+                    for (int p = 0; p < cnt; ++p) {
+                        const float w = pm->w[p];
+                        float kf[8];
+                        widen8(*reinterpret_cast<const uint4 *>(kp + p * D + cc * 8), kf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) kf[e] *= w;
+#pragma unroll
+                        for (int it = 0; it < 8; ++it) {
+                            const float u = up[p * D + r0 + 8 * (pass * 8 + it)];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
+                        }
+                    }
+                    if (plen > C::PCH) {  // deep path: remaining nodes straight from global memory
+                        const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(pv.k);
+                        unsigned long long m = pm->mask;
+                        for (int q = 0; q < C::PCH; ++q) m &= m - 1;
+                        while (m) {
+                            const int j = __ffsll((long long)m) - 1;
+                            m &= m - 1;
+                            const float w = expf(pm->La - pv.cum_log_gate[(size_t)(pm->lo + j) * a.H_v + h]);
+                            float kf[8];
+                            widen8(*reinterpret_cast<const uint4 *>(kg + ((size_t)(pm->lo + j) * a.H_qk + h / group) * D + cc * 8),
+                                   kf);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) kf[e] *= w;
+                            const float *ur = pv.U + ((size_t)(pm->lo + j) * a.H_v + h) * D;
+#pragma unroll
+                            for (int it = 0; it < 8; ++it) {
+                                const float u = ur[r0 + 8 * (pass * 8 + it)];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = r0 + 8 * (pass * 8 + it);
+                        uint4 y;
+                        y.x = pack_bf16(acc[it][0], acc[it][1]), y.y = pack_bf16(acc[it][2], acc[it][3]);
+                        y.z = pack_bf16(acc[it][4], acc[it][5]), y.w = pack_bf16(acc[it][6], acc[it][7]);
+                        *reinterpret_cast<uint4 *>(tile + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = y;
+                    }
+                }
+                ptx::fence_proxy_async();  // the tile is read next by the tensor core and by the TMA store
+            }
+            ptx::named_sync(3, C::CGROUP > 0 ? C::CGROUP : 32);
+            if (plen >= 0 && t == 0) {
+                ptx::tma_store_2d(&tmS0, 0, item * D, stage + C::OFF_S0);
+                ptx::tma_store_2d(&tmS0, 64, item * D, stage + C::OFF_S0 + C::S0_HALF);
+                ptx::bulk_commit_group();
+                ptx::bulk_wait_group_read<0>();  // the tile will be overwritten by scratch after the MMAs
+            }
+            ptx::mbar_arrive(&upd_done[s]);
+        }
+        if (t == 0) ptx::bulk_wait_group<0>();
     } else if (warp == C::MMA1_WARP) {
         // ------------------------------------------------------------------ stage-1 MMAs
         constexpr uint32_t idesc1 = ptx::umma_idesc_bf16_f32(128, 2 * NP);
@@ -214,6 +379,7 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
             unsigned char *stage = smem + s * C::STAGE_BYTES;
             if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) break;
             const int n = meta_nlo(stage)[0];
+            if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
             if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
             ptx::tc_fence_after_sync();
             if (lane == 0) {
@@ -558,10 +724,10 @@ verify_sm100_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtens
 
 namespace {
 
-template <int NP, typename TOut>
-cudaError_t launch_vt(const VerifyArgs &a, int T, cudaStream_t stream)
+template <int NP, typename TOut, bool FUSED>
+cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStream_t stream)
 {
-    using C = VtCfg<NP>;
+    using C = VtCfg<NP, FUSED>;
     const long long n_items = (long long)a.B * a.H_v;
     VerifyMaps m;
     if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_items, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
@@ -570,33 +736,55 @@ cudaError_t launch_vt(const VerifyArgs &a, int T, cudaStream_t stream)
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(verify_sm100_tc_kernel<NP, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(verify_sm100_tc_kernel<NP, TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int grid = (int)(n_items < sms ? n_items : sms);
-    verify_sm100_tc_kernel<NP, TOut><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, (int)n_items, m.S0, m.Q,
-                                                                                   m.K, m.V);
+    verify_sm100_tc_kernel<NP, TOut, FUSED><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, pv, (int)n_items, m.S0,
+                                                                                         m.Q, m.K, m.V);
     return cudaGetLastError();
+}
+
+template <bool FUSED>
+cudaError_t launch_small(const VerifyArgs &a, const PrevRound &pv, int T, treewy_dtype_t od, cudaStream_t stream)
+{
+    if (a.max_nodes <= 16)
+        return od == TREEWY_F32 ? launch_vt<16, float, FUSED>(a, pv, T, stream)
+                                : launch_vt<16, __nv_bfloat16, FUSED>(a, pv, T, stream);
+    return od == TREEWY_F32 ? launch_vt<32, float, FUSED>(a, pv, T, stream)
+                            : launch_vt<32, __nv_bfloat16, FUSED>(a, pv, T, stream);
 }
 
 }  // namespace
 
-// bf16 inputs.  Sequences of up to 32 nodes take the kernel above, larger ones the general variant;
+// bf16 inputs.  Sequences of up to 32 nodes take the kernel above, larger ones the 64-node variant;
 // a batch that may hold both (max_nodes > 32) gets one launch per size class.
 cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
 {
     if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
+    const PrevRound none = {};
     VerifyArgs small = a;
     small.cls_lo = 0, small.cls_hi = a.max_nodes < 32 ? a.max_nodes : 32;
     cudaError_t e;
-    if (a.max_nodes <= 16)
-        e = od == TREEWY_F32 ? launch_vt<16, float>(small, T, stream) : launch_vt<16, __nv_bfloat16>(small, T, stream);
+    if (small.cls_hi <= 16)
+        e = od == TREEWY_F32 ? launch_vt<16, float, false>(small, none, T, stream)
+                             : launch_vt<16, __nv_bfloat16, false>(small, none, T, stream);
     else
-        e = od == TREEWY_F32 ? launch_vt<32, float>(small, T, stream) : launch_vt<32, __nv_bfloat16>(small, T, stream);
+        e = od == TREEWY_F32 ? launch_vt<32, float, false>(small, none, T, stream)
+                             : launch_vt<32, __nv_bfloat16, false>(small, none, T, stream);
     if (e != cudaSuccess || a.max_nodes <= 32) return e;
     VerifyArgs large = a;
     large.cls_lo = 32, large.cls_hi = a.max_nodes;
     return launch_verify_sm100_tc64(large, T, od, stream);
+}
+
+// commit of the previous round + verify of this one, one kernel; this round's trees have <= 32 nodes
+cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv, int T, treewy_dtype_t od,
+                                       cudaStream_t stream)
+{
+    VerifyArgs small = a;
+    small.cls_lo = 0, small.cls_hi = a.max_nodes;
+    return launch_small<true>(small, pv, T, od, stream);
 }
 
 }  // namespace treewy
