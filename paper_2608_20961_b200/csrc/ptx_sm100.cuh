@@ -135,6 +135,13 @@ __device__ __forceinline__ void named_sync(int id, int count)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+// arrival at a named barrier without waiting: the `count` threads are those that arrive plus those
+// that wait in named_sync on the same id
+__device__ __forceinline__ void named_arrive(int id, int count)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
 // named barrier that also ORs a predicate over the participating threads
 __device__ __forceinline__ bool named_sync_or(int id, int count, bool pred)
 {

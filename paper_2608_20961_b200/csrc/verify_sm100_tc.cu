@@ -46,13 +46,16 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int GROUPS = 2;
     static constexpr int STAGES = FUSED ? 3 : 4;
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
-    static constexpr int TBUF = 5;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
+    static constexpr int TBUF = 6;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
+    static constexpr int GBUF = 4;  // ... and a ring of short-lived Gram blocks
     static constexpr int CONSUMERS = VT_GROUP * GROUPS;
-    static constexpr int COMMIT_WARP0 = CONSUMERS / 32;
+    static constexpr int TW = 64;  // threads of a group's solver warps (one per row of T and of W)
+    static constexpr int TW_WARP0 = CONSUMERS / 32;
+    static constexpr int COMMIT_WARP0 = TW_WARP0 + GROUPS * TW / 32;
     static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
     static constexpr int MMA2_WARP = MMA1_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
-    static constexpr int THREADS = CONSUMERS + CGROUP + 64 + 32 * STAGES;
+    static constexpr int THREADS = CONSUMERS + GROUPS * TW + CGROUP + 64 + 32 * STAGES;
     // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
     // (the v rows arrive later, into the dead S0 tile)
     static constexpr int QK_HALF = 2 * NP * 128;
@@ -63,7 +66,11 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int PCH = 16;  // previous-round path nodes staged per item (fused mode)
     static constexpr int OFF_KP = OFF_S0 + S0_BYTES, OFF_UP = OFF_KP + PCH * D * 2;
     static constexpr int OFF_META = FUSED ? OFF_UP + PCH * D * 4 : OFF_S0 + S0_BYTES;
-    static constexpr int META_BYTES = NP * 16 + 16;  // mask u64, L f32, beta f32 per node; n, lo
+    // mask u64, L f32, beta f32 per node; n, lo, deep; then the producer-built path lists of the
+    // first 8 ancestors of every node: gate ratios e^{L_i - L_j} as [d / 4][node][d % 4] floats and
+    // the ancestors' indices as [d / 4][node] words of four bytes
+    static constexpr int META_RAT = NP * 16 + 16, META_IDX = META_RAT + 2 * NP * 16;
+    static constexpr int META_BYTES = META_IDX + 2 * NP * 4;
     static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
     static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
     // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
@@ -75,22 +82,29 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
     static constexpr int XLD = NP + 1;
     static constexpr int OFF_RAW = OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;
-    static constexpr int OFF_VS = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 127) / 128 * 128;  // v rows [NP][128] bf16
+    // ... and, for trees with a path of more than 8 ancestors, the full-length lists
+    static constexpr int OFF_DAP = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 15) / 16 * 16;
+    static constexpr int OFF_DPP = OFF_DAP + NP * NP * 4, OFF_DIDX = OFF_DPP + NP * NP * 4;
+    static_assert(OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
     static constexpr int V_BYTES = NP * D * 2;
-    static_assert(OFF_VS + V_BYTES <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
-    // group-private: path lists, per-node scalars (double-buffered), ancestor indices
-    static constexpr int GP_AP = 0, GP_PP = NP * NP * 4, GP_SCAL = 2 * NP * NP * 4;
-    static constexpr int GP_IDX = GP_SCAL + 2 * NP * 16;
-    static constexpr int GP_BYTES = (GP_IDX + NP * NP + 15) / 16 * 16;
+    // group-private: path lists of the first 8 ancestors, per-node scalars (double-buffered), and
+    // the v rows [NP][128] bf16 of the group's next item (loaded one item ahead)
+    static constexpr int GP_AP = 0, GP_PP = 2 * NP * 16, GP_SCAL = 4 * NP * 16;
+    static constexpr int GP_VS = (GP_SCAL + 2 * NP * 16 + 127) / 128 * 128;
+    static constexpr int GP_BYTES = GP_VS + V_BYTES;
     static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + GROUPS) * 8 + 16 + 1024;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + GBUF + 3 * GROUPS) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
-    // per TMEM buffer: SQ | SK | D2; stage 2 writes DO over SK and DU over D2 (both dead by then)
-    static constexpr int TM_COLS = 3 * NP;
-    static constexpr int TM_DO = NP, TM_DU = 2 * NP;
-    static_assert(TBUF * TM_COLS <= 512, "tensor memory");
+    // per TMEM buffer: SQ | SK.  The group scales SQ by the nodes' gates in place and stage 2
+    // accumulates O on top of it; U lands over SK (dead by then).  The Gram block D2 is read out
+    // at the very start of an item's solve, so it cycles through a small ring of its own.
+    static constexpr int TM_COLS = 2 * NP;
+    static constexpr int TM_DO = 0, TM_DU = NP;
+    static constexpr int TM_GRAM = TBUF * TM_COLS;
+    static constexpr int GRAM_READERS = (2 * NP + 31) / 32 * 32;  // threads whose lanes hold [Q;K] rows
+    static_assert(TM_GRAM + GBUF * NP <= 512, "tensor memory");
 };
 
 // fused mode: what the commit of the previous round needs for one (sequence, head)
@@ -118,8 +132,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *ops_ready = mma1_done + C::TBUF;
     uint64_t *mma2_done = ops_ready + C::TBUF;
     uint64_t *tmem_free = mma2_done + C::TBUF;
-    uint64_t *v_ready = tmem_free + C::TBUF;
-    uint64_t *upd_done = v_ready + C::GROUPS;  // fused mode: the state tile of a stage carries the commit
+    uint64_t *gram_free = tmem_free + C::TBUF;
+    uint64_t *v_ready = gram_free + C::GBUF;
+    uint64_t *lists_ready = v_ready + C::GROUPS;  // group -> its solver warps: path lists written
+    uint64_t *t_done = lists_ready + C::GROUPS;   // solver warps -> group: rows of T / W written, lists read
+    uint64_t *upd_done = t_done + C::GROUPS;      // fused mode: the state tile of a stage carries the commit
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(upd_done + C::STAGES);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -131,11 +148,16 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         }
         for (int i = 0; i < C::TBUF; ++i) {
             ptx::mbar_init(&mma1_done[i], 1);
-            ptx::mbar_init(&ops_ready[i], VT_GROUP);
+            ptx::mbar_init(&ops_ready[i], VT_GROUP + C::TW);
             ptx::mbar_init(&mma2_done[i], 1);
             ptx::mbar_init(&tmem_free[i], VT_GROUP);
         }
-        for (int g = 0; g < C::GROUPS; ++g) ptx::mbar_init(&v_ready[g], 1);
+        for (int i = 0; i < C::GBUF; ++i) ptx::mbar_init(&gram_free[i], C::GRAM_READERS);
+        for (int g = 0; g < C::GROUPS; ++g) {
+            ptx::mbar_init(&v_ready[g], 1);
+            ptx::mbar_init(&lists_ready[g], VT_GROUP);
+            ptx::mbar_init(&t_done[g], C::TW);
+        }
         for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128);
         ptx::fence_barrier_init();
     }
@@ -152,6 +174,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     auto meta_L = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 8); };
     auto meta_beta = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 12); };
     auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
+    auto meta_rat = [&](unsigned char *stage) { return reinterpret_cast<float4 *>(stage + C::OFF_META + C::META_RAT); };
+    auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
 
     if (warp >= C::PROD_WARP0) {
         // ------------------------------------------------------------------ producer warp
@@ -168,6 +192,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             int item, b, h, lo, n, bad, flag;
             unsigned long long mk;
             float Lv, bv;
+            // path lists of the node this lane owns (first 8 ancestors), and whether any path is longer
+            float rat[8];
+            uint32_t iw[2];
+            int deep;
             // fused mode: the previous round's accepted path of this sequence
             int plo, pbad, plen, cnt, pj;
             unsigned long long pmask;
@@ -177,6 +205,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             Pre p;
             p.item = blockIdx.x + kk * gridDim.x;
             p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
+            p.deep = 0, p.iw[0] = 0u, p.iw[1] = 0u;
+#pragma unroll
+            for (int d = 0; d < 8; ++d) p.rat[d] = 0.f;
             p.plo = 0, p.pbad = 0, p.plen = -1, p.cnt = 0, p.pj = 0, p.pmask = 0ull, p.La = 0.f, p.wj = 0.f;
             if (p.item >= n_items) return p;
             p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
@@ -196,6 +227,21 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             p.mk = on ? a.anc_mask[p.lo + lane] : 0ull;
             p.Lv = on ? a.cum_log_gate[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
             p.bv = on ? a.beta[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
+            {
+                // Only the gate ratios depend on the head; building the lists here, a round ahead of
+                // their use, takes the ffs / exp chain off the consumers' critical path.
+                uint32_t m = (uint32_t)p.mk & ~(1u << lane);
+                p.deep = __any_sync(0xffffffffu, __popc(m) > 8);
+                p.iw[0] = 0u, p.iw[1] = 0u;
+#pragma unroll
+                for (int d = 0; d < 8; ++d) {
+                    const int j = m ? __ffs(m) - 1 : 0;
+                    const float Lj = __shfl_sync(0xffffffffu, p.Lv, j);
+                    p.rat[d] = m ? __expf(p.Lv - Lj) : 0.f;
+                    p.iw[d >> 2] |= (uint32_t)j << (8 * (d & 3));
+                    m &= m - 1;
+                }
+            }
             if constexpr (FUSED) {
                 p.plo = pv.node_offsets[p.b];
                 const int pn = pv.node_offsets[p.b + 1] - p.plo;
@@ -235,7 +281,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 break;
             }
             if (lane < NP) meta_mask(stage)[lane] = p.mk, meta_L(stage)[lane] = p.Lv, meta_beta(stage)[lane] = p.bv;
-            if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo;
+            if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep;
+            if (lane < NP) {
+                meta_rat(stage)[lane] = make_float4(p.rat[0], p.rat[1], p.rat[2], p.rat[3]);
+                meta_rat(stage)[NP + lane] = make_float4(p.rat[4], p.rat[5], p.rat[6], p.rat[7]);
+                meta_idx(stage)[lane] = p.iw[0], meta_idx(stage)[NP + lane] = p.iw[1];
+            }
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
@@ -381,11 +432,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int n = meta_nlo(stage)[0];
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
             if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
+            if (!ptx::mbar_wait(&gram_free[kk % C::GBUF], ((kk / C::GBUF) & 1) ^ 1)) break;
             ptx::tc_fence_after_sync();
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
-                    const uint32_t d1 = tmem_base + buf * C::TM_COLS, d2 = d1 + 2 * NP;
+                    const uint32_t d1 = tmem_base + buf * C::TM_COLS;
+                    const uint32_t d2 = tmem_base + C::TM_GRAM + (kk % C::GBUF) * NP;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks & 3) * 32;
@@ -437,7 +490,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
                             ptx::umma_tf32(dO, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
-                                      ptx::umma_desc_k_sw128(ww[p] + ks * 32), idesc, (p | ks) != 0);
+                                      ptx::umma_desc_k_sw128(ww[p] + ks * 32), idesc, true);  // on top of g.S0q
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
                 } else {
@@ -447,149 +500,72 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             __syncwarp();
         }
-    } else {
-        // ------------------------------------------------------------------ consumer groups
-        const int grp = warp >> 2, t = tid & (VT_GROUP - 1);
+    } else if (warp >= C::TW_WARP0 && warp < C::COMMIT_WARP0) {
+        // ------------------------------------------------------------------ solver warps
+        // Rows of T = (I + A)^-1 (one thread per node) and of W = P T (another) by back-substitution
+        // along node i's root path j_0 .. j_{dp-1}, j_dp = i:
+        //   x_dp = 1 (T) or P[i][i] (W);  x_e = p_e - sum_{f > e} x_f A[j_f][j_e]
+        // This needs shared memory only, so it runs beside the group's own work on R^T.
+        const int grp = (warp - C::TW_WARP0) / (C::TW / 32);
+        const int tt = tid - C::TW_WARP0 * 32 - grp * C::TW;
         unsigned char *gp = smem + C::OFF_GP + grp * C::GP_BYTES;
-        float *Ap = reinterpret_cast<float *>(gp + C::GP_AP);
-        float *Pp = reinterpret_cast<float *>(gp + C::GP_PP);
-        float4 *scal2 = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
-        unsigned char *idx = gp + C::GP_IDX;
-        TOut *Og = static_cast<TOut *>(a.O);
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
-
-        // Software pipeline: the front half of an item (lists, T / W rows, R^T -> ops_ready) is done
-        // before the back half (epilogue) of the group's previous item, so the stage-2 MMAs of
-        // one item run under the front half of the next.
-        int b_kk = -1, b_n = 0, b_lo = 0;  // the item whose back half is pending
-        bool dead = false;
-        for (int kk = grp; !dead; kk += C::GROUPS) {
+        const float4 *Ap4 = reinterpret_cast<const float4 *>(gp + C::GP_AP);
+        const float4 *Pp4 = reinterpret_cast<const float4 *>(gp + C::GP_PP);
+        const float4 *scal2 = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
+        const int i = tt & (NP - 1);
+        const bool wrow = (tt / NP) & 1;
+        for (int kk = grp;; kk += C::GROUPS) {
             const int item = blockIdx.x + kk * gridDim.x;
-            const bool have = item < n_items;
-            int f_n = 0, f_lo = 0;
-            if (have) {
+            if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
-            float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            const float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
-            if (!ptx::mbar_wait(&mma1_done[buf], (kk / C::TBUF) & 1)) {
-                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
-                dead = true;
-                break;
-            }
-            ptx::tc_fence_after_sync();
+            if (!ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1)) break;
             ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
             const int n = meta_nlo(stage)[0];
-            const int lo = meta_nlo(stage)[1];
-            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK | D2 (DO over SK, DU over D2)
-            if (t == 0) {  // the v rows of this item go to a free corner of the dead S0 tile
-                if (n > 0) {
-                    ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
-                    ptx::tma_load_2d(stage + C::OFF_VS, &tmV, (item % a.H_v) * D, lo, &v_ready[grp]);
-                } else {
-                    ptx::mbar_arrive(&v_ready[grp]);
-                }
-            }
-            if (n > 0) {
-                const unsigned long long *mask = meta_mask(stage);
-                const float *Lm = meta_L(stage);
-                float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
+            if (n > 0 && tt < 2 * NP && i < n) {
+                const bool deep = meta_nlo(stage)[2] != 0;
+                const float *Ap = reinterpret_cast<const float *>(stage + C::OFF_DAP);
+                const float *Pp = reinterpret_cast<const float *>(stage + C::OFF_DPP);
+                const unsigned char *idx = stage + C::OFF_DIDX;
                 float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
-                const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_VS);
-
-                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
-                for (int q = t; q < 4 * NP * 128 / 16; q += VT_GROUP)
-                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
-
-                // ---- phase G1: the rows of the Gram matrix leave tensor memory (row owner = lane)
-                if ((warp & 3) * 32 < 2 * NP) {  // warps whose lanes hold [Q;K] rows
-#pragma unroll
-                    for (int c0 = 0; c0 < NP; c0 += 16) {
-                        if (c0 < n) {
-                            uint32_t g[16];
-                            ptx::tmem_ld16(tm + 2 * NP + c0, g);
-                            ptx::tmem_wait_ld();
-                            if (t < 2 * NP) {
-                                float4 *dst = reinterpret_cast<float4 *>(raw + t * C::RLD + c0);
-#pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
-                                                         __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
-                            }
-                        }
-                    }
-                }
-                ptx::named_sync(1 + grp, VT_GROUP);
-
-                // ---- phase G2: scaled ancestor lists, PARTS threads per node, a few entries each
-                //   P[i][d] = e^{L_i-L_j} q_i.k_j ,  A[i][d] = beta_i e^{L_i-L_j} k_i.k_j ,  idx[i][d] = j
-                //   for j the d-th ancestor of i; lists are stored [d / 4][node][d % 4]
-                constexpr int HALF = C::PARTS / 2;
-                const int i = t & (NP - 1), part = t / NP;
-                const bool valid = i < n;
-                const bool a_kind = part >= HALF;
-                const int sub = a_kind ? part - HALF : part;
-                const uint32_t mi = valid ? (uint32_t)mask[i] : 0u;
-                const int dp = valid ? __popc(mi) - 1 : 0;  // ancestors of node i
-                const float Li = Lm[i];
-                const float bi = meta_beta(stage)[i];
-                {
-                    const float scale = a_kind ? bi : 1.f;
-                    const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
-                    uint32_t m = mi & ~(1u << i);
-                    for (int q = 0; q < sub; ++q) m &= m - 1;
-                    for (int d = sub; d < dp; d += HALF) {
-                        const int j = __ffs(m) - 1;
-                        const float val = scale * __expf(Li - Lm[j]) * row[j];
-                        const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
-                        if (a_kind) Ap[at] = val;
-                        else Pp[at] = val, idx[at] = (unsigned char)j;
-#pragma unroll
-                        for (int q = 0; q < HALF; ++q) m &= m - 1;
-                    }
-                    if (part == 0 && valid) {
-                        const float gi = __expf(Li);
-                        scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
-                    }
-                }
-                // lists, scalars and the zero fill are in place; learn whether any path is deep
-                const bool deep = ptx::named_sync_or(1 + grp, VT_GROUP, dp > 8);
-
-                // ---- phase T: rows of T = (I + A)^-1 (one thread) and W = P T (another) by
-                // back-substitution along node i's root path j_0 .. j_{dp-1}, j_dp = i:
-                //   x_dp = 1 (T) or P[i][i] (W);  x_e = p_e - sum_{f > e} x_f A[j_f][j_e]
-                if (valid && sub == 0) {
-                    const bool wrow = !a_kind;
+                const int dp = __popc((uint32_t)meta_mask(stage)[i]) - 1;  // ancestors of node i
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
-                    if (!deep) {  // registers only; every load is unconditional (all addresses are valid)
-                                  // and masked by a select, so the phase has no branches
+                    if (!deep) {  // registers only, no branches: entries beyond the path are zeros
+                        const uint32_t iw0 = meta_idx(stage)[i], iw1 = meta_idx(stage)[NP + i];
                         int jf[9];
                         float x[9], pe[8], co[9][8];
 #pragma unroll
-                        for (int e = 0; e < 9; ++e) {
-                            const int ee = e < 8 ? e : 7;
-                            const int j = idx[((ee >> 2) * NP + i) * 4 + (ee & 3)];
+                        for (int e = 0; e < 8; ++e) {
+                            const int j = ((e < 4 ? iw0 : iw1) >> (8 * (e & 3))) & 255u;
                             jf[e] = e < dp ? j : i;
-                            x[e] = e == dp ? top : 0.f;
+                            x[e] = 0.f;
+                        }
+                        jf[8] = i, x[8] = dp == 8 ? top : 0.f;
+                        {
+                            const float4 p0 = Pp4[i], p1 = Pp4[NP + i];
+                            pe[0] = p0.x, pe[1] = p0.y, pe[2] = p0.z, pe[3] = p0.w;
+                            pe[4] = p1.x, pe[5] = p1.y, pe[6] = p1.z, pe[7] = p1.w;
                         }
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float pv = Pp[((e >> 2) * NP + i) * 4 + (e & 3)];
-                            pe[e] = (wrow && e < dp) ? pv : 0.f;
-#pragma unroll
-                            for (int f = e + 1; f < 9; ++f) {
-                                const float cv = Ap[((e >> 2) * NP + jf[f]) * 4 + (e & 3)];
-                                co[f][e] = f <= dp ? cv : 0.f;
+                        for (int f = 1; f < 9; ++f) {  // A-list of the path node at depth f
+                            const float4 c0 = Ap4[jf[f]];
+                            co[f][0] = c0.x, co[f][1] = c0.y, co[f][2] = c0.z, co[f][3] = c0.w;
+                            if (f > 4) {
+                                const float4 c1 = Ap4[NP + jf[f]];
+                                co[f][4] = c1.x, co[f][5] = c1.y, co[f][6] = c1.z, co[f][7] = c1.w;
                             }
                         }
+                        // x_f = 0 beyond the path, so the lists of the padding entries (node i itself)
+                        // contribute nothing; only the diagonal entry e = dp must keep its value
 #pragma unroll
                         for (int e = 7; e >= 0; --e) {
-                            float acc = pe[e];
+                            float acc = wrow ? pe[e] : 0.f;
 #pragma unroll
                             for (int f = e + 1; f < 9; ++f) acc = fmaf(-x[f], co[f][e], acc);
-                            x[e] = e < dp ? acc : x[e];
+                            x[e] = e == dp ? top : acc;
                         }
                         // entries beyond the path all aim at the diagonal and carry 0; going down from
                         // e = 8 the real diagonal entry (e = dp) is written after them
@@ -621,14 +597,171 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                             *reinterpret_cast<float *>(Mlo + off) = val - hi;
                         }
                     }
-                }
+            }
+            ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
+            ptx::mbar_arrive(&t_done[grp]);
+            ptx::mbar_arrive(&ops_ready[buf]);
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer groups
+        const int grp = warp >> 2, t = tid & (VT_GROUP - 1);
+        unsigned char *gp = smem + C::OFF_GP + grp * C::GP_BYTES;
+        float4 *Ap4 = reinterpret_cast<float4 *>(gp + C::GP_AP);
+        float4 *Pp4 = reinterpret_cast<float4 *>(gp + C::GP_PP);
+        float4 *scal2 = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
+        const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
+        TOut *Og = static_cast<TOut *>(a.O);
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
 
-                // this thread's column of the v rows leaves the S0 tile before R^T lands on it
+        // Software pipeline: the front half of an item (lists, T / W rows, R^T -> ops_ready) is done
+        // before the back half (epilogue) of the group's previous item, so the stage-2 MMAs of
+        // one item run under the front half of the next.
+        int b_kk = -1, b_n = 0, b_lo = 0;  // the item whose back half is pending
+        bool dead = false;
+        // The v rows of the group's NEXT item are fetched as soon as the current ones have been
+        // read (thread 0 of the group; the first packed node is looked up one item further ahead,
+        // so the fetch never waits on node_offsets).  Rows past a tree's end belong to other
+        // sequences or are zero fill: they are loaded and never used.
+        int v_pending = -1;  // thread 0: the item whose v rows are in flight or unread
+        auto first_node = [&](int kx) {
+            const int it = blockIdx.x + kx * gridDim.x;
+            return it < n_items ? a.node_offsets[it / a.H_v] : 0;
+        };
+        auto fetch_v = [&](int kx, int lo_x) {
+            const int it = blockIdx.x + kx * gridDim.x;
+            v_pending = -1;
+            if (it >= n_items) return;
+            v_pending = kx;
+            ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
+            ptx::tma_load_2d(gp + C::GP_VS, &tmV, (it % a.H_v) * D, lo_x, &v_ready[grp]);
+        };
+        int v_lo_next = 0;
+        if (t == 0) {
+            ptx::prefetch_tmap(&tmV);
+            fetch_v(grp, first_node(grp));
+            v_lo_next = first_node(grp + C::GROUPS);
+        }
+        for (int kk = grp; !dead; kk += C::GROUPS) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            const bool have = item < n_items;
+            int f_n = 0, f_lo = 0;
+            if (have) {
+            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+            float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            if (!ptx::mbar_wait(&mma1_done[buf], (kk / C::TBUF) & 1)) {
+                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                dead = true;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
+            const int n = meta_nlo(stage)[0];
+            const int lo = meta_nlo(stage)[1];
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK  (O over SQ, U over SK)
+            const uint32_t tg = tmem_base + lane_base + C::TM_GRAM + (kk % C::GBUF) * NP;
+            const bool gram_reader = (warp & 3) * 32 < 2 * NP;  // warps whose lanes hold [Q;K] rows
+            if (n > 0) {
+                const unsigned long long *mask = meta_mask(stage);
+                const float *Lm = meta_L(stage);
+                float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
+                float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
+                const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
+                float *Ap = deep ? reinterpret_cast<float *>(stage + C::OFF_DAP) : reinterpret_cast<float *>(Ap4);
+                float *Pp = deep ? reinterpret_cast<float *>(stage + C::OFF_DPP) : reinterpret_cast<float *>(Pp4);
+                unsigned char *idx = stage + C::OFF_DIDX;
+
+                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
+                for (int q = t; q < 4 * NP * 128 / 16; q += VT_GROUP)
+                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
+
+                // ---- phase G1: the rows of the Gram matrix leave tensor memory (row owner = lane)
+                if (gram_reader) {
+#pragma unroll
+                    for (int c0 = 0; c0 < NP; c0 += 16) {
+                        if (c0 < n) {
+                            uint32_t g[16];
+                            ptx::tmem_ld16(tg + c0, g);
+                            ptx::tmem_wait_ld();
+                            if (t < 2 * NP) {
+                                float4 *dst = reinterpret_cast<float4 *>(raw + t * C::RLD + c0);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
+                                                         __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
+                            }
+                        }
+                    }
+                }
+                if (gram_reader) {
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive(&gram_free[kk % C::GBUF]);
+                }
+                ptx::named_sync(1 + grp, VT_GROUP);
+
+                // ---- phase G2: scaled ancestor lists
+                //   P[i][d] = e^{L_i-L_j} q_i.k_j ,  A[i][d] = beta_i e^{L_i-L_j} k_i.k_j ,  idx[i][d] = j
+                //   for j the d-th ancestor of i; lists are stored [d / 4][node][d % 4]
+                constexpr int HALF = C::PARTS / 2;
+                const int i = t & (NP - 1), part = t / NP;
+                const bool valid = i < n;
+                const bool a_kind = part >= HALF;
+                const int sub = a_kind ? part - HALF : part;
+                const uint32_t mi = valid ? (uint32_t)mask[i] : 0u;
+                const int dp = valid ? __popc(mi) - 1 : 0;  // ancestors of node i
+                const float Li = Lm[i];
+                const float bi = meta_beta(stage)[i];
+                // the solver warps must have read the previous item's lists
+                if (kk >= C::GROUPS) ptx::mbar_wait(&t_done[grp], ((kk / C::GROUPS) - 1) & 1);
+                if (!deep) {
+                    // the producer left indices and gate ratios of the first 8 ancestors: one thread
+                    // scales four Gram entries, no dependent chain
+                    if (sub < 2) {
+                        const float scale = a_kind ? bi : 1.f;
+                        const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
+                        const uint32_t iw = meta_idx(stage)[sub * NP + i];
+                        const float4 rt = meta_rat(stage)[sub * NP + i];
+                        float4 val;
+                        val.x = scale * rt.x * row[iw & 255u], val.y = scale * rt.y * row[(iw >> 8) & 255u];
+                        val.z = scale * rt.z * row[(iw >> 16) & 255u], val.w = scale * rt.w * row[iw >> 24];
+                        (a_kind ? Ap4 : Pp4)[sub * NP + i] = val;
+                    }
+                } else {
+                    const float scale = a_kind ? bi : 1.f;
+                    const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
+                    uint32_t m = mi & ~(1u << i);
+                    for (int q = 0; q < sub; ++q) m &= m - 1;
+                    for (int d = sub; d < dp; d += HALF) {
+                        const int j = __ffs(m) - 1;
+                        const float val = scale * __expf(Li - Lm[j]) * row[j];
+                        const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
+                        if (a_kind) Ap[at] = val;
+                        else Pp[at] = val, idx[at] = (unsigned char)j;
+#pragma unroll
+                        for (int q = 0; q < HALF; ++q) m &= m - 1;
+                    }
+                }
+                if (part == 0 && valid) {
+                    const float gi = __expf(Li);
+                    scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
+                }
+                ptx::mbar_arrive(&lists_ready[grp]);  // lists, scalars and the zero fill are in place
+
+                // this thread's column of the v rows; once every thread has its copy the buffer takes
+                // the rows of the group's next item.  The barrier also keeps R^T off the Gram stash
+                // until every thread has built its list entries, and, with deep paths, off the scratch
+                // (lists, back-substitution rows) the solver warps are still reading.
                 ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);
                 __nv_bfloat16 vreg[NP];
 #pragma unroll
                 for (int j = 0; j < NP; ++j) vreg[j] = vs[j * D + t];
-                ptx::named_sync(1 + grp, VT_GROUP);
+                if (deep) ptx::mbar_wait(&t_done[grp], (kk / C::GROUPS) & 1);
+                ptx::named_sync(5 + grp, VT_GROUP);
+                if (t == 0) {
+                    fetch_v(kk + C::GROUPS, v_lo_next);
+                    v_lo_next = first_node(kk + 2 * C::GROUPS);
+                }
 
                 // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo
                 float r[32];
@@ -666,7 +799,31 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         *reinterpret_cast<float4 *>(row_lo + off) = lo;
                     }
                 }
+                // g_j (S0 q_j) in place: stage 2 accumulates the rest of o_j on top of it
+#pragma unroll
+                for (int c0 = 0; c0 < NP; c0 += 16) {
+                    if (c0 < n) {
+                        uint32_t sq[16];
+                        ptx::tmem_ld16(tm + c0, sq);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            sq[jj] = __float_as_uint(scal[c0 + jj].z * __uint_as_float(sq[jj]));
+                        ptx::tmem_st16(tm + c0, sq);
+                    }
+                }
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before_sync();
                 ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
+            } else {
+                if (gram_reader) ptx::mbar_arrive(&gram_free[kk % C::GBUF]);
+                if (kk >= C::GROUPS) ptx::mbar_wait(&t_done[grp], ((kk / C::GROUPS) - 1) & 1);
+                ptx::mbar_arrive(&lists_ready[grp]);
+                ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);  // rows of a skipped item: unused
+                if (t == 0) {
+                    fetch_v(kk + C::GROUPS, v_lo_next);
+                    v_lo_next = first_node(kk + 2 * C::GROUPS);
+                }
             }
             ptx::mbar_arrive(&ops_ready[buf]);
             f_n = n, f_lo = lo;
@@ -676,7 +833,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int kk = b_kk, n = b_n, lo = b_lo;
             const int item = blockIdx.x + kk * gridDim.x, h = item % a.H_v;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
-            const float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;
             if (!ptx::mbar_wait(&mma2_done[buf], (kk / C::TBUF) & 1)) {
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
@@ -684,23 +840,21 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             ptx::tc_fence_after_sync();
             if (n > 0) {
-                // ---- epilogue: u_i = DU[i], o_i = g_i (S0 q_i) + DO[i]
+                // ---- epilogue: u_i and o_i leave tensor memory
                 float *Ub = a.U + ((size_t)lo * a.H_v + h) * D + t;
                 TOut *Ob = Og + ((size_t)lo * a.H_v + h) * D + t;
 #pragma unroll
                 for (int c0 = 0; c0 < NP; c0 += 16) {
                     if (c0 < n) {
-                        uint32_t du[16], dout[16], sq[16];
+                        uint32_t du[16], dout[16];
                         ptx::tmem_ld16(tm + C::TM_DU + c0, du);
                         ptx::tmem_ld16(tm + C::TM_DO + c0, dout);
-                        ptx::tmem_ld16(tm + c0, sq);
                         ptx::tmem_wait_ld();
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int node = c0 + jj;
-                            const float o = fmaf(scal[node].z, __uint_as_float(sq[jj]), __uint_as_float(dout[jj]));
                             st_global_if(Ub + node * rs, __uint_as_float(du[jj]), node < n);
-                            st_global_if(Ob + node * rs, o, node < n);
+                            st_global_if(Ob + node * rs, __uint_as_float(dout[jj]), node < n);
                         }
                     }
                 }
@@ -711,6 +865,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (!have) break;
             b_kk = kk, b_n = f_n, b_lo = f_lo;
         }
+        // after a give-up a fetch may still be in flight: it must land before the CTA exits
+        if (t == 0 && v_pending >= 0) ptx::mbar_wait(&v_ready[grp], (v_pending / C::GROUPS) & 1);
     }
 
     // common exit: tensor memory goes back once every role is done with it
