@@ -46,8 +46,8 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int GROUPS = 2;
     static constexpr int STAGES = FUSED ? 3 : 4;
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
-    static constexpr int TBUF = 6;  // TMEM buffers: stage-1 MMAs run well ahead of the groups' solves
-    static constexpr int GBUF = 4;  // ... and a ring of short-lived Gram blocks
+    static constexpr int TBUF = 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
+    static constexpr int RBUF = 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
     static constexpr int CONSUMERS = VT_GROUP * GROUPS;
     static constexpr int TW = 64;  // threads of a group's solver warps (one per row of T and of W)
     static constexpr int TW_WARP0 = CONSUMERS / 32;
@@ -74,9 +74,9 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
     static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
     // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
-    static constexpr int OFF_T_HI = 0, OFF_T_LO = NP * 128, OFF_W_HI = 2 * NP * 128, OFF_W_LO = 3 * NP * 128;
-    static constexpr int OFF_RT_HI = OFF_S0, OFF_RT_LO = OFF_S0 + D * 128;
-    static_assert(4 * NP * 128 <= QK_BYTES && 2 * D * 128 <= S0_BYTES, "operand overlays fit");
+    // (W rows above T rows: [W;T] is one B operand of 2 NP rows, so one MMA yields O and U together)
+    static constexpr int OFF_W_HI = 0, OFF_T_HI = NP * 128, OFF_W_LO = 2 * NP * 128, OFF_T_LO = 3 * NP * 128;
+    static_assert(4 * NP * 128 <= QK_BYTES, "operand overlays fit");
     // scratch over the dead S0 tile, used before R^T is written there: the raw Gram rows and the
     // back-substitution rows of deep paths
     static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
@@ -95,16 +95,18 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + GBUF + 3 * GROUPS) * 8 + 16 + 1024;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * GROUPS) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
-    // per TMEM buffer: SQ | SK.  The group scales SQ by the nodes' gates in place and stage 2
-    // accumulates O on top of it; U lands over SK (dead by then).  The Gram block D2 is read out
-    // at the very start of an item's solve, so it cycles through a small ring of its own.
+    // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the group
+    // turns it, in its own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
+    // epilogue frees it.  A block of the second takes the Gram block D2 from stage 1; the group
+    // reads it out, writes R^T (hi) over it and R^T (lo) behind it, stage 2 takes both as its A
+    // operand, and its completion frees the block (long before the epilogue runs).
     static constexpr int TM_COLS = 2 * NP;
     static constexpr int TM_DO = 0, TM_DU = NP;
-    static constexpr int TM_GRAM = TBUF * TM_COLS;
-    static constexpr int GRAM_READERS = (2 * NP + 31) / 32 * 32;  // threads whose lanes hold [Q;K] rows
-    static_assert(TM_GRAM + GBUF * NP <= 512, "tensor memory");
+    static constexpr int TM_R0 = TBUF * TM_COLS;  // second ring
+    static constexpr int TM_RHI = 0, TM_RLO = NP;
+    static_assert(TM_R0 + RBUF * 2 * NP <= 512, "tensor memory");
 };
 
 // fused mode: what the commit of the previous round needs for one (sequence, head)
@@ -132,9 +134,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *ops_ready = mma1_done + C::TBUF;
     uint64_t *mma2_done = ops_ready + C::TBUF;
     uint64_t *tmem_free = mma2_done + C::TBUF;
-    uint64_t *gram_free = tmem_free + C::TBUF;
-    uint64_t *v_ready = gram_free + C::GBUF;
-    uint64_t *lists_ready = v_ready + C::GROUPS;  // group -> its solver warps: path lists written
+    uint64_t *r_free = tmem_free + C::TBUF;
+    uint64_t *v_ready = r_free + C::RBUF;
+    uint64_t *v_free = v_ready + C::GROUPS;       // group -> its solver warps: v rows copied to registers
+    uint64_t *lists_ready = v_free + C::GROUPS;   // group -> its solver warps: path lists written
     uint64_t *t_done = lists_ready + C::GROUPS;   // solver warps -> group: rows of T / W written, lists read
     uint64_t *upd_done = t_done + C::GROUPS;      // fused mode: the state tile of a stage carries the commit
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(upd_done + C::STAGES);
@@ -152,9 +155,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&mma2_done[i], 1);
             ptx::mbar_init(&tmem_free[i], VT_GROUP);
         }
-        for (int i = 0; i < C::GBUF; ++i) ptx::mbar_init(&gram_free[i], C::GRAM_READERS);
+        for (int i = 0; i < C::RBUF; ++i) ptx::mbar_init(&r_free[i], 1);
         for (int g = 0; g < C::GROUPS; ++g) {
             ptx::mbar_init(&v_ready[g], 1);
+            ptx::mbar_init(&v_free[g], VT_GROUP);
             ptx::mbar_init(&lists_ready[g], VT_GROUP);
             ptx::mbar_init(&t_done[g], C::TW);
         }
@@ -432,13 +436,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int n = meta_nlo(stage)[0];
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
             if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
-            if (!ptx::mbar_wait(&gram_free[kk % C::GBUF], ((kk / C::GBUF) & 1) ^ 1)) break;
+            if (!ptx::mbar_wait(&r_free[kk % C::RBUF], ((kk / C::RBUF) & 1) ^ 1)) break;
             ptx::tc_fence_after_sync();
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
                     const uint32_t d1 = tmem_base + buf * C::TM_COLS;
-                    const uint32_t d2 = tmem_base + C::TM_GRAM + (kk % C::GBUF) * NP;
+                    const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks & 3) * 32;
@@ -462,7 +466,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         }
     } else if (warp == C::MMA2_WARP) {
         // ------------------------------------------------------------------ stage-2 MMAs
-        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, NP);
+        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -474,28 +478,22 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
-                    const uint32_t dU = tmem_base + buf * C::TM_COLS + C::TM_DU;
-                    const uint32_t dO = tmem_base + buf * C::TM_COLS + C::TM_DO;
-                    const uint32_t rt[3] = {base + C::OFF_RT_HI, base + C::OFF_RT_LO, base + C::OFF_RT_HI};
-                    const uint32_t tt[3] = {base + C::OFF_T_HI, base + C::OFF_T_HI, base + C::OFF_T_LO};
-                    const uint32_t ww[3] = {base + C::OFF_W_HI, base + C::OFF_W_HI, base + C::OFF_W_LO};
+                    const uint32_t tb = tmem_base + buf * C::TM_COLS;
+                    const uint32_t tr = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
+                    const uint32_t ra[3] = {tr + C::TM_RHI, tr + C::TM_RLO, tr + C::TM_RHI};
+                    const uint32_t wt[3] = {base + C::OFF_W_HI, base + C::OFF_W_HI, base + C::OFF_W_LO};
 #pragma unroll
                     for (int p = 0; p < 3; ++p)
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            ptx::umma_tf32(dU, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
-                                      ptx::umma_desc_k_sw128(tt[p] + ks * 32), idesc, (p | ks) != 0);
-#pragma unroll
-                    for (int p = 0; p < 3; ++p)
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            ptx::umma_tf32(dO, ptx::umma_desc_k_sw128(rt[p] + ks * 32),
-                                      ptx::umma_desc_k_sw128(ww[p] + ks * 32), idesc, true);  // on top of g.S0q
+                        for (int ks = 0; ks < NP / 8; ++ks)  // on top of g.S0q (O) and zeros (U)
+                            ptx::umma_tf32_ts(tb, ra[p] + ks * 8, ptx::umma_desc_k_sw128(wt[p] + ks * 32), idesc, 1u);
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
+                    ptx::umma_commit(&r_free[kk % C::RBUF]);
                 } else {
                     ptx::mbar_arrive(&mma2_done[buf]);
                     ptx::mbar_arrive(&empty[s]);
+                    ptx::mbar_arrive(&r_free[kk % C::RBUF]);
                 }
             }
             __syncwarp();
@@ -514,13 +512,41 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const float4 *scal2 = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
         const int i = tt & (NP - 1);
         const bool wrow = (tt / NP) & 1;
+        // The v rows of the group's NEXT item are fetched (last thread of the solver warps) as soon
+        // as the group has copied the current ones to registers; the first packed node is looked
+        // up one item further ahead, so the fetch never waits on node_offsets.  Rows past a tree's
+        // end belong to other sequences or are zero fill: they are loaded and never used.
+        int v_pending = -1;  // the item whose v rows are in flight or unread
+        auto first_node = [&](int kx) {
+            const int it = blockIdx.x + kx * gridDim.x;
+            return it < n_items ? a.node_offsets[it / a.H_v] : 0;
+        };
+        auto fetch_v = [&](int kx, int lo_x) {
+            const int it = blockIdx.x + kx * gridDim.x;
+            v_pending = -1;
+            if (it >= n_items) return;
+            v_pending = kx;
+            ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
+            ptx::tma_load_2d(gp + C::GP_VS, &tmV, (it % a.H_v) * D, lo_x, &v_ready[grp]);
+        };
+        int v_lo_next = 0;
+        const bool v_thread = tt == C::TW - 1;
+        if (v_thread) {
+            ptx::prefetch_tmap(&tmV);
+            fetch_v(grp, first_node(grp));
+            v_lo_next = first_node(grp + C::GROUPS);
+        }
+        bool gave_up = false;
         for (int kk = grp;; kk += C::GROUPS) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
             const float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
-            if (!ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1)) break;
+            if (!ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1)) {
+                gave_up = true;
+                break;
+            }
             ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
             const int n = meta_nlo(stage)[0];
             if (n > 0 && tt < 2 * NP && i < n) {
@@ -601,7 +627,17 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
             ptx::mbar_arrive(&t_done[grp]);
             ptx::mbar_arrive(&ops_ready[buf]);
+            if (v_thread) {
+                if (!ptx::mbar_wait(&v_free[grp], (kk / C::GROUPS) & 1)) {
+                    gave_up = true;
+                    break;
+                }
+                fetch_v(kk + C::GROUPS, v_lo_next);
+                v_lo_next = first_node(kk + 2 * C::GROUPS);
+            }
         }
+        // after a give-up a fetch may still be in flight: it must land before the CTA exits
+        if (v_thread && gave_up && v_pending >= 0) ptx::mbar_wait(&v_ready[grp], (v_pending / C::GROUPS) & 1);
     } else {
         // ------------------------------------------------------------------ consumer groups
         const int grp = warp >> 2, t = tid & (VT_GROUP - 1);
@@ -619,29 +655,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // one item run under the front half of the next.
         int b_kk = -1, b_n = 0, b_lo = 0;  // the item whose back half is pending
         bool dead = false;
-        // The v rows of the group's NEXT item are fetched as soon as the current ones have been
-        // read (thread 0 of the group; the first packed node is looked up one item further ahead,
-        // so the fetch never waits on node_offsets).  Rows past a tree's end belong to other
-        // sequences or are zero fill: they are loaded and never used.
-        int v_pending = -1;  // thread 0: the item whose v rows are in flight or unread
-        auto first_node = [&](int kx) {
-            const int it = blockIdx.x + kx * gridDim.x;
-            return it < n_items ? a.node_offsets[it / a.H_v] : 0;
-        };
-        auto fetch_v = [&](int kx, int lo_x) {
-            const int it = blockIdx.x + kx * gridDim.x;
-            v_pending = -1;
-            if (it >= n_items) return;
-            v_pending = kx;
-            ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
-            ptx::tma_load_2d(gp + C::GP_VS, &tmV, (it % a.H_v) * D, lo_x, &v_ready[grp]);
-        };
-        int v_lo_next = 0;
-        if (t == 0) {
-            ptx::prefetch_tmap(&tmV);
-            fetch_v(grp, first_node(grp));
-            v_lo_next = first_node(grp + C::GROUPS);
-        }
         for (int kk = grp; !dead; kk += C::GROUPS) {
             const int item = blockIdx.x + kk * gridDim.x;
             const bool have = item < n_items;
@@ -659,8 +672,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
             const int n = meta_nlo(stage)[0];
             const int lo = meta_nlo(stage)[1];
-            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK  (O over SQ, U over SK)
-            const uint32_t tg = tmem_base + lane_base + C::TM_GRAM + (kk % C::GBUF) * NP;
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK
+            const uint32_t tr = tmem_base + lane_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;  // D2 | -
             const bool gram_reader = (warp & 3) * 32 < 2 * NP;  // warps whose lanes hold [Q;K] rows
             if (n > 0) {
                 const unsigned long long *mask = meta_mask(stage);
@@ -682,7 +695,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     for (int c0 = 0; c0 < NP; c0 += 16) {
                         if (c0 < n) {
                             uint32_t g[16];
-                            ptx::tmem_ld16(tg + c0, g);
+                            ptx::tmem_ld16(tr + c0, g);
                             ptx::tmem_wait_ld();
                             if (t < 2 * NP) {
                                 float4 *dst = reinterpret_cast<float4 *>(raw + t * C::RLD + c0);
@@ -693,10 +706,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                             }
                         }
                     }
-                }
-                if (gram_reader) {
-                    ptx::tc_fence_before_sync();
-                    ptx::mbar_arrive(&gram_free[kk % C::GBUF]);
                 }
                 ptx::named_sync(1 + grp, VT_GROUP);
 
@@ -748,82 +757,56 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
                 ptx::mbar_arrive(&lists_ready[grp]);  // lists, scalars and the zero fill are in place
 
-                // this thread's column of the v rows; once every thread has its copy the buffer takes
-                // the rows of the group's next item.  The barrier also keeps R^T off the Gram stash
-                // until every thread has built its list entries, and, with deep paths, off the scratch
-                // (lists, back-substitution rows) the solver warps are still reading.
+                // this thread's column of the v rows; once every thread has its copy a solver warp
+                // fetches the rows of the group's next item into the buffer
                 ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);
                 __nv_bfloat16 vreg[NP];
 #pragma unroll
                 for (int j = 0; j < NP; ++j) vreg[j] = vs[j * D + t];
-                if (deep) ptx::mbar_wait(&t_done[grp], (kk / C::GROUPS) & 1);
-                ptx::named_sync(5 + grp, VT_GROUP);
-                if (t == 0) {
-                    fetch_v(kk + C::GROUPS, v_lo_next);
-                    v_lo_next = first_node(kk + 2 * C::GROUPS);
-                }
+                ptx::mbar_arrive(&v_free[grp]);
+                // the per-node scalars were written by other threads of the group
+                ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1);
 
-                // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo
-                float r[32];
+                // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo, stays in
+                // tensor memory (the A operand of stage 2); g_j (S0 q_j) in place and zeros over S0 k_j
+                // are what stage 2 accumulates o_j and u_j on
 #pragma unroll
-                for (int c0 = 0; c0 < 32; c0 += 16) {
-                    if (c0 < NP && c0 < n) {
-                        uint32_t sk[16];
+                for (int c0 = 0; c0 < NP; c0 += 16) {
+                    uint32_t hi[16], lo[16];
+                    if (c0 < n) {
+                        uint32_t sk[16], sq[16];
                         ptx::tmem_ld16(tm + NP + c0, sk);
+                        ptx::tmem_ld16(tm + c0, sq);
                         ptx::tmem_wait_ld();
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int j = c0 + jj;
-                            const float4 sc = scal[j < NP ? j : 0];
-                            const float v = __bfloat162float(vreg[j < NP ? j : 0]);
+                            const float4 sc = scal[j];
+                            const float v = __bfloat162float(vreg[j]);
                             const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v);
-                            r[j] = j < n ? val : 0.f;
+                            const float rj = j < n ? val : 0.f;
+                            const float h = ptx::tf32_hi(rj);
+                            hi[jj] = __float_as_uint(h), lo[jj] = __float_as_uint(rj - h);
+                            sq[jj] = __float_as_uint(sc.z * __uint_as_float(sq[jj]));
+                            sk[jj] = 0u;
                         }
+                        ptx::tmem_st16(tm + c0, sq);
+                        ptx::tmem_st16(tm + NP + c0, sk);
                     } else {
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) r[c0 + jj] = 0.f;
+                        for (int jj = 0; jj < 16; ++jj) hi[jj] = 0u, lo[jj] = 0u;
                     }
-                }
-                {
-                    unsigned char *row_hi = stage + C::OFF_RT_HI + t * 128;
-                    unsigned char *row_lo = stage + C::OFF_RT_LO + t * 128;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        float4 hi, lo;
-                        hi.x = ptx::tf32_hi(r[4 * q]), hi.y = ptx::tf32_hi(r[4 * q + 1]);
-                        hi.z = ptx::tf32_hi(r[4 * q + 2]), hi.w = ptx::tf32_hi(r[4 * q + 3]);
-                        lo.x = r[4 * q] - hi.x, lo.y = r[4 * q + 1] - hi.y;
-                        lo.z = r[4 * q + 2] - hi.z, lo.w = r[4 * q + 3] - hi.w;
-                        const int off = ((q ^ (t & 7)) << 4);
-                        *reinterpret_cast<float4 *>(row_hi + off) = hi;
-                        *reinterpret_cast<float4 *>(row_lo + off) = lo;
-                    }
-                }
-                // g_j (S0 q_j) in place: stage 2 accumulates the rest of o_j on top of it
-#pragma unroll
-                for (int c0 = 0; c0 < NP; c0 += 16) {
-                    if (c0 < n) {
-                        uint32_t sq[16];
-                        ptx::tmem_ld16(tm + c0, sq);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj)
-                            sq[jj] = __float_as_uint(scal[c0 + jj].z * __uint_as_float(sq[jj]));
-                        ptx::tmem_st16(tm + c0, sq);
-                    }
+                    ptx::tmem_st16(tr + C::TM_RHI + c0, hi);
+                    ptx::tmem_st16(tr + C::TM_RLO + c0, lo);
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
             } else {
-                if (gram_reader) ptx::mbar_arrive(&gram_free[kk % C::GBUF]);
                 if (kk >= C::GROUPS) ptx::mbar_wait(&t_done[grp], ((kk / C::GROUPS) - 1) & 1);
                 ptx::mbar_arrive(&lists_ready[grp]);
                 ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);  // rows of a skipped item: unused
-                if (t == 0) {
-                    fetch_v(kk + C::GROUPS, v_lo_next);
-                    v_lo_next = first_node(kk + 2 * C::GROUPS);
-                }
+                ptx::mbar_arrive(&v_free[grp]);
             }
             ptx::mbar_arrive(&ops_ready[buf]);
             f_n = n, f_lo = lo;
@@ -865,8 +848,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (!have) break;
             b_kk = kk, b_n = f_n, b_lo = f_lo;
         }
-        // after a give-up a fetch may still be in flight: it must land before the CTA exits
-        if (t == 0 && v_pending >= 0) ptx::mbar_wait(&v_ready[grp], (v_pending / C::GROUPS) & 1);
     }
 
     // common exit: tensor memory goes back once every role is done with it
