@@ -65,14 +65,20 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t *bar, uint32_t par
 }
 // Bounded wait: false when the phase did not complete within about two seconds of SM clocks,
 // so a kernel can raise a status bit and leave instead of hanging the GPU.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// (the slow path is kept out of line: the kernels wait in dozens of places and their code has to
+// stay small enough for the instruction cache)
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
         if (clock64() - t0 > 4000000000ll) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity);
 }
 
 // ----------------------------------------------------------------------------- bulk copies
@@ -266,6 +272,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
+                 "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 

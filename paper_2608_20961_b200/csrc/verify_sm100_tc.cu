@@ -2,7 +2,7 @@
 // read-out), with BOTH contractions of the method on the tcgen05 tensor cores:
 //
 //   stage 1 (bf16 x bf16 -> fp32):   D1 = S0 [Q;K]^T  (S0 q_i, S0 k_i),   D2 = [Q;K] K^T  (Gram)
-//   stage 2 (tf32 split, ~fp32):     U^T = R^T T^T ,   (O - g.S0q)^T = R^T W^T
+//   stage 2 (tf32 split, ~fp32):     [O | U]^T = [g.S0q | 0]^T + R^T [W;T]^T
 //
 // where R[j] = beta_j (v_j - g_j S0 k_j) is the right-hand side of Eq. 2, T = (I + A)^{-1} and
 // W = P T.  The triangular system is not solved column by column: because A only couples a
@@ -16,16 +16,30 @@
 // bits cleared (exactly representable in tf32) and lo = x - hi; the kernel accumulates
 // hi.hi + lo.hi + hi.lo in fp32, dropping only lo.lo (relative 2^-22).
 //
-// Roles (persistent CTA, one per SM; item = one (sequence, value head)):
-//   producer warps   TMA tensor-map loads of S0 / [Q;K] / V into a stage ring, node scalars
-//   MMA-1 warp       stage-1 MMAs into a TMEM buffer           -> mma1_done
-//   consumer groups  (2 x 128 threads, alternate items; thread c = TMEM lane c = row c of d_v)
-//       G: Gram rows -> scaled ancestor lists (A, P, indices), branch-free column scan
-//       T: per-node back-substitution -> rows of T and W, scattered (hi, lo) into the swizzled
-//          operand tiles that overlay the stage's dead [Q;K] tile
-//       R: R^T rows (hi, lo) into the tiles that overlay the dead S0 tile    -> ops_ready
-//   MMA-2 warp       stage-2 MMAs (3 passes each for U and O)   -> mma2_done, stage released
-//   consumer groups  epilogue: u_i = DU[i], o_i = g_i (S0 q_i) + DO[i]; coalesced stores
+// Roles (persistent CTA, one per SM; item = one (sequence, value head)).  Every phase of an item
+// has its own warps and every role walks all items in order, so the per-item cost is that of the
+// slowest role, not their sum; rings of buffers (4 load stages, 5 + 3 tensor-memory blocks, 2 slots
+// for lists / scalars / v rows) let consecutive items overlap:
+//   producer warps   TMA tensor-map loads of S0 and [Q;K] into a stage ring; node scalars and the
+//                    path lists (index and gate ratio of every node's first 8 ancestors)
+//   MMA-1 warp       stage-1 MMAs: SQ | SK into a block of the first TMEM ring, the Gram block
+//                    into a block of the second                            -> mma1_done
+//   Gram warps       Gram rows -> stash -> scaled ancestor lists (A, P), per-node scalars; zero the
+//                    stage-2 B tiles (they overlay the dead [Q;K] tile)    -> lists_ready
+//   solver warps     per-node back-substitution -> rows of T and W, scattered (hi, lo) into the
+//                    swizzled B tiles; they also keep the v rows coming    -> ops_ready
+//   R^T warps        (thread c = TMEM lane c = row c of d_v) row c of R^T as hi / lo back into
+//                    tensor memory over the Gram block, g.S0q in place, zeros over S0k
+//                                                                          -> ops_ready
+//   MMA-2 warp       stage-2 MMAs, A = R^T from tensor memory, B = [W;T] from shared memory, three
+//                    passes (hi.hi, lo.hi, hi.lo) accumulated on [g.S0q | 0]: [O | U]
+//                                                                          -> mma2_done, stage and
+//                                                                             R^T block released
+//   epilogue warps   o_i and u_i leave tensor memory: coalesced stores     -> block released
+//
+// The kernel's code has to stay small: with this many roles in flight it was instruction-cache
+// bound (a third of the instruction fetches missed) until the long loops were rolled and the slow
+// path of the waits went out of line.
 //
 // Every mbarrier wait is bounded; on give-up the role leaves its loop, TREEWY_SEQ_TIMEOUT is
 // raised, and the CTA still reaches the common exit where tensor memory is freed.
@@ -38,24 +52,23 @@
 
 namespace treewy {
 
-constexpr int VT_GROUP = 128;
 constexpr uint32_t VT_TMEM_COLS = 512;
 
 template <int NP, bool FUSED> struct VtCfg {
     static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
-    static constexpr int GROUPS = 2;
+    static constexpr int SLOTS = 2;  // list / scalar / v-row buffers alternate between consecutive items
     static constexpr int STAGES = FUSED ? 3 : 4;
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     static constexpr int TBUF = 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
     static constexpr int RBUF = 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
-    static constexpr int CONSUMERS = VT_GROUP * GROUPS;
-    static constexpr int TW = 64;  // threads of a group's solver warps (one per row of T and of W)
-    static constexpr int TW_WARP0 = CONSUMERS / 32;
-    static constexpr int COMMIT_WARP0 = TW_WARP0 + GROUPS * TW / 32;
+    // every phase of an item has its own warps, and every role walks all items in order
+    static constexpr int G_THREADS = 64, T_THREADS = 64, R_THREADS = 128, E_THREADS = 128;
+    static constexpr int G_WARP0 = 0, T_WARP0 = 2, R_WARP0 = 4, E_WARP0 = 8;  // R / E: warp % 4 = TMEM lane quarter
+    static constexpr int COMMIT_WARP0 = 12;
     static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
     static constexpr int MMA2_WARP = MMA1_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
-    static constexpr int THREADS = CONSUMERS + GROUPS * TW + CGROUP + 64 + 32 * STAGES;
+    static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 64 + 32 * STAGES;
     // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
     // (the v rows arrive later, into the dead S0 tile)
     static constexpr int QK_HALF = 2 * NP * 128;
@@ -90,12 +103,12 @@ template <int NP, bool FUSED> struct VtCfg {
     // group-private: path lists of the first 8 ancestors, per-node scalars (double-buffered), and
     // the v rows [NP][128] bf16 of the group's next item (loaded one item ahead)
     static constexpr int GP_AP = 0, GP_PP = 2 * NP * 16, GP_SCAL = 4 * NP * 16;
-    static constexpr int GP_VS = (GP_SCAL + 2 * NP * 16 + 127) / 128 * 128;
+    static constexpr int GP_VS = (GP_SCAL + NP * 16 + 127) / 128 * 128;
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
-    static constexpr int PARTS = VT_GROUP / NP;  // threads per node in the list-building phase
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
-    static constexpr int OFF_BAR = OFF_GP + GROUPS * GP_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * GROUPS) * 8 + 16 + 1024;
+    static constexpr int OFF_EINFO = OFF_GP + SLOTS * GP_BYTES;  // (n, first node) of the item in a TMEM block
+    static constexpr int OFF_BAR = OFF_EINFO + TBUF * 8;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * SLOTS) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the group
     // turns it, in its own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
@@ -135,12 +148,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *mma2_done = ops_ready + C::TBUF;
     uint64_t *tmem_free = mma2_done + C::TBUF;
     uint64_t *r_free = tmem_free + C::TBUF;
-    uint64_t *v_ready = r_free + C::RBUF;
-    uint64_t *v_free = v_ready + C::GROUPS;       // group -> its solver warps: v rows copied to registers
-    uint64_t *lists_ready = v_free + C::GROUPS;   // group -> its solver warps: path lists written
-    uint64_t *t_done = lists_ready + C::GROUPS;   // solver warps -> group: rows of T / W written, lists read
-    uint64_t *upd_done = t_done + C::GROUPS;      // fused mode: the state tile of a stage carries the commit
+    uint64_t *v_ready = r_free + C::RBUF;              // v rows of a slot have landed
+    uint64_t *v_free = v_ready + C::SLOTS;             // R^T warps -> fetching thread: v rows copied to registers
+    uint64_t *lists_ready = v_free + C::SLOTS;         // Gram warps -> solver / R^T warps: lists and scalars written
+    uint64_t *lists_free = lists_ready + C::SLOTS;     // solver + R^T warps -> Gram warps: the slot may be rewritten
+    uint64_t *upd_done = lists_free + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(upd_done + C::STAGES);
+    int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -151,16 +165,16 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         }
         for (int i = 0; i < C::TBUF; ++i) {
             ptx::mbar_init(&mma1_done[i], 1);
-            ptx::mbar_init(&ops_ready[i], VT_GROUP + C::TW);
+            ptx::mbar_init(&ops_ready[i], C::R_THREADS + C::T_THREADS);
             ptx::mbar_init(&mma2_done[i], 1);
-            ptx::mbar_init(&tmem_free[i], VT_GROUP);
+            ptx::mbar_init(&tmem_free[i], C::E_THREADS);
         }
         for (int i = 0; i < C::RBUF; ++i) ptx::mbar_init(&r_free[i], 1);
-        for (int g = 0; g < C::GROUPS; ++g) {
+        for (int g = 0; g < C::SLOTS; ++g) {
             ptx::mbar_init(&v_ready[g], 1);
-            ptx::mbar_init(&v_free[g], VT_GROUP);
-            ptx::mbar_init(&lists_ready[g], VT_GROUP);
-            ptx::mbar_init(&t_done[g], C::TW);
+            ptx::mbar_init(&v_free[g], C::R_THREADS);
+            ptx::mbar_init(&lists_ready[g], C::G_THREADS);
+            ptx::mbar_init(&lists_free[g], C::R_THREADS + C::T_THREADS);
         }
         for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128);
         ptx::fence_barrier_init();
@@ -196,10 +210,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             int item, b, h, lo, n, bad, flag;
             unsigned long long mk;
             float Lv, bv;
-            // path lists of the node this lane owns (first 8 ancestors), and whether any path is longer
-            float rat[8];
-            uint32_t iw[2];
-            int deep;
+            int deep;  // whether any path has more than 8 ancestors
             // fused mode: the previous round's accepted path of this sequence
             int plo, pbad, plen, cnt, pj;
             unsigned long long pmask;
@@ -209,9 +220,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             Pre p;
             p.item = blockIdx.x + kk * gridDim.x;
             p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
-            p.deep = 0, p.iw[0] = 0u, p.iw[1] = 0u;
-#pragma unroll
-            for (int d = 0; d < 8; ++d) p.rat[d] = 0.f;
+            p.deep = 0;
             p.plo = 0, p.pbad = 0, p.plen = -1, p.cnt = 0, p.pj = 0, p.pmask = 0ull, p.La = 0.f, p.wj = 0.f;
             if (p.item >= n_items) return p;
             p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
@@ -231,21 +240,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             p.mk = on ? a.anc_mask[p.lo + lane] : 0ull;
             p.Lv = on ? a.cum_log_gate[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
             p.bv = on ? a.beta[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
-            {
-                // Only the gate ratios depend on the head; building the lists here, a round ahead of
-                // their use, takes the ffs / exp chain off the consumers' critical path.
-                uint32_t m = (uint32_t)p.mk & ~(1u << lane);
-                p.deep = __any_sync(0xffffffffu, __popc(m) > 8);
-                p.iw[0] = 0u, p.iw[1] = 0u;
-#pragma unroll
-                for (int d = 0; d < 8; ++d) {
-                    const int j = m ? __ffs(m) - 1 : 0;
-                    const float Lj = __shfl_sync(0xffffffffu, p.Lv, j);
-                    p.rat[d] = m ? __expf(p.Lv - Lj) : 0.f;
-                    p.iw[d >> 2] |= (uint32_t)j << (8 * (d & 3));
-                    m &= m - 1;
-                }
-            }
+            p.deep = __any_sync(0xffffffffu, __popc((uint32_t)p.mk & ~(1u << lane)) > 8);
             if constexpr (FUSED) {
                 p.plo = pv.node_offsets[p.b];
                 const int pn = pv.node_offsets[p.b + 1] - p.plo;
@@ -275,6 +270,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             return p;
         };
         Pre cur = fetch(s);
+#pragma unroll 1
         for (int kk = s;; kk += C::STAGES) {
             if (cur.item >= n_items) break;
             const Pre p = cur;
@@ -286,24 +282,18 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             if (lane < NP) meta_mask(stage)[lane] = p.mk, meta_L(stage)[lane] = p.Lv, meta_beta(stage)[lane] = p.bv;
             if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep;
-            if (lane < NP) {
-                meta_rat(stage)[lane] = make_float4(p.rat[0], p.rat[1], p.rat[2], p.rat[3]);
-                meta_rat(stage)[NP + lane] = make_float4(p.rat[4], p.rat[5], p.rat[6], p.rat[7]);
-                meta_idx(stage)[lane] = p.iw[0], meta_idx(stage)[NP + lane] = p.iw[1];
-            }
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
                 if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = expf(p.La), pm->plen = p.plen, pm->lo = p.plo;
             }
-            __syncwarp();
+            // The copies are issued first and announced (expect_tx, with the warp's one arrival) last:
+            // the phase cannot complete before that arrival, and the path lists below are written
+            // while the data is on its way.
             const bool need_tile = !p.bad || p.plen >= 0;  // the state tile serves verify, commit or both
+            const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
             if (lane == 0) {
-                const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
-                if (tx == 0) {
-                    ptx::mbar_arrive(&full[s]);
-                } else {
-                    ptx::mbar_arrive_expect_tx(&full[s], tx);
+                if (tx != 0) {
                     const int hq = p.h / group;
                     if (need_tile) {
                         ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.item * D, &full[s]);
@@ -327,6 +317,27 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                                   D * 4, &full[s]);
                 }
             }
+            {
+                // Path lists of the node this lane owns: index and gate ratio e^{L_i - L_j} of its first
+                // 8 ancestors.  Only the ratios depend on the head; building them here takes the
+                // ffs / exp chain off the consumers' critical path.  (Rolled: code size.)
+                uint32_t m = (uint32_t)p.mk & ~(1u << lane);
+                float *ratp = reinterpret_cast<float *>(meta_rat(stage)) + lane * 4;
+                unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(stage)) + lane * 4;
+#pragma unroll 1
+                for (int d = 0; d < 8; ++d) {
+                    const int j = m ? __ffs(m) - 1 : 0;
+                    const float Lj = __shfl_sync(0xffffffffu, p.Lv, j);
+                    const float r = m ? __expf(p.Lv - Lj) : 0.f;
+                    if (lane < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = r, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
+                    m &= m - 1;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (tx == 0) ptx::mbar_arrive(&full[s]);
+                else ptx::mbar_arrive_expect_tx(&full[s], tx);
+            }
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
         }
     } else if (FUSED && warp >= C::COMMIT_WARP0 && warp < C::MMA1_WARP) {
@@ -339,6 +350,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const int t = tid - C::COMMIT_WARP0 * 32;
         const int cc = t & 15, r0 = t >> 4;  // 16-byte column chunk; first of every eighth row
         const int group = a.H_v / a.H_qk;
+#pragma unroll 1
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -427,6 +439,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // ------------------------------------------------------------------ stage-1 MMAs
         constexpr uint32_t idesc1 = ptx::umma_idesc_bf16_f32(128, 2 * NP);
         constexpr uint32_t idesc2 = ptx::umma_idesc_bf16_f32(128, NP);
+#pragma unroll 1
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -443,14 +456,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
                     const uint32_t d1 = tmem_base + buf * C::TM_COLS;
                     const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
-#pragma unroll
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks & 3) * 32;
                         const uint64_t da = ptx::umma_desc_k_sw128(s0 + (ks >> 2) * C::S0_HALF + ko);
                         const uint64_t db = ptx::umma_desc_k_sw128(qk + (ks >> 2) * C::QK_HALF + ko);
                         ptx::umma_bf16(d1, da, db, idesc1, ks > 0);
                     }
-#pragma unroll
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks & 3) * 32;
                         const uint32_t base = qk + (ks >> 2) * C::QK_HALF + ko;
@@ -467,6 +480,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     } else if (warp == C::MMA2_WARP) {
         // ------------------------------------------------------------------ stage-2 MMAs
         constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
+#pragma unroll 1
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -480,13 +494,15 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     const uint32_t base = ptx::smem_u32(stage);
                     const uint32_t tb = tmem_base + buf * C::TM_COLS;
                     const uint32_t tr = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
-                    const uint32_t ra[3] = {tr + C::TM_RHI, tr + C::TM_RLO, tr + C::TM_RHI};
-                    const uint32_t wt[3] = {base + C::OFF_W_HI, base + C::OFF_W_HI, base + C::OFF_W_LO};
-#pragma unroll
-                    for (int p = 0; p < 3; ++p)
-#pragma unroll
-                        for (int ks = 0; ks < NP / 8; ++ks)  // on top of g.S0q (O) and zeros (U)
-                            ptx::umma_tf32_ts(tb, ra[p] + ks * 8, ptx::umma_desc_k_sw128(wt[p] + ks * 32), idesc, 1u);
+                    // three passes (hi.hi, lo.hi, hi.lo), each NP / 8 steps of K = 8, on top of g.S0q (O)
+                    // and zeros (U); rolled: the issue loop is short and code size matters
+#pragma unroll 1
+                    for (int q = 0; q < 3 * (NP / 8); ++q) {
+                        const int p = q / (NP / 8), ks = q % (NP / 8);
+                        const uint32_t ra = tr + (p == 1 ? C::TM_RLO : C::TM_RHI) + ks * 8;
+                        const uint32_t wt = base + (p == 2 ? C::OFF_W_LO : C::OFF_W_HI) + ks * 32;
+                        ptx::umma_tf32_ts(tb, ra, ptx::umma_desc_k_sw128(wt), idesc, 1u);
+                    }
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
                     ptx::umma_commit(&r_free[kk % C::RBUF]);
@@ -498,57 +514,153 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             __syncwarp();
         }
-    } else if (warp >= C::TW_WARP0 && warp < C::COMMIT_WARP0) {
+    } else if (warp >= C::G_WARP0 && warp < C::T_WARP0) {
+        // ------------------------------------------------------------------ Gram warps
+        // Per item: the Gram rows leave tensor memory into a stash, the stage-2 B tiles are zeroed,
+        // and the scaled ancestor lists are built for the solver warps:
+        //   P[i][d] = e^{L_i-L_j} q_i.k_j ,  A[i][d] = beta_i e^{L_i-L_j} k_i.k_j ,  idx[i][d] = j
+        // for j the d-th ancestor of i; lists are stored [d / 4][node][d % 4].
+        const int tg = tid - C::G_WARP0 * 32;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const bool gram_reader = (warp - C::G_WARP0) * 32 < 2 * NP;  // warps whose lanes hold [Q;K] rows
+        const int i = tg & (NP - 1), kind = (tg / NP) & 1;  // kind 0: P list (q rows), 1: A list (k rows)
+#pragma unroll 1
+        for (int kk = 0;; ++kk) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            if (item >= n_items) break;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
+            unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
+            float4 *Ap4 = reinterpret_cast<float4 *>(gp + C::GP_AP);
+            float4 *Pp4 = reinterpret_cast<float4 *>(gp + C::GP_PP);
+            float4 *scal = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
+            if (!ptx::mbar_wait(&mma1_done[buf], (kk / C::TBUF) & 1)) {
+                if (tg == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
+            const int n = meta_nlo(stage)[0];
+            if (tg == 0) einfo[buf] = make_int2(n, meta_nlo(stage)[1]);
+            if (n > 0) {
+                const float *Lm = meta_L(stage);
+                float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
+                const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
+                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
+                for (int q = tg; q < 4 * NP * 128 / 16; q += C::G_THREADS)
+                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
+                // the rows of the Gram block (row owner = lane)
+                if (gram_reader) {
+                    const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;
+#pragma unroll
+                    for (int c0 = 0; c0 < NP; c0 += 16) {
+                        if (c0 < n) {
+                            uint32_t g[16];
+                            ptx::tmem_ld16(tr + c0, g);
+                            ptx::tmem_wait_ld();
+                            if (tg < 2 * NP) {
+                                float4 *dst = reinterpret_cast<float4 *>(raw + tg * C::RLD + c0);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
+                                                         __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
+                            }
+                        }
+                    }
+                    ptx::tc_fence_before_sync();
+                }
+                ptx::named_sync(1, C::G_THREADS);
+                // the slot's previous lists and scalars must have been read
+                ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
+                const bool valid = i < n;
+                const float Li = Lm[i];
+                const float bi = meta_beta(stage)[i];
+                const float scale = kind ? bi : 1.f;
+                const float *row = raw + (kind ? NP + i : i) * C::RLD;
+                if (!deep) {
+                    // the producer left indices and gate ratios of the first 8 ancestors: four Gram
+                    // entries are scaled at a time, no dependent chain
+                    for (int hf = tg / (2 * NP); hf < 2; hf += C::G_THREADS / (2 * NP)) {
+                        const uint32_t iw = meta_idx(stage)[hf * NP + i];
+                        const float4 rt = meta_rat(stage)[hf * NP + i];
+                        float4 val;
+                        val.x = scale * rt.x * row[iw & 255u], val.y = scale * rt.y * row[(iw >> 8) & 255u];
+                        val.z = scale * rt.z * row[(iw >> 16) & 255u], val.w = scale * rt.w * row[iw >> 24];
+                        (kind ? Ap4 : Pp4)[hf * NP + i] = val;
+                    }
+                } else if (tg < 2 * NP) {  // full-length lists, in the scratch over the dead S0 tile
+                    float *Ap = reinterpret_cast<float *>(stage + C::OFF_DAP);
+                    float *Pp = reinterpret_cast<float *>(stage + C::OFF_DPP);
+                    unsigned char *idx = stage + C::OFF_DIDX;
+                    uint32_t m = valid ? (uint32_t)meta_mask(stage)[i] & ~(1u << i) : 0u;
+                    for (int d = 0; m; ++d) {
+                        const int j = __ffs(m) - 1;
+                        m &= m - 1;
+                        const float val = scale * __expf(Li - Lm[j]) * row[j];
+                        const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
+                        if (kind) Ap[at] = val;
+                        else Pp[at] = val, idx[at] = (unsigned char)j;
+                    }
+                }
+                if (tg < NP && valid) {
+                    const float gi = __expf(Li);
+                    scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
+                }
+                ptx::fence_proxy_async();  // the zero fill is read by the tensor core
+            } else {
+                ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
+            }
+            ptx::mbar_arrive(&lists_ready[L]);  // lists, scalars and the zero fill are in place
+        }
+    } else if (warp >= C::T_WARP0 && warp < C::R_WARP0) {
         // ------------------------------------------------------------------ solver warps
         // Rows of T = (I + A)^-1 (one thread per node) and of W = P T (another) by back-substitution
         // along node i's root path j_0 .. j_{dp-1}, j_dp = i:
         //   x_dp = 1 (T) or P[i][i] (W);  x_e = p_e - sum_{f > e} x_f A[j_f][j_e]
-        // This needs shared memory only, so it runs beside the group's own work on R^T.
-        const int grp = (warp - C::TW_WARP0) / (C::TW / 32);
-        const int tt = tid - C::TW_WARP0 * 32 - grp * C::TW;
-        unsigned char *gp = smem + C::OFF_GP + grp * C::GP_BYTES;
-        const float4 *Ap4 = reinterpret_cast<const float4 *>(gp + C::GP_AP);
-        const float4 *Pp4 = reinterpret_cast<const float4 *>(gp + C::GP_PP);
-        const float4 *scal2 = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
+        // scattered (hi, lo) into the swizzled B tiles of stage 2.  Shared memory only.
+        const int tt = tid - C::T_WARP0 * 32;
         const int i = tt & (NP - 1);
         const bool wrow = (tt / NP) & 1;
-        // The v rows of the group's NEXT item are fetched (last thread of the solver warps) as soon
-        // as the group has copied the current ones to registers; the first packed node is looked
-        // up one item further ahead, so the fetch never waits on node_offsets.  Rows past a tree's
+        // The last solver thread also keeps the v rows coming: as soon as the R^T warps have copied
+        // the rows of item k to registers, the slot takes the rows of item k + 2.  Rows past a tree's
         // end belong to other sequences or are zero fill: they are loaded and never used.
-        int v_pending = -1;  // the item whose v rows are in flight or unread
+        const bool v_thread = tt == C::T_THREADS - 1;
+        int v_pending[2] = {-1, -1};  // per slot: the item whose v rows are in flight or unread
         auto first_node = [&](int kx) {
             const int it = blockIdx.x + kx * gridDim.x;
             return it < n_items ? a.node_offsets[it / a.H_v] : 0;
         };
         auto fetch_v = [&](int kx, int lo_x) {
             const int it = blockIdx.x + kx * gridDim.x;
-            v_pending = -1;
+            v_pending[kx & 1] = -1;
             if (it >= n_items) return;
-            v_pending = kx;
-            ptx::mbar_arrive_expect_tx(&v_ready[grp], C::V_BYTES);
-            ptx::tma_load_2d(gp + C::GP_VS, &tmV, (it % a.H_v) * D, lo_x, &v_ready[grp]);
+            v_pending[kx & 1] = kx;
+            ptx::mbar_arrive_expect_tx(&v_ready[kx & 1], C::V_BYTES);
+            ptx::tma_load_2d(smem + C::OFF_GP + (kx & 1) * C::GP_BYTES + C::GP_VS, &tmV, (it % a.H_v) * D, lo_x,
+                             &v_ready[kx & 1]);
         };
-        int v_lo_next = 0;
-        const bool v_thread = tt == C::TW - 1;
         if (v_thread) {
             ptx::prefetch_tmap(&tmV);
-            fetch_v(grp, first_node(grp));
-            v_lo_next = first_node(grp + C::GROUPS);
+            fetch_v(0, first_node(0));
+            fetch_v(1, first_node(1));
         }
         bool gave_up = false;
-        for (int kk = grp;; kk += C::GROUPS) {
+#pragma unroll 1
+        for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
-            const int s = kk % C::STAGES, buf = kk % C::TBUF;
-            const float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
-            if (!ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1)) {
+            unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
+            const float4 *Ap4 = reinterpret_cast<const float4 *>(gp + C::GP_AP);
+            const float4 *Pp4 = reinterpret_cast<const float4 *>(gp + C::GP_PP);
+            const float4 *scal = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
+            const int v_lo_next = v_thread ? first_node(kk + 2) : 0;  // needed only after this item's rows
+            if (!ptx::mbar_wait(&lists_ready[L], (kk >> 1) & 1)) {
                 gave_up = true;
                 break;
             }
-            ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
-            const int n = meta_nlo(stage)[0];
+            const int n = meta_nlo(stage)[0];  // (the Gram warps read the meta block before they signalled)
             if (n > 0 && tt < 2 * NP && i < n) {
                 const bool deep = meta_nlo(stage)[2] != 0;
                 const float *Ap = reinterpret_cast<const float *>(stage + C::OFF_DAP);
@@ -625,228 +737,124 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
             }
             ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
-            ptx::mbar_arrive(&t_done[grp]);
+            ptx::mbar_arrive(&lists_free[L]);
             ptx::mbar_arrive(&ops_ready[buf]);
             if (v_thread) {
-                if (!ptx::mbar_wait(&v_free[grp], (kk / C::GROUPS) & 1)) {
+                if (!ptx::mbar_wait(&v_free[L], (kk >> 1) & 1)) {
                     gave_up = true;
                     break;
                 }
-                fetch_v(kk + C::GROUPS, v_lo_next);
-                v_lo_next = first_node(kk + 2 * C::GROUPS);
+                fetch_v(kk + 2, v_lo_next);
             }
         }
         // after a give-up a fetch may still be in flight: it must land before the CTA exits
-        if (v_thread && gave_up && v_pending >= 0) ptx::mbar_wait(&v_ready[grp], (v_pending / C::GROUPS) & 1);
-    } else {
-        // ------------------------------------------------------------------ consumer groups
-        const int grp = warp >> 2, t = tid & (VT_GROUP - 1);
-        unsigned char *gp = smem + C::OFF_GP + grp * C::GP_BYTES;
-        float4 *Ap4 = reinterpret_cast<float4 *>(gp + C::GP_AP);
-        float4 *Pp4 = reinterpret_cast<float4 *>(gp + C::GP_PP);
-        float4 *scal2 = reinterpret_cast<float4 *>(gp + C::GP_SCAL);
-        const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
-        TOut *Og = static_cast<TOut *>(a.O);
+        if (v_thread && gave_up) {
+            for (int q = 0; q < 2; ++q)
+                if (v_pending[q] >= 0) ptx::mbar_wait(&v_ready[q], (v_pending[q] >> 1) & 1);
+        }
+    } else if (warp >= C::R_WARP0 && warp < C::E_WARP0) {
+        // ------------------------------------------------------------------ R^T warps
+        // Thread c = TMEM lane c = row c of d_v.  Row c of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j),
+        // goes back to tensor memory as hi / lo (the A operand of stage 2); g_j (S0 q_j) in place and
+        // zeros over S0 k_j are what stage 2 accumulates o_j and u_j on.
+        const int t = tid - C::R_WARP0 * 32;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
-
-        // Software pipeline: the front half of an item (lists, T / W rows, R^T -> ops_ready) is done
-        // before the back half (epilogue) of the group's previous item, so the stage-2 MMAs of
-        // one item run under the front half of the next.
-        int b_kk = -1, b_n = 0, b_lo = 0;  // the item whose back half is pending
-        bool dead = false;
-        for (int kk = grp; !dead; kk += C::GROUPS) {
+#pragma unroll 1
+        for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
-            const bool have = item < n_items;
-            int f_n = 0, f_lo = 0;
-            if (have) {
-            const int s = kk % C::STAGES, buf = kk % C::TBUF;
-            float4 *scal = scal2 + ((kk / C::GROUPS) & 1) * NP;
+            if (item >= n_items) break;
+            const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
-            if (!ptx::mbar_wait(&mma1_done[buf], (kk / C::TBUF) & 1)) {
-                if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
-                dead = true;
-                break;
-            }
+            unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
+            const float4 *scal = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
+            const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
+            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;                 // SQ | SK
+            const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;            // D2 | -
+            // The Gram warps signal after they have seen stage 1 complete, read the Gram block out and
+            // recorded the item's size: one wait covers all three.
+            if (!ptx::mbar_wait(&lists_ready[L], (kk >> 1) & 1)) break;
             ptx::tc_fence_after_sync();
-            ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
-            const int n = meta_nlo(stage)[0];
-            const int lo = meta_nlo(stage)[1];
-            const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;  // SQ | SK
-            const uint32_t tr = tmem_base + lane_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;  // D2 | -
-            const bool gram_reader = (warp & 3) * 32 < 2 * NP;  // warps whose lanes hold [Q;K] rows
+            const int n = einfo[buf].x;
+            ptx::mbar_wait(&v_ready[L], (kk >> 1) & 1);
             if (n > 0) {
-                const unsigned long long *mask = meta_mask(stage);
-                const float *Lm = meta_L(stage);
-                float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
-                float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
-                const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
-                float *Ap = deep ? reinterpret_cast<float *>(stage + C::OFF_DAP) : reinterpret_cast<float *>(Ap4);
-                float *Pp = deep ? reinterpret_cast<float *>(stage + C::OFF_DPP) : reinterpret_cast<float *>(Pp4);
-                unsigned char *idx = stage + C::OFF_DIDX;
-
-                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
-                for (int q = t; q < 4 * NP * 128 / 16; q += VT_GROUP)
-                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
-
-                // ---- phase G1: the rows of the Gram matrix leave tensor memory (row owner = lane)
-                if (gram_reader) {
-#pragma unroll
-                    for (int c0 = 0; c0 < NP; c0 += 16) {
-                        if (c0 < n) {
-                            uint32_t g[16];
-                            ptx::tmem_ld16(tr + c0, g);
-                            ptx::tmem_wait_ld();
-                            if (t < 2 * NP) {
-                                float4 *dst = reinterpret_cast<float4 *>(raw + t * C::RLD + c0);
-#pragma unroll
-                                for (int q = 0; q < 4; ++q)
-                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
-                                                         __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
-                            }
-                        }
-                    }
-                }
-                ptx::named_sync(1 + grp, VT_GROUP);
-
-                // ---- phase G2: scaled ancestor lists
-                //   P[i][d] = e^{L_i-L_j} q_i.k_j ,  A[i][d] = beta_i e^{L_i-L_j} k_i.k_j ,  idx[i][d] = j
-                //   for j the d-th ancestor of i; lists are stored [d / 4][node][d % 4]
-                constexpr int HALF = C::PARTS / 2;
-                const int i = t & (NP - 1), part = t / NP;
-                const bool valid = i < n;
-                const bool a_kind = part >= HALF;
-                const int sub = a_kind ? part - HALF : part;
-                const uint32_t mi = valid ? (uint32_t)mask[i] : 0u;
-                const int dp = valid ? __popc(mi) - 1 : 0;  // ancestors of node i
-                const float Li = Lm[i];
-                const float bi = meta_beta(stage)[i];
-                // the solver warps must have read the previous item's lists
-                if (kk >= C::GROUPS) ptx::mbar_wait(&t_done[grp], ((kk / C::GROUPS) - 1) & 1);
-                if (!deep) {
-                    // the producer left indices and gate ratios of the first 8 ancestors: one thread
-                    // scales four Gram entries, no dependent chain
-                    if (sub < 2) {
-                        const float scale = a_kind ? bi : 1.f;
-                        const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
-                        const uint32_t iw = meta_idx(stage)[sub * NP + i];
-                        const float4 rt = meta_rat(stage)[sub * NP + i];
-                        float4 val;
-                        val.x = scale * rt.x * row[iw & 255u], val.y = scale * rt.y * row[(iw >> 8) & 255u];
-                        val.z = scale * rt.z * row[(iw >> 16) & 255u], val.w = scale * rt.w * row[iw >> 24];
-                        (a_kind ? Ap4 : Pp4)[sub * NP + i] = val;
-                    }
-                } else {
-                    const float scale = a_kind ? bi : 1.f;
-                    const float *row = raw + (a_kind ? NP + i : i) * C::RLD;
-                    uint32_t m = mi & ~(1u << i);
-                    for (int q = 0; q < sub; ++q) m &= m - 1;
-                    for (int d = sub; d < dp; d += HALF) {
-                        const int j = __ffs(m) - 1;
-                        const float val = scale * __expf(Li - Lm[j]) * row[j];
-                        const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
-                        if (a_kind) Ap[at] = val;
-                        else Pp[at] = val, idx[at] = (unsigned char)j;
-#pragma unroll
-                        for (int q = 0; q < HALF; ++q) m &= m - 1;
-                    }
-                }
-                if (part == 0 && valid) {
-                    const float gi = __expf(Li);
-                    scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
-                }
-                ptx::mbar_arrive(&lists_ready[grp]);  // lists, scalars and the zero fill are in place
-
-                // this thread's column of the v rows; once every thread has its copy a solver warp
-                // fetches the rows of the group's next item into the buffer
-                ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);
-                __nv_bfloat16 vreg[NP];
-#pragma unroll
-                for (int j = 0; j < NP; ++j) vreg[j] = vs[j * D + t];
-                ptx::mbar_arrive(&v_free[grp]);
-                // the per-node scalars were written by other threads of the group
-                ptx::mbar_wait(&lists_ready[grp], (kk / C::GROUPS) & 1);
-
-                // ---- phase R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), as hi / lo, stays in
-                // tensor memory (the A operand of stage 2); g_j (S0 q_j) in place and zeros over S0 k_j
-                // are what stage 2 accumulates o_j and u_j on
-#pragma unroll
-                for (int c0 = 0; c0 < NP; c0 += 16) {
-                    uint32_t hi[16], lo[16];
+#pragma unroll 1
+                for (int c0 = 0; c0 < NP; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
+                    uint32_t hi[8], lo[8];
                     if (c0 < n) {
-                        uint32_t sk[16], sq[16];
-                        ptx::tmem_ld16(tm + NP + c0, sk);
-                        ptx::tmem_ld16(tm + c0, sq);
+                        uint32_t sk[8], sq[8];
+                        ptx::tmem_ld8(tm + NP + c0, sk);
+                        ptx::tmem_ld8(tm + c0, sq);
+                        float v[8];
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) v[jj] = __bfloat162float(vs[(c0 + jj) * D + t]);
                         ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) {
+                        for (int jj = 0; jj < 8; ++jj) {
                             const int j = c0 + jj;
                             const float4 sc = scal[j];
-                            const float v = __bfloat162float(vreg[j]);
-                            const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v);
+                            const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v[jj]);
                             const float rj = j < n ? val : 0.f;
                             const float h = ptx::tf32_hi(rj);
                             hi[jj] = __float_as_uint(h), lo[jj] = __float_as_uint(rj - h);
                             sq[jj] = __float_as_uint(sc.z * __uint_as_float(sq[jj]));
                             sk[jj] = 0u;
                         }
-                        ptx::tmem_st16(tm + c0, sq);
-                        ptx::tmem_st16(tm + NP + c0, sk);
+                        ptx::tmem_st8(tm + c0, sq);
+                        ptx::tmem_st8(tm + NP + c0, sk);
                     } else {
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) hi[jj] = 0u, lo[jj] = 0u;
+                        for (int jj = 0; jj < 8; ++jj) hi[jj] = 0u, lo[jj] = 0u;
                     }
-                    ptx::tmem_st16(tr + C::TM_RHI + c0, hi);
-                    ptx::tmem_st16(tr + C::TM_RLO + c0, lo);
+                    ptx::tmem_st8(tr + C::TM_RHI + c0, hi);
+                    ptx::tmem_st8(tr + C::TM_RLO + c0, lo);
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
-                ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
-            } else {
-                if (kk >= C::GROUPS) ptx::mbar_wait(&t_done[grp], ((kk / C::GROUPS) - 1) & 1);
-                ptx::mbar_arrive(&lists_ready[grp]);
-                ptx::mbar_wait(&v_ready[grp], (kk / C::GROUPS) & 1);  // rows of a skipped item: unused
-                ptx::mbar_arrive(&v_free[grp]);
             }
+            ptx::mbar_arrive(&v_free[L]);
+            ptx::mbar_arrive(&lists_free[L]);
             ptx::mbar_arrive(&ops_ready[buf]);
-            f_n = n, f_lo = lo;
-            }
-
-            if (b_kk >= 0) {
-            const int kk = b_kk, n = b_n, lo = b_lo;
-            const int item = blockIdx.x + kk * gridDim.x, h = item % a.H_v;
-            const int s = kk % C::STAGES, buf = kk % C::TBUF;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        // u_i and o_i leave tensor memory: coalesced predicated stores, thread c = element c of a row
+        const int t = tid - C::E_WARP0 * 32;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        TOut *Og = static_cast<TOut *>(a.O);
+        const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
+#pragma unroll 1
+        for (int kk = 0;; ++kk) {
+            const int item = blockIdx.x + kk * gridDim.x;
+            if (item >= n_items) break;
+            const int buf = kk % C::TBUF, h = item % a.H_v;
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;
             if (!ptx::mbar_wait(&mma2_done[buf], (kk / C::TBUF) & 1)) {
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                 break;
             }
             ptx::tc_fence_after_sync();
+            const int2 info = einfo[buf];
+            const int n = info.x, lo = info.y;
             if (n > 0) {
-                // ---- epilogue: u_i and o_i leave tensor memory
                 float *Ub = a.U + ((size_t)lo * a.H_v + h) * D + t;
                 TOut *Ob = Og + ((size_t)lo * a.H_v + h) * D + t;
+#pragma unroll 1
+                for (int c0 = 0; c0 < n; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
+                    uint32_t du[8], dout[8];
+                    ptx::tmem_ld8(tm + C::TM_DU + c0, du);
+                    ptx::tmem_ld8(tm + C::TM_DO + c0, dout);
+                    ptx::tmem_wait_ld();
+                    float *Uc = Ub + (size_t)c0 * rs;
+                    TOut *Oc = Ob + (size_t)c0 * rs;
 #pragma unroll
-                for (int c0 = 0; c0 < NP; c0 += 16) {
-                    if (c0 < n) {
-                        uint32_t du[16], dout[16];
-                        ptx::tmem_ld16(tm + C::TM_DU + c0, du);
-                        ptx::tmem_ld16(tm + C::TM_DO + c0, dout);
-                        ptx::tmem_wait_ld();
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) {
-                            const int node = c0 + jj;
-                            st_global_if(Ub + node * rs, __uint_as_float(du[jj]), node < n);
-                            st_global_if(Ob + node * rs, __uint_as_float(dout[jj]), node < n);
-                        }
+                    for (int jj = 0; jj < 8; ++jj) {
+                        st_global_if(Uc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
+                        st_global_if(Oc + jj * rs, __uint_as_float(dout[jj]), c0 + jj < n);
                     }
                 }
             }
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&tmem_free[buf]);
-            }
-            if (!have) break;
-            b_kk = kk, b_n = f_n, b_lo = f_lo;
         }
     }
 
