@@ -81,6 +81,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
     return mbar_wait_slow(bar, parity);
 }
 
+// One arrival for the whole warp: every lane's earlier writes are ordered before it by the warp
+// barrier.  (A per-thread arrive is one shared-memory atomic per lane; 128 or 192 of them on one
+// barrier take a couple of thousand cycles to drain.)
+__device__ __forceinline__ void mbar_arrive_warp(uint64_t *bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 // ----------------------------------------------------------------------------- bulk copies
 // generic-proxy writes to shared memory -> visible to the async proxy (before a bulk store)
 __device__ __forceinline__ void fence_proxy_async()

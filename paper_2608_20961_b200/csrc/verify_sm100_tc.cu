@@ -66,9 +66,10 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int G_WARP0 = 0, T_WARP0 = 2, R_WARP0 = 4, E_WARP0 = 8;  // R / E: warp % 4 = TMEM lane quarter
     static constexpr int COMMIT_WARP0 = 12;
     static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
-    static constexpr int MMA2_WARP = MMA1_WARP + 1;
+    static constexpr int MMA1B_WARP = MMA1_WARP + 1;  // the Gram chain of stage 1 has its own issuing warp
+    static constexpr int MMA2_WARP = MMA1B_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
-    static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 64 + 32 * STAGES;
+    static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 96 + 32 * STAGES;
     // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
     // (the v rows arrive later, into the dead S0 tile)
     static constexpr int QK_HALF = 2 * NP * 128;
@@ -157,6 +158,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Item kk of this CTA (>= n_items when there is none).  When an even number of value heads
+    // share a q/k head, a CTA takes the heads two by two: both items of a pair have the same tree
+    // and the same [Q;K] rows, so the second reuses the first one's Gram entries.
+    const bool pair_mode = ((a.H_v / a.H_qk) & 1) == 0;
+    auto item_of = [&](int kk) {
+        return pair_mode ? 2 * ((int)blockIdx.x + (kk >> 1) * (int)gridDim.x) + (kk & 1) : (int)blockIdx.x + kk * (int)gridDim.x;
+    };
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -164,19 +172,19 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&empty[s], 1);
         }
         for (int i = 0; i < C::TBUF; ++i) {
-            ptx::mbar_init(&mma1_done[i], 1);
-            ptx::mbar_init(&ops_ready[i], C::R_THREADS + C::T_THREADS);
+            ptx::mbar_init(&mma1_done[i], 2);
+            ptx::mbar_init(&ops_ready[i], (C::R_THREADS + C::T_THREADS) / 32);  // one arrival per warp
             ptx::mbar_init(&mma2_done[i], 1);
-            ptx::mbar_init(&tmem_free[i], C::E_THREADS);
+            ptx::mbar_init(&tmem_free[i], C::E_THREADS / 32);
         }
         for (int i = 0; i < C::RBUF; ++i) ptx::mbar_init(&r_free[i], 1);
         for (int g = 0; g < C::SLOTS; ++g) {
             ptx::mbar_init(&v_ready[g], 1);
-            ptx::mbar_init(&v_free[g], C::R_THREADS);
-            ptx::mbar_init(&lists_ready[g], C::G_THREADS);
-            ptx::mbar_init(&lists_free[g], C::R_THREADS + C::T_THREADS);
+            ptx::mbar_init(&v_free[g], C::R_THREADS / 32);
+            ptx::mbar_init(&lists_ready[g], C::G_THREADS / 32);
+            ptx::mbar_init(&lists_free[g], (C::R_THREADS + C::T_THREADS) / 32);
         }
-        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128);
+        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32);
         ptx::fence_barrier_init();
     }
     if (warp == C::MMA1_WARP) {
@@ -218,7 +226,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         };
         auto fetch = [&](int kk) {
             Pre p;
-            p.item = blockIdx.x + kk * gridDim.x;
+            p.item = item_of(kk);
             p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
             p.deep = 0;
             p.plo = 0, p.pbad = 0, p.plen = -1, p.cnt = 0, p.pj = 0, p.pmask = 0ull, p.La = 0.f, p.wj = 0.f;
@@ -352,7 +360,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const int group = a.H_v / a.H_qk;
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -432,24 +440,31 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 ptx::bulk_commit_group();
                 ptx::bulk_wait_group_read<0>();  // the tile will be overwritten by scratch after the MMAs
             }
-            ptx::mbar_arrive(&upd_done[s]);
+            ptx::mbar_arrive_warp(&upd_done[s]);
         }
         if (t == 0) ptx::bulk_wait_group<0>();
-    } else if (warp == C::MMA1_WARP) {
+    } else if (warp == C::MMA1_WARP || warp == C::MMA1B_WARP) {
         // ------------------------------------------------------------------ stage-1 MMAs
+        // One tcgen05.mma of these sizes keeps its issuing thread for ~120 cycles, so the two
+        // accumulation chains (S0 [Q;K]^T and the Gram block) are issued by two warps.
+        const bool gram_chain = warp == C::MMA1B_WARP;
         constexpr uint32_t idesc1 = ptx::umma_idesc_bf16_f32(128, 2 * NP);
         constexpr uint32_t idesc2 = ptx::umma_idesc_bf16_f32(128, NP);
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
             if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) break;
-            const int n = meta_nlo(stage)[0];
+            const bool reuse_gram = pair_mode && (kk & 1) && meta_nlo(stage)[2] == 0;
+            const int n = gram_chain && reuse_gram ? 0 : meta_nlo(stage)[0];
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
-            if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
-            if (!ptx::mbar_wait(&r_free[kk % C::RBUF], ((kk / C::RBUF) & 1) ^ 1)) break;
+            if (gram_chain) {
+                if (!ptx::mbar_wait(&r_free[kk % C::RBUF], ((kk / C::RBUF) & 1) ^ 1)) break;
+            } else {
+                if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
+            }
             ptx::tc_fence_after_sync();
             if (lane == 0) {
                 if (n > 0) {
@@ -458,17 +473,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
 #pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t ko = (ks & 3) * 32;
-                        const uint64_t da = ptx::umma_desc_k_sw128(s0 + (ks >> 2) * C::S0_HALF + ko);
-                        const uint64_t db = ptx::umma_desc_k_sw128(qk + (ks >> 2) * C::QK_HALF + ko);
-                        ptx::umma_bf16(d1, da, db, idesc1, ks > 0);
-                    }
-#pragma unroll 1
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t ko = (ks & 3) * 32;
-                        const uint32_t base = qk + (ks >> 2) * C::QK_HALF + ko;
-                        ptx::umma_bf16(d2, ptx::umma_desc_k_sw128(base), ptx::umma_desc_k_sw128(base + NP * 128),
-                                       idesc2, ks > 0);
+                        const uint32_t ko = (ks >> 2) * C::QK_HALF + (ks & 3) * 32;
+                        const uint64_t dq = ptx::umma_desc_k_sw128(qk + ko);
+                        if (gram_chain) {
+                            ptx::umma_bf16(d2, dq, ptx::umma_desc_k_sw128(qk + ko + NP * 128), idesc2, ks > 0);
+                        } else {
+                            const uint64_t da = ptx::umma_desc_k_sw128(s0 + (ks >> 2) * C::S0_HALF + (ks & 3) * 32);
+                            ptx::umma_bf16(d1, da, dq, idesc1, ks > 0);
+                        }
                     }
                     ptx::umma_commit(&mma1_done[buf]);
                 } else {
@@ -482,7 +494,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -524,9 +536,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const bool gram_reader = (warp - C::G_WARP0) * 32 < 2 * NP;  // warps whose lanes hold [Q;K] rows
         const int i = tg & (NP - 1), kind = (tg / NP) & 1;  // kind 0: P list (q rows), 1: A list (k rows)
+        float4 gram4[2];         // this thread's Gram entries (its node's first 8 ancestors), kept for the
+        float gram_diag = 0.f;   // second item of a pair; q_i.k_i
+        gram4[0] = gram4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -546,11 +561,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const float *Lm = meta_L(stage);
                 float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
                 const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
+                // second item of a pair: same tree, same [Q;K] rows; the Gram entries are in registers
+                const bool reuse_gram = pair_mode && (kk & 1) && !deep;
                 // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
                 for (int q = tg; q < 4 * NP * 128 / 16; q += C::G_THREADS)
                     reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
                 // the rows of the Gram block (row owner = lane)
-                if (gram_reader) {
+                if (gram_reader && !reuse_gram) {
                     const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;
 #pragma unroll
                     for (int c0 = 0; c0 < NP; c0 += 16) {
@@ -569,7 +586,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
                     ptx::tc_fence_before_sync();
                 }
-                ptx::named_sync(1, C::G_THREADS);
+                if (!reuse_gram) ptx::named_sync(1, C::G_THREADS);
                 // the slot's previous lists and scalars must have been read
                 ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
                 const bool valid = i < n;
@@ -580,12 +597,18 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (!deep) {
                     // the producer left indices and gate ratios of the first 8 ancestors: four Gram
                     // entries are scaled at a time, no dependent chain
-                    for (int hf = tg / (2 * NP); hf < 2; hf += C::G_THREADS / (2 * NP)) {
-                        const uint32_t iw = meta_idx(stage)[hf * NP + i];
+                    constexpr int HSTEP = C::G_THREADS / (2 * NP), HN = 2 / HSTEP;
+#pragma unroll
+                    for (int q = 0; q < HN; ++q) {
+                        const int hf = tg / (2 * NP) + q * HSTEP;
                         const float4 rt = meta_rat(stage)[hf * NP + i];
+                        if (!reuse_gram) {
+                            const uint32_t iw = meta_idx(stage)[hf * NP + i];
+                            gram4[q] = make_float4(row[iw & 255u], row[(iw >> 8) & 255u], row[(iw >> 16) & 255u], row[iw >> 24]);
+                        }
                         float4 val;
-                        val.x = scale * rt.x * row[iw & 255u], val.y = scale * rt.y * row[(iw >> 8) & 255u];
-                        val.z = scale * rt.z * row[(iw >> 16) & 255u], val.w = scale * rt.w * row[iw >> 24];
+                        val.x = scale * rt.x * gram4[q].x, val.y = scale * rt.y * gram4[q].y;
+                        val.z = scale * rt.z * gram4[q].z, val.w = scale * rt.w * gram4[q].w;
                         (kind ? Ap4 : Pp4)[hf * NP + i] = val;
                     }
                 } else if (tg < 2 * NP) {  // full-length lists, in the scratch over the dead S0 tile
@@ -604,13 +627,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
                 if (tg < NP && valid) {
                     const float gi = __expf(Li);
-                    scal[i] = make_float4(bi, bi * gi, gi, raw[i * C::RLD + i]);
+                    if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
+                    scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
                 }
                 ptx::fence_proxy_async();  // the zero fill is read by the tensor core
             } else {
                 ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
             }
-            ptx::mbar_arrive(&lists_ready[L]);  // lists, scalars and the zero fill are in place
+            ptx::mbar_arrive_warp(&lists_ready[L]);  // lists, scalars and the zero fill are in place
         }
     } else if (warp >= C::T_WARP0 && warp < C::R_WARP0) {
         // ------------------------------------------------------------------ solver warps
@@ -627,11 +651,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const bool v_thread = tt == C::T_THREADS - 1;
         int v_pending[2] = {-1, -1};  // per slot: the item whose v rows are in flight or unread
         auto first_node = [&](int kx) {
-            const int it = blockIdx.x + kx * gridDim.x;
+            const int it = item_of(kx);
             return it < n_items ? a.node_offsets[it / a.H_v] : 0;
         };
         auto fetch_v = [&](int kx, int lo_x) {
-            const int it = blockIdx.x + kx * gridDim.x;
+            const int it = item_of(kx);
             v_pending[kx & 1] = -1;
             if (it >= n_items) return;
             v_pending[kx & 1] = kx;
@@ -647,7 +671,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         bool gave_up = false;
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -737,14 +761,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
             }
             ptx::fence_proxy_async();  // operand tiles were written by ordinary stores
-            ptx::mbar_arrive(&lists_free[L]);
-            ptx::mbar_arrive(&ops_ready[buf]);
-            if (v_thread) {
-                if (!ptx::mbar_wait(&v_free[L], (kk >> 1) & 1)) {
-                    gave_up = true;
-                    break;
-                }
-                fetch_v(kk + 2, v_lo_next);
+            ptx::mbar_arrive_warp(&lists_free[L]);
+            ptx::mbar_arrive_warp(&ops_ready[buf]);
+            if (v_thread && !gave_up) {  // (no break: the warp's other lanes go on and meet this one at the next arrival)
+                if (ptx::mbar_wait(&v_free[L], (kk >> 1) & 1)) fetch_v(kk + 2, v_lo_next);
+                else gave_up = true;
             }
         }
         // after a give-up a fetch may still be in flight: it must land before the CTA exits
@@ -761,7 +782,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -811,9 +832,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
             }
-            ptx::mbar_arrive(&v_free[L]);
-            ptx::mbar_arrive(&lists_free[L]);
-            ptx::mbar_arrive(&ops_ready[buf]);
+            ptx::mbar_arrive_warp(&v_free[L]);
+            ptx::mbar_arrive_warp(&lists_free[L]);
+            ptx::mbar_arrive_warp(&ops_ready[buf]);
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -824,7 +845,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const int rs = a.H_v * D;  // elements between a sequence's consecutive node rows
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
-            const int item = blockIdx.x + kk * gridDim.x;
+            const int item = item_of(kk);
             if (item >= n_items) break;
             const int buf = kk % C::TBUF, h = item % a.H_v;
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;
@@ -854,7 +875,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
             }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&tmem_free[buf]);
+            ptx::mbar_arrive_warp(&tmem_free[buf]);
         }
     }
 
@@ -884,7 +905,8 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     e = cudaFuncSetAttribute(verify_sm100_tc_kernel<NP, TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    const int grid = (int)(n_items < sms ? n_items : sms);
+    const long long units = (a.H_v / a.H_qk) % 2 == 0 ? n_items / 2 : n_items;  // the kernel takes heads in pairs
+    const int grid = (int)(units < sms ? units : sms);
     verify_sm100_tc_kernel<NP, TOut, FUSED><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, pv, (int)n_items, m.S0,
                                                                                          m.Q, m.K, m.V);
     return cudaGetLastError();
