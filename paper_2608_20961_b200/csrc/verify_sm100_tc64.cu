@@ -42,9 +42,14 @@ constexpr int V6_STAGE_BYTES = (V6_OFF_META + V6_META_BYTES + 1023) / 1024 * 102
 constexpr uint32_t V6_TX_BYTES = V6_QK_BYTES + V6_S0_BYTES + V6_V_BYTES;
 // overlays on the dead tiles: raw Gram rows first, then the four operand tiles
 constexpr int V6_RLD = V6_NP + 4;
-constexpr int V6_TILE = V6_NP * 256;  // one fp32 operand tile [64 rows][64 cols] = two 8 KiB atoms
-constexpr int V6_ATOM = V6_NP * 128;
-constexpr int V6_OFF_T_HI = 0, V6_OFF_T_LO = V6_TILE, V6_OFF_W_HI = 2 * V6_TILE, V6_OFF_W_LO = 3 * V6_TILE;
+// The stage-2 B operand is [W;T]: 128 rows (W rows above T rows) of 64 fp32 columns, as two
+// 128-byte-swizzled atoms of 128 rows each, once for the hi parts and once for the lo parts; one
+// MMA then yields O and U together.
+constexpr int V6_TILE = V6_NP * 256;       // bytes of one 64-row operand [64 rows][64 cols]
+constexpr int V6_ATOM = 2 * V6_NP * 128;   // one atom of the stacked operand: 128 rows x 128 bytes
+constexpr int V6_OFF_X_HI = 0, V6_OFF_X_LO = 2 * V6_ATOM;
+constexpr int V6_OFF_W_HI = V6_OFF_X_HI, V6_OFF_T_HI = V6_OFF_X_HI + V6_NP * 128;
+constexpr int V6_OFF_W_LO = V6_OFF_X_LO, V6_OFF_T_LO = V6_OFF_X_LO + V6_NP * 128;
 static_assert(4 * V6_TILE <= V6_QK_BYTES + V6_S0_BYTES, "operand tiles fit the dead tiles");
 static_assert(2 * V6_NP * V6_RLD * 4 <= V6_QK_BYTES + V6_S0_BYTES, "raw Gram rows fit the dead tiles");
 // group-private: path lists [d / 4][node][d % 4], per-node scalars, ancestor indices
@@ -94,9 +99,9 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
         }
         for (int i = 0; i < V6_TBUF; ++i) {
             ptx::mbar_init(&mma1_done[i], 1);
-            ptx::mbar_init(&ops_ready[i], V6_GROUP);
+            ptx::mbar_init(&ops_ready[i], V6_GROUP / 32);  // one arrival per warp
             ptx::mbar_init(&mma2_done[i], 1);
-            ptx::mbar_init(&tmem_free[i], V6_GROUP);
+            ptx::mbar_init(&tmem_free[i], V6_GROUP / 32);
         }
         ptx::fence_barrier_init();
     }
@@ -239,7 +244,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
         //   O^T[c, i] += sum_j R^T[c,j] W[i,j]   on top of g_i (S0 q_i)[c]
         // A = R^T from tensor memory (hi | lo), B = T / W tiles from shared memory; three passes
         // hi.hi + lo.hi + hi.lo each.
-        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, NP);
+        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
         for (int kk = 0;; ++kk) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -252,22 +257,14 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
                     const uint32_t tb = tmem_base + buf * V6_TM_COLS;
-                    const uint32_t ra[3] = {tb + V6_TM_D2, tb + V6_TM_RLO, tb + V6_TM_D2};
-                    const uint32_t tt[3] = {base + V6_OFF_T_HI, base + V6_OFF_T_HI, base + V6_OFF_T_LO};
-                    const uint32_t ww[3] = {base + V6_OFF_W_HI, base + V6_OFF_W_HI, base + V6_OFF_W_LO};
-#pragma unroll
-                    for (int p = 0; p < 3; ++p)
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            ptx::umma_tf32_ts(tb + V6_TM_SK, ra[p] + ks * 8,
-                                              ptx::umma_desc_k_sw128(tt[p] + (ks >> 2) * V6_ATOM + (ks & 3) * 32), idesc,
-                                              (p | ks) != 0);
-#pragma unroll
-                    for (int p = 0; p < 3; ++p)
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            ptx::umma_tf32_ts(tb + V6_TM_SQ, ra[p] + ks * 8,
-                                              ptx::umma_desc_k_sw128(ww[p] + (ks >> 2) * V6_ATOM + (ks & 3) * 32), idesc, 1u);
+                    // three passes (hi.hi, lo.hi, hi.lo) of 8 steps of K = 8, accumulated on [g.S0q | 0]
+#pragma unroll 1
+                    for (int q = 0; q < 24; ++q) {
+                        const int p = q >> 3, ks = q & 7;
+                        const uint32_t ra = tb + (p == 1 ? V6_TM_RLO : V6_TM_D2) + ks * 8;
+                        const uint32_t xb = base + (p == 2 ? V6_OFF_X_LO : V6_OFF_X_HI) + (ks >> 2) * V6_ATOM + (ks & 3) * 32;
+                        ptx::umma_tf32_ts(tb + V6_TM_SQ, ra, ptx::umma_desc_k_sw128(xb), idesc, 1u);
+                    }
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
                 } else {
@@ -453,7 +450,9 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                                 const float val = j < n ? fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v) : 0.f;
                                 const float h = ptx::tf32_hi(val);
                                 hi[jj] = __float_as_uint(h), lo[jj] = __float_as_uint(val - h);
+                                sk[jj] = 0u;
                             }
+                            ptx::tmem_st16(tm + V6_TM_SK + c0, sk);  // u_j accumulates on zeros
                         } else {
 #pragma unroll
                             for (int jj = 0; jj < 16; ++jj) hi[jj] = 0u, lo[jj] = 0u;
@@ -477,7 +476,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                     ptx::fence_proxy_async();  // T / W tiles were written by ordinary stores
                 }
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&ops_ready[buf]);
+                ptx::mbar_arrive_warp(&ops_ready[buf]);
                 f_n = n, f_lo = lo;
             }
 
@@ -512,7 +511,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                     }
                 }
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&tmem_free[buf]);
+                ptx::mbar_arrive_warp(&tmem_free[buf]);
             }
             if (!have) break;
             b_kk = kk, b_n = f_n, b_lo = f_lo;
