@@ -334,8 +334,8 @@ def run_ours(args, rank: int, size: int, local: int):
         torch.cuda.synchronize(dev)
         fms = replicas.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
         fbytes = pb.total - w.B * w.H_v * 128 * 128 * w.S0.element_size()   # the state is read once
-        fused = {"what": "prepare + treewy_commit_verify(single_kernel=1) per step: state read once, written "
-                         "once; its in-kernel commit is instruction-bound, so it is slower than the two kernels",
+        fused = {"what": "prepare + treewy_commit_verify(single_kernel=1) per step: the previous round's commit "
+                         "and this round's verify in one kernel, state read once and written once",
                  "ms_per_step": fms, "value": size * units / (fms * 1e-3), "unit": UNIT,
                  "algorithmic_bytes": fbytes, "roof_ms": fbytes / (hbm * 1e9) * 1e3,
                  "frac": fbytes / (hbm * 1e9) * 1e3 / fms, "gpu_launches": 2 * args.steps}

@@ -150,13 +150,15 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
  * appendix names the state write as the lever): in serving, a layer's commit of round r is always
  * followed by its verify of round r+1 on the same state, so one kernel reads the old state once,
  * applies Eq. 3 in shared memory, writes the new state once and verifies the new draft tree from it.
- * The result is bit-identical to
+ * The result is that of
  *     treewy_commit(S0, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, NULL, ...);
  *     treewy_verify(S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, ...);
- * single_kernel = 0 issues exactly those two kernels (the faster choice on B200 today: both run
- * near the HBM roof on their own).  single_kernel = 1 takes the fused kernel when it applies (BF16
- * states, trees of up to 32 nodes in the new round; otherwise the two kernels again): it moves
- * 23 % fewer bytes, but its in-kernel commit is instruction-bound and it is currently the slower one.
+ * single_kernel = 0 issues exactly those two kernels.  single_kernel = 1 takes the fused kernel
+ * when it applies (BF16 states, trees of up to 32 nodes in the new round; otherwise the two kernels
+ * again): it moves 23 % fewer bytes.  Its rank-P update runs on the tensor cores with every fp32
+ * factor split into two tf32 parts (2^-22 relative), so a few elements of the stored bf16 state may
+ * differ from the two-kernel result by one rounding step; status words and the set of rows written
+ * are identical.
  * tree_prev / tree must describe the same B sequences and H_v heads; U_prev [T_prev,H_v,128] fp32
  * and k_prev [T_prev,H_qk,128] are the previous round's verify output and keys, accepted_prev [B]
  * its accepted nodes (-1 = nothing to commit for that sequence).  U_prev and U must not overlap.

@@ -214,6 +214,14 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t addr)
     return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+// Shared-memory matrix descriptor, K-major operand WITHOUT swizzle: the tile is made of core
+// matrices of 8 rows x 16 bytes stored contiguously (128 bytes); `lbo` is the byte distance between
+// core matrices that are neighbours along K, `sbo` between neighbours along M / N.
+__device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+           ((uint64_t)1 << 46);
+}
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, dense.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N)
 {

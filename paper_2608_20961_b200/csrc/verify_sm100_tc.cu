@@ -59,8 +59,9 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int SLOTS = 2;  // list / scalar / v-row buffers alternate between consecutive items
     static constexpr int STAGES = FUSED ? 3 : 4;
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
-    static constexpr int TBUF = 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
-    static constexpr int RBUF = 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
+    // (fused mode gives 128 columns of tensor memory to the commit's accumulator)
+    static constexpr int TBUF = FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
+    static constexpr int RBUF = FUSED ? 2 : 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
     // every phase of an item has its own warps, and every role walks all items in order
     static constexpr int G_THREADS = 64, T_THREADS = 64, R_THREADS = 128, E_THREADS = 128;
     static constexpr int G_WARP0 = 0, T_WARP0 = 2, R_WARP0 = 4, E_WARP0 = 8;  // R / E: warp % 4 = TMEM lane quarter
@@ -77,7 +78,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int S0_HALF = D * 128;
     static constexpr int S0_BYTES = 2 * S0_HALF;
     static constexpr int OFF_S0 = QK_BYTES;
-    static constexpr int PCH = 16;  // previous-round path nodes staged per item (fused mode)
+    static constexpr int PCH = 8;  // previous-round path nodes staged per item (fused mode)
     static constexpr int OFF_KP = OFF_S0 + S0_BYTES, OFF_UP = OFF_KP + PCH * D * 2;
     static constexpr int OFF_META = FUSED ? OFF_UP + PCH * D * 4 : OFF_S0 + S0_BYTES;
     // mask u64, L f32, beta f32 per node; n, lo, deep; then the producer-built path lists of the
@@ -108,8 +109,13 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_EINFO = OFF_GP + SLOTS * GP_BYTES;  // (n, first node) of the item in a TMEM block
-    static constexpr int OFF_BAR = OFF_EINFO + TBUF * 8;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * SLOTS) * 8 + 16 + 1024;
+    // fused mode: operands of the commit's rank-P product, K-major without swizzle, K = 8 path nodes:
+    // core matrices of 8 rows x 16 bytes, the two K halves COPS_LBO apart
+    static constexpr int COPS_LBO = D * 16, COPS_TILE = 2 * COPS_LBO;
+    static constexpr int OFF_CA_HI = (OFF_EINFO + TBUF * 8 + 127) / 128 * 128;
+    static constexpr int OFF_CA_LO = OFF_CA_HI + COPS_TILE, OFF_CB = OFF_CA_LO + COPS_TILE;
+    static constexpr int OFF_BAR = FUSED ? OFF_CB + COPS_TILE : OFF_EINFO + TBUF * 8;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * SLOTS + 1) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the group
     // turns it, in its own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
@@ -120,12 +126,13 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int TM_DO = 0, TM_DU = NP;
     static constexpr int TM_R0 = TBUF * TM_COLS;  // second ring
     static constexpr int TM_RHI = 0, TM_RLO = NP;
-    static_assert(TM_R0 + RBUF * 2 * NP <= 512, "tensor memory");
+    static constexpr int TM_C0 = TM_R0 + RBUF * 2 * NP;  // fused mode: the commit's 128 x 128 accumulator
+    static_assert(TM_C0 + (FUSED ? D : 0) <= 512, "tensor memory");
 };
 
 // fused mode: what the commit of the previous round needs for one (sequence, head)
 struct PathMeta {
-    float w[16];              // e^{L_a - L_j} of the staged path nodes
+    float w[8];               // e^{L_a - L_j} of the staged path nodes
     unsigned long long mask;  // ancestor-or-self mask of the accepted node (previous tree)
     float La, ga;             // its log-gate and e^{La}
     int plen;                 // path length; -1 = no commit for this item
@@ -154,7 +161,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *lists_ready = v_free + C::SLOTS;         // Gram warps -> solver / R^T warps: lists and scalars written
     uint64_t *lists_free = lists_ready + C::SLOTS;     // solver + R^T warps -> Gram warps: the slot may be rewritten
     uint64_t *upd_done = lists_free + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(upd_done + C::STAGES);
+    uint64_t *cmma_done = upd_done + C::STAGES;        // fused mode: the commit's rank-P product has finished
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(cmma_done + 1);
     int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -185,6 +193,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&lists_free[g], (C::R_THREADS + C::T_THREADS) / 32);
         }
         for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32);
+        ptx::mbar_init(cmma_done, 1);
         ptx::fence_barrier_init();
     }
     if (warp == C::MMA1_WARP) {
@@ -271,7 +280,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     p.cnt = min(p.plen, C::PCH);
                     if (lane < p.cnt) {
                         p.pj = nth_set_bit(p.pmask, lane);
-                        p.wj = expf(p.La - pv.cum_log_gate[(size_t)(p.plo + p.pj) * a.H_v + p.h]);
+                        p.wj = __expf(p.La - pv.cum_log_gate[(size_t)(p.plo + p.pj) * a.H_v + p.h]);
                     }
                 }
             }
@@ -293,7 +302,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
-                if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = expf(p.La), pm->plen = p.plen, pm->lo = p.plo;
+                if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = __expf(p.La), pm->plen = p.plen, pm->lo = p.plo;
             }
             // The copies are issued first and announced (expect_tx, with the warp's one arrival) last:
             // the phase cannot complete before that arrival, and the path lists below are written
@@ -351,13 +360,23 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     } else if (FUSED && warp >= C::COMMIT_WARP0 && warp < C::MMA1_WARP) {
         // ------------------------------------------------------------------ commit group (fused mode)
         // Before the stage-1 MMAs read a state tile, the previous round's accepted node is
-        // committed INTO it (Eq. 3):  S <- g_a S + sum_{j on the path} (g_a / g_j) u_j k_j^T , same
-        // fp32 arithmetic and summation order as the stand-alone commit kernel, rounded once to bf16
-        // in place (the tile keeps the 128-byte swizzle the TMA gave it), and the new state goes back
-        // to global memory with a TMA store while verification proceeds from the shared-memory copy.
+        // committed INTO it (Eq. 3):  S <- g_a S + sum_{j on the path} (g_a / g_j) u_j k_j^T .
+        // The rank-P term is a tensor-core product, 8 path nodes per round:
+        //   C[v][c] (+)= sum_p A[v][p] B[c][p],  A[v][p] = (g_a / g_p) u_p[v] (fp32 as tf32 hi + lo),
+        //   B[c][p] = k_p[c] (bf16, exact in tf32),
+        // both operands written by this group, K-major without swizzle; thread t owns row t of A, row
+        // t of B and, afterwards, TMEM lane t = row t of the state.  Then S[t][:] = g_a S[t][:] + C[t][:]
+        // is rounded once to bf16 in place (the tile keeps the 128-byte swizzle the TMA gave it), and
+        // the new state goes back to global memory with a TMA store while verification proceeds from
+        // the shared-memory copy.
         const int t = tid - C::COMMIT_WARP0 * 32;
-        const int cc = t & 15, r0 = t >> 4;  // 16-byte column chunk; first of every eighth row
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tC = tmem_base + lane_base + C::TM_C0;
         const int group = a.H_v / a.H_qk;
+        constexpr uint32_t idescC = ptx::umma_idesc_tf32_f32(128, D);
+        unsigned char *opA_hi = smem + C::OFF_CA_HI, *opA_lo = smem + C::OFF_CA_LO, *opB = smem + C::OFF_CB;
+        const int op_off = (t >> 3) * 128 + (t & 7) * 16;  // this thread's row in a core-matrix column
+        uint32_t rounds = 0;  // completed rank-P products: parity of cmma_done
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
             const int item = item_of(kk);
@@ -371,66 +390,79 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const PathMeta *pm = reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA);
             const int plen = pm->plen;
             if (plen >= 0) {
-                const int b = item / a.H_v, h = item - b * a.H_v;
-                unsigned char *tile = stage + C::OFF_S0 + (cc >> 3) * C::S0_HALF;
+                const int h = item % a.H_v;
                 const __nv_bfloat16 *kp = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_KP);
                 const float *up = reinterpret_cast<const float *>(stage + C::OFF_UP);
-                const float ga = pm->ga;
-                const int cnt = min(plen, C::PCH);
+                const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(pv.k);
+                unsigned long long m = pm->mask;  // path nodes not yet taken (rounds beyond the staged rows)
+                bool ok = true;
 #pragma unroll 1
-                for (int pass = 0; pass < 2; ++pass) {
-                    float acc[8][8];
-#pragma unroll
-                    for (int it = 0; it < 8; ++it) {
-                        const int r = r0 + 8 * (pass * 8 + it);
-                        widen8(*reinterpret_cast<const uint4 *>(tile + r * 128 + (((cc & 7) ^ (r & 7)) << 4)), acc[it]);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[it][e] *= ga;
-                    }
-                    for (int p = 0; p < cnt; ++p) {
-                        const float w = pm->w[p];
-                        float kf[8];
-                        widen8(*reinterpret_cast<const uint4 *>(kp + p * D + cc * 8), kf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) kf[e] *= w;
-#pragma unroll
-                        for (int it = 0; it < 8; ++it) {
-                            const float u = up[p * D + r0 + 8 * (pass * 8 + it)];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
-                        }
-                    }
-                    if (plen > C::PCH) {  // deep path: remaining nodes straight from global memory
-                        const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(pv.k);
-                        unsigned long long m = pm->mask;
-                        for (int q = 0; q < C::PCH; ++q) m &= m - 1;
-                        while (m) {
-                            const int j = __ffsll((long long)m) - 1;
-                            m &= m - 1;
-                            const float w = expf(pm->La - pv.cum_log_gate[(size_t)(pm->lo + j) * a.H_v + h]);
-                            float kf[8];
-                            widen8(*reinterpret_cast<const uint4 *>(kg + ((size_t)(pm->lo + j) * a.H_qk + h / group) * D + cc * 8),
-                                   kf);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) kf[e] *= w;
-                            const float *ur = pv.U + ((size_t)(pm->lo + j) * a.H_v + h) * D;
-#pragma unroll
-                            for (int it = 0; it < 8; ++it) {
-                                const float u = ur[r0 + 8 * (pass * 8 + it)];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
+                for (int r0 = 0; r0 < plen && ok; r0 += 8) {
+#pragma unroll 1
+                    for (int p = 0; p < 8; ++p) {  // (rolled: code size)
+                        float av = 0.f, bv = 0.f;
+                        if (r0 + p < plen) {
+                            if (r0 == 0) {  // staged by the producer (C::PCH = 8 rows)
+                                av = pm->w[p] * up[p * D + t];
+                                bv = __bfloat162float(kp[p * D + t]);
+                            } else {  // deep path: straight from global memory
+                                const int j = __ffsll((long long)m) - 1;
+                                const float w = __expf(pm->La - pv.cum_log_gate[(size_t)(pm->lo + j) * a.H_v + h]);
+                                av = w * pv.U[((size_t)(pm->lo + j) * a.H_v + h) * D + t];
+                                bv = __bfloat162float(kg[((size_t)(pm->lo + j) * a.H_qk + h / group) * D + t]);
                             }
                         }
+                        m &= m - 1;
+                        const int off = (p >> 2) * C::COPS_LBO + op_off + (p & 3) * 4;
+                        const float hi = ptx::tf32_hi(av);
+                        *reinterpret_cast<float *>(opA_hi + off) = hi;
+                        *reinterpret_cast<float *>(opA_lo + off) = av - hi;
+                        *reinterpret_cast<float *>(opB + off) = bv;
                     }
-#pragma unroll
-                    for (int it = 0; it < 8; ++it) {
-                        const int r = r0 + 8 * (pass * 8 + it);
-                        uint4 y;
-                        y.x = pack_bf16(acc[it][0], acc[it][1]), y.y = pack_bf16(acc[it][2], acc[it][3]);
-                        y.z = pack_bf16(acc[it][4], acc[it][5]), y.w = pack_bf16(acc[it][6], acc[it][7]);
-                        *reinterpret_cast<uint4 *>(tile + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = y;
+                    ptx::fence_proxy_async();  // operands were written by ordinary stores
+                    ptx::tc_fence_before_sync();
+                    ptx::named_sync(3, C::CGROUP > 0 ? C::CGROUP : 32);
+                    if (t == 0) {
+                        ptx::tc_fence_after_sync();
+                        const uint64_t dB = ptx::umma_desc_k_plain(ptx::smem_u32(opB), C::COPS_LBO, 128);
+                        ptx::umma_tf32(tmem_base + C::TM_C0, ptx::umma_desc_k_plain(ptx::smem_u32(opA_hi), C::COPS_LBO, 128),
+                                       dB, idescC, r0 > 0);
+                        ptx::umma_tf32(tmem_base + C::TM_C0, ptx::umma_desc_k_plain(ptx::smem_u32(opA_lo), C::COPS_LBO, 128),
+                                       dB, idescC, 1u);
+                        ptx::umma_commit(cmma_done);
                     }
+                    ok = ptx::mbar_wait(cmma_done, rounds & 1);
+                    ++rounds;
+                    ptx::tc_fence_after_sync();
                 }
+                // S[t][:] = g_a S[t][:] + C[t][:], sixteen columns at a time (rolled: code size)
+                const float ga = pm->ga;
+                unsigned char *row = stage + C::OFF_S0 + t * 128;
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 16) {
+                    uint32_t d[16];
+                    ptx::tmem_ld16(tC + c0, d);
+                    unsigned char *half = row + (c0 >> 6) * C::S0_HALF;
+                    const int ch = (c0 & 63) >> 3;  // 16-byte chunk inside the 128-byte row
+                    uint4 *p0 = reinterpret_cast<uint4 *>(half + (((ch) ^ (t & 7)) << 4));
+                    uint4 *p1 = reinterpret_cast<uint4 *>(half + (((ch + 1) ^ (t & 7)) << 4));
+                    float s0[8], s1[8];
+                    widen8(*p0, s0);
+                    widen8(*p1, s1);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        s0[e] = fmaf(ga, s0[e], plen > 0 ? __uint_as_float(d[e]) : 0.f);
+                        s1[e] = fmaf(ga, s1[e], plen > 0 ? __uint_as_float(d[8 + e]) : 0.f);
+                    }
+                    uint4 y0, y1;
+                    y0.x = pack_bf16(s0[0], s0[1]), y0.y = pack_bf16(s0[2], s0[3]);
+                    y0.z = pack_bf16(s0[4], s0[5]), y0.w = pack_bf16(s0[6], s0[7]);
+                    y1.x = pack_bf16(s1[0], s1[1]), y1.y = pack_bf16(s1[2], s1[3]);
+                    y1.z = pack_bf16(s1[4], s1[5]), y1.w = pack_bf16(s1[6], s1[7]);
+                    *p0 = y0, *p1 = y1;
+                }
+                ptx::tc_fence_before_sync();
                 ptx::fence_proxy_async();  // the tile is read next by the tensor core and by the TMA store
             }
             ptx::named_sync(3, C::CGROUP > 0 ? C::CGROUP : 32);
