@@ -63,7 +63,8 @@ __device__ __forceinline__ float warp_sum(float x)
 
 __device__ __forceinline__ int nth_set_bit(unsigned long long m, int p)
 {
-    for (int q = 0; q < p; ++q) m &= m - 1;
+#pragma unroll 1
+    for (int q = 0; q < p; ++q) m &= m - 1;  // (rolled: the callers' code has to stay small)
     return __ffsll((long long)m) - 1;
 }
 

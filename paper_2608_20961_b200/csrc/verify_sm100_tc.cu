@@ -266,6 +266,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     p.pbad = TREEWY_SEQ_TOO_MANY_NODES;
                 } else {
                     int bp = 0;
+#pragma unroll 1
                     for (int i = lane; i < pn; i += 32) {
                         const int par = pv.parent[p.plo + i];
                         bp |= (par < -1 || par >= i);
@@ -398,26 +399,45 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 bool ok = true;
 #pragma unroll 1
                 for (int r0 = 0; r0 < plen && ok; r0 += 8) {
+                    if (r0 == 0) {  // the rows the producer staged (C::PCH = 8)
+                        float av[8], bv[8];
+#pragma unroll
+                        for (int p = 0; p < 8; ++p) {
+                            const float u = up[p * D + t], kf = __bfloat162float(kp[p * D + t]);
+                            av[p] = p < plen ? pm->w[p] * u : 0.f;  // rows past the path hold stale data
+                            bv[p] = p < plen ? kf : 0.f;
+                        }
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            float4 hi, lo;
+                            hi.x = ptx::tf32_hi(av[4 * c]), hi.y = ptx::tf32_hi(av[4 * c + 1]);
+                            hi.z = ptx::tf32_hi(av[4 * c + 2]), hi.w = ptx::tf32_hi(av[4 * c + 3]);
+                            lo.x = av[4 * c] - hi.x, lo.y = av[4 * c + 1] - hi.y;
+                            lo.z = av[4 * c + 2] - hi.z, lo.w = av[4 * c + 3] - hi.w;
+                            *reinterpret_cast<float4 *>(opA_hi + c * C::COPS_LBO + op_off) = hi;
+                            *reinterpret_cast<float4 *>(opA_lo + c * C::COPS_LBO + op_off) = lo;
+                            *reinterpret_cast<float4 *>(opB + c * C::COPS_LBO + op_off) =
+                                make_float4(bv[4 * c], bv[4 * c + 1], bv[4 * c + 2], bv[4 * c + 3]);
+                        }
 #pragma unroll 1
-                    for (int p = 0; p < 8; ++p) {  // (rolled: code size)
-                        float av = 0.f, bv = 0.f;
-                        if (r0 + p < plen) {
-                            if (r0 == 0) {  // staged by the producer (C::PCH = 8 rows)
-                                av = pm->w[p] * up[p * D + t];
-                                bv = __bfloat162float(kp[p * D + t]);
-                            } else {  // deep path: straight from global memory
+                        for (int p = 0; p < 8; ++p) m &= m - 1;
+                    } else {  // deep path: straight from global memory, one node at a time (rolled: code size)
+#pragma unroll 1
+                        for (int p = 0; p < 8; ++p) {
+                            float av = 0.f, bv = 0.f;
+                            if (r0 + p < plen) {
                                 const int j = __ffsll((long long)m) - 1;
                                 const float w = __expf(pm->La - pv.cum_log_gate[(size_t)(pm->lo + j) * a.H_v + h]);
                                 av = w * pv.U[((size_t)(pm->lo + j) * a.H_v + h) * D + t];
                                 bv = __bfloat162float(kg[((size_t)(pm->lo + j) * a.H_qk + h / group) * D + t]);
                             }
+                            m &= m - 1;
+                            const int off = (p >> 2) * C::COPS_LBO + op_off + (p & 3) * 4;
+                            const float hi = ptx::tf32_hi(av);
+                            *reinterpret_cast<float *>(opA_hi + off) = hi;
+                            *reinterpret_cast<float *>(opA_lo + off) = av - hi;
+                            *reinterpret_cast<float *>(opB + off) = bv;
                         }
-                        m &= m - 1;
-                        const int off = (p >> 2) * C::COPS_LBO + op_off + (p & 3) * 4;
-                        const float hi = ptx::tf32_hi(av);
-                        *reinterpret_cast<float *>(opA_hi + off) = hi;
-                        *reinterpret_cast<float *>(opA_lo + off) = av - hi;
-                        *reinterpret_cast<float *>(opB + off) = bv;
                     }
                     ptx::fence_proxy_async();  // operands were written by ordinary stores
                     ptx::tc_fence_before_sync();
@@ -435,13 +455,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     ++rounds;
                     ptx::tc_fence_after_sync();
                 }
-                // S[t][:] = g_a S[t][:] + C[t][:], sixteen columns at a time (rolled: code size)
+                // S[t][:] = g_a S[t][:] + C[t][:], sixteen columns at a time; the next sixteen columns of
+                // C are on their way from tensor memory while the current ones are worked on
                 const float ga = pm->ga;
                 unsigned char *row = stage + C::OFF_S0 + t * 128;
-#pragma unroll 1
-                for (int c0 = 0; c0 < D; c0 += 16) {
-                    uint32_t d[16];
-                    ptx::tmem_ld16(tC + c0, d);
+                auto fix16 = [&](int c0, const uint32_t (&d)[16]) {
                     unsigned char *half = row + (c0 >> 6) * C::S0_HALF;
                     const int ch = (c0 & 63) >> 3;  // 16-byte chunk inside the 128-byte row
                     uint4 *p0 = reinterpret_cast<uint4 *>(half + (((ch) ^ (t & 7)) << 4));
@@ -449,11 +467,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     float s0[8], s1[8];
                     widen8(*p0, s0);
                     widen8(*p1, s1);
-                    ptx::tmem_wait_ld();
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        s0[e] = fmaf(ga, s0[e], plen > 0 ? __uint_as_float(d[e]) : 0.f);
-                        s1[e] = fmaf(ga, s1[e], plen > 0 ? __uint_as_float(d[8 + e]) : 0.f);
+                        s0[e] = fmaf(ga, s0[e], __uint_as_float(d[e]));
+                        s1[e] = fmaf(ga, s1[e], __uint_as_float(d[8 + e]));
                     }
                     uint4 y0, y1;
                     y0.x = pack_bf16(s0[0], s0[1]), y0.y = pack_bf16(s0[2], s0[3]);
@@ -461,20 +478,23 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     y1.x = pack_bf16(s1[0], s1[1]), y1.y = pack_bf16(s1[2], s1[3]);
                     y1.z = pack_bf16(s1[4], s1[5]), y1.w = pack_bf16(s1[6], s1[7]);
                     *p0 = y0, *p1 = y1;
+                };
+                uint32_t da[16], db[16];
+                ptx::tmem_ld16(tC, da);
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    ptx::tmem_wait_ld();
+                    ptx::tmem_ld16(tC + c0 + 16, db);
+                    fix16(c0, da);
+                    ptx::tmem_wait_ld();
+                    if (c0 + 32 < D) ptx::tmem_ld16(tC + c0 + 32, da);
+                    fix16(c0 + 16, db);
                 }
                 ptx::tc_fence_before_sync();
                 ptx::fence_proxy_async();  // the tile is read next by the tensor core and by the TMA store
             }
-            ptx::named_sync(3, C::CGROUP > 0 ? C::CGROUP : 32);
-            if (plen >= 0 && t == 0) {
-                ptx::tma_store_2d(&tmS0, 0, item * D, stage + C::OFF_S0);
-                ptx::tma_store_2d(&tmS0, 64, item * D, stage + C::OFF_S0 + C::S0_HALF);
-                ptx::bulk_commit_group();
-                ptx::bulk_wait_group_read<0>();  // the tile will be overwritten by scratch after the MMAs
-            }
-            ptx::mbar_arrive_warp(&upd_done[s]);
+            ptx::mbar_arrive_warp(&upd_done[s]);  // (the first stage-1 MMA warp sends the new state to global memory)
         }
-        if (t == 0) ptx::bulk_wait_group<0>();
     } else if (warp == C::MMA1_WARP || warp == C::MMA1B_WARP) {
         // ------------------------------------------------------------------ stage-1 MMAs
         // One tcgen05.mma of these sizes keeps its issuing thread for ~120 cycles, so the two
@@ -492,6 +512,16 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const bool reuse_gram = pair_mode && (kk & 1) && meta_nlo(stage)[2] == 0;
             const int n = gram_chain && reuse_gram ? 0 : meta_nlo(stage)[0];
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
+            bool stored = false;
+            if constexpr (FUSED) {
+                // the new state goes back to global memory while verification proceeds from this copy
+                if (!gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
+                    ptx::tma_store_2d(&tmS0, 0, item * D, stage + C::OFF_S0);
+                    ptx::tma_store_2d(&tmS0, 64, item * D, stage + C::OFF_S0 + C::S0_HALF);
+                    ptx::bulk_commit_group();
+                    stored = true;
+                }
+            }
             if (gram_chain) {
                 if (!ptx::mbar_wait(&r_free[kk % C::RBUF], ((kk / C::RBUF) & 1) ^ 1)) break;
             } else {
@@ -514,13 +544,18 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                             ptx::umma_bf16(d1, da, dq, idesc1, ks > 0);
                         }
                     }
+                    // (the Gram warps may write their stash over the state tile once stage 1 is done: the
+                    // store must have read it by then)
+                    if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::umma_commit(&mma1_done[buf]);
                 } else {
+                    if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::mbar_arrive(&mma1_done[buf]);
                 }
             }
             __syncwarp();
         }
+        if (FUSED && !gram_chain && lane == 0) ptx::bulk_wait_group<0>();
     } else if (warp == C::MMA2_WARP) {
         // ------------------------------------------------------------------ stage-2 MMAs
         constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
@@ -648,6 +683,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     float *Pp = reinterpret_cast<float *>(stage + C::OFF_DPP);
                     unsigned char *idx = stage + C::OFF_DIDX;
                     uint32_t m = valid ? (uint32_t)meta_mask(stage)[i] & ~(1u << i) : 0u;
+#pragma unroll 1
                     for (int d = 0; m; ++d) {
                         const int j = __ffs(m) - 1;
                         m &= m - 1;
@@ -774,15 +810,18 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     } else {  // deep paths: the same recurrence through shared memory
                         float *x = xr + (wrow ? i : NP + i) * C::XLD;
                         x[dp] = top;
+#pragma unroll 1
                         for (int e = dp - 1; e >= 0; --e) {
                             const int col_e = ((e >> 2) * NP) * 4 + (e & 3);
                             float acc = wrow ? Pp[col_e + i * 4] : 0.f;
+#pragma unroll 1
                             for (int f = e + 1; f <= dp; ++f) {
                                 const int jf = (f == dp) ? i : idx[((f >> 2) * NP + i) * 4 + (f & 3)];
                                 acc = fmaf(-x[f], Ap[col_e + jf * 4], acc);
                             }
                             x[e] = acc;
                         }
+#pragma unroll 1
                         for (int e = 0; e <= dp; ++e) {
                             const int col = (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)];
                             const float val = x[e], hi = ptx::tf32_hi(val);
