@@ -57,7 +57,7 @@ constexpr uint32_t VT_TMEM_COLS = 512;
 template <int NP, bool FUSED> struct VtCfg {
     static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
     static constexpr int SLOTS = 2;  // list / scalar / v-row buffers alternate between consecutive items
-    static constexpr int STAGES = FUSED ? 3 : 4;
+    static constexpr int STAGES = (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     // (fused mode gives 128 columns of tensor memory to the commit's accumulator)
     static constexpr int TBUF = FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
@@ -128,6 +128,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int TM_RHI = 0, TM_RLO = NP;
     static constexpr int TM_C0 = TM_R0 + RBUF * 2 * NP;  // fused mode: the commit's 128 x 128 accumulator
     static_assert(TM_C0 + (FUSED ? D : 0) <= 512, "tensor memory");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 };
 
 // fused mode: what the commit of the previous round needs for one (sequence, head)
