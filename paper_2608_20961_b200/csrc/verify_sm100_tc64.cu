@@ -219,13 +219,13 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                 if (n > 0) {
                     const uint32_t qk = ptx::smem_u32(stage), s0 = qk + V6_OFF_S0;
                     const uint32_t d1 = tmem_base + buf * V6_TM_COLS + V6_TM_SQ, d2 = tmem_base + buf * V6_TM_COLS + V6_TM_D2;
-#pragma unroll
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks & 3) * 32;
                         ptx::umma_bf16(d1, ptx::umma_desc_k_sw128(s0 + (ks >> 2) * V6_S0_HALF + ko),
                                        ptx::umma_desc_k_sw128(qk + (ks >> 2) * V6_QK_HALF + ko), idesc1, ks > 0);
                     }
-#pragma unroll
+#pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t base = qk + (ks >> 2) * V6_QK_HALF + (ks & 3) * 32;
                         ptx::umma_bf16(d2, ptx::umma_desc_k_sw128(base), ptx::umma_desc_k_sw128(base + NP * 128),
@@ -312,7 +312,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                     float *raw = reinterpret_cast<float *>(stage);  // over the dead [Q;K] / S0 tiles
 
                     // ---- G1: every thread's Gram row (q row of node t, or k row of node t - 64)
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < NP; c0 += 16) {
                         if (c0 < n) {
                             uint32_t g[16];
@@ -339,6 +339,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                         const float scale = a_kind ? bi : 1.f;
                         const float *row = raw + t * V6_RLD;
                         unsigned long long m = mi & ~(1ull << i);
+#pragma unroll 1
                         for (int d = 0; d < dp; d += 2) {  // two ancestors per round: independent chains
                             const int j0 = __ffsll((long long)m) - 1;
                             m &= m - 1;
@@ -415,8 +416,10 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                             }
                         } else {  // deep paths: x_e is kept in the hi tile at its final column
                             *reinterpret_cast<float *>(Mhi + v6_tile_off(i, i)) = top;
+#pragma unroll 1
                             for (int e = dp - 1; e >= 0; --e) {
                                 float acc = wrow ? Pp[v6_at(i, e)] : 0.f;
+#pragma unroll 1
                                 for (int f = e + 1; f <= dp; ++f) {
                                     const int j = (f == dp) ? i : idx[v6_at(i, f)];
                                     acc = fmaf(-*reinterpret_cast<const float *>(Mhi + v6_tile_off(i, j)),
@@ -424,6 +427,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                                 }
                                 *reinterpret_cast<float *>(Mhi + v6_tile_off(i, idx[v6_at(i, e)])) = acc;
                             }
+#pragma unroll 1
                             for (int e = 0; e <= dp; ++e) {
                                 const int off = v6_tile_off(i, (e == dp) ? i : idx[v6_at(i, e)]);
                                 const float val = *reinterpret_cast<const float *>(Mhi + off), hi = ptx::tf32_hi(val);
@@ -435,7 +439,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
 
                     // ---- R: row t of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j), hi | lo into tensor
                     // memory over the consumed Gram columns; then g_i (S0 q_i) in place
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < NP; c0 += 16) {
                         uint32_t hi[16], lo[16];
                         if (c0 < n) {
@@ -460,7 +464,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                         ptx::tmem_st16(tm + V6_TM_D2 + c0, hi);
                         ptx::tmem_st16(tm + V6_TM_RLO + c0, lo);
                     }
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < NP; c0 += 16) {
                         if (c0 < n) {
                             uint32_t sq[16];
@@ -494,7 +498,7 @@ verify_sm100_tc64_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUte
                 if (n > 0) {
                     float *Ub = a.U + ((size_t)lo * a.H_v + h) * D + t;
                     TOut *Ob = Og + ((size_t)lo * a.H_v + h) * D + t;
-#pragma unroll
+#pragma unroll 1
                     for (int c0 = 0; c0 < NP; c0 += 16) {
                         if (c0 < n) {
                             uint32_t du[16], dout[16];
