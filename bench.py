@@ -362,6 +362,15 @@ def run_ours(args, rank: int, size: int, local: int):
                     "time_over_commit": snap_ms / kt[2],
                     "state_bytes_over_commit": snap_bytes / (w.B * w.H_v * 128 * 128 * w.S0.element_size())}
 
+    set_bytes = sum(t.numel() * t.element_size()
+                    for t in (sets[0].S0, sets[0].q, sets[0].k, sets[0].v, sets[0].O, sets[0].U))
+    if set_bytes > 126e6:
+        l2_note = (f"inputs larger than L2: two layer sets ({set_bytes / 1e9:.2f} GB each) rotated, commit "
+                   "runs one step after its verify")
+    else:
+        l2_note = (f"two layer sets ({set_bytes / 1e6:.0f} MB each, {2 * set_bytes / 1e6:.0f} MB together against a "
+                   "126 MB L2) rotated, commit runs one step after its verify: this small configuration is "
+                   "partly L2-resident and is not the headline workload")
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -369,8 +378,7 @@ def run_ours(args, rank: int, size: int, local: int):
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "H_v": w.H_v, "H_qk": w.H_qk, "T": w.T,
                    "max_nodes": w.max_nodes, "seed": w.seed,
-                   "l2": "inputs larger than L2: two layer sets (~0.6 GB each) rotated, commit "
-                         "runs one step after its verify",
+                   "l2": l2_note,
                    "parallelism": f"replicas x{size}, no collective"},
         "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 3 * args.steps,
         "roofline": roofline,

@@ -95,3 +95,28 @@ def test_fused_falls_back_for_large_new_trees():
     w2.H_qk = w1.H_qk
     w2.q, w2.k = w2.q[:, :w1.H_qk].contiguous(), w2.k[:, :w1.H_qk].contiguous()
     _check(w1, w2, 32, 64)
+
+
+def test_fused_round_matches_the_oracle(oracle):
+    """Two rounds against the oracle itself (not against the two-kernel path): round 1 is verified
+    and committed by the oracle, its committed state -- rounded to the bf16 the library stores --
+    starts the oracle's round 2; the GPU runs verify(1), then commit(1) + verify(2) in ONE kernel."""
+    import numpy as np
+    from tests import parity_util as pu
+    w1 = wl.make_workload(2, seed=31, B=6, H_v=4)
+    w2 = wl.make_workload(2, seed=32, B=6, H_v=4)
+    _, ref1 = pu.run_oracle(oracle, w1)
+    w2.S0 = torch.from_numpy(ref1.S_commit).to(torch.bfloat16)
+    _, ref2 = pu.run_oracle(oracle, w2)
+    S, O, U, status = _two_rounds(w1, w2, True, 32, 32)
+    assert not status.any()
+    off = w2.node_offsets.numpy()
+    for name, got, want, offs, per_node in (
+            ("O", O.double().numpy(), ref2.O, off, True), ("U", U.double().numpy(), ref2.U, off, True),
+            ("S", S.double().numpy(), ref1.S_commit, np.arange(w1.B + 1), False)):
+        m, f = pu.worst_errors(got, want, offs, per_node)
+        # (the stored state is bf16: its largest elements are off by up to 2^-9 of their own size, which
+        # is why the max-abs gate is applied to the fp32 outputs and the Frobenius gate to all three)
+        assert f <= pu.FROB_GATE and (name == "S" or m <= pu.MAXABS_GATE), (name, m, f)
+    want = torch.from_numpy(ref1.S_commit).to(torch.bfloat16).float()
+    assert not bool(((S.float() - want).abs() > 2.0 ** -7 * want.abs() + 1e-6 * float(want.abs().max())).any())
