@@ -55,17 +55,20 @@ namespace treewy {
 constexpr uint32_t VT_TMEM_COLS = 512;
 
 template <int NP, bool FUSED> struct VtCfg {
-    static_assert(NP == 16 || NP == 32, "tensor-core solve is built for up to 32 nodes");
+    static_assert(NP == 16 || NP == 32 || (NP == 64 && !FUSED), "up to 64 nodes; the fused mode up to 32");
+    static constexpr bool BIG = NP == 64;  // 33..64 nodes: shared memory and tensor memory hold two items
+    static constexpr int NPL = (NP + 31) / 32;  // nodes per producer lane
     static constexpr int SLOTS = 2;  // list / scalar / v-row buffers alternate between consecutive items
-    static constexpr int STAGES = (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
+    static constexpr int STAGES = BIG ? 2 : (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     // (fused mode gives 128 columns of tensor memory to the commit's accumulator)
-    static constexpr int TBUF = FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
-    static constexpr int RBUF = FUSED ? 2 : 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
+    static constexpr int TBUF = BIG ? 2 : FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
+    static constexpr int RBUF = BIG ? 2 : FUSED ? 2 : 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
     // every phase of an item has its own warps, and every role walks all items in order
-    static constexpr int G_THREADS = 64, T_THREADS = 64, R_THREADS = 128, E_THREADS = 128;
-    static constexpr int G_WARP0 = 0, T_WARP0 = 2, R_WARP0 = 4, E_WARP0 = 8;  // R / E: warp % 4 = TMEM lane quarter
-    static constexpr int COMMIT_WARP0 = 12;
+    static constexpr int G_THREADS = BIG ? 128 : 64, T_THREADS = BIG ? 128 : 64, R_THREADS = 128, E_THREADS = 128;
+    static constexpr int G_WARP0 = 0, T_WARP0 = G_THREADS / 32, R_WARP0 = T_WARP0 + T_THREADS / 32;
+    static constexpr int E_WARP0 = R_WARP0 + 4;  // Gram (when 4 warps) / R / E: warp % 4 = TMEM lane quarter
+    static constexpr int COMMIT_WARP0 = E_WARP0 + 4;
     static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
     static constexpr int MMA1B_WARP = MMA1_WARP + 1;  // the Gram chain of stage 1 has its own issuing warp
     static constexpr int MMA2_WARP = MMA1B_WARP + 1;
@@ -88,19 +91,27 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int META_BYTES = META_IDX + 2 * NP * 4;
     static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
     static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
-    // stage-2 operands, fp32 rows of 32 columns (128 bytes, 128-byte swizzle), overlaying dead tiles
-    // (W rows above T rows: [W;T] is one B operand of 2 NP rows, so one MMA yields O and U together)
-    static constexpr int OFF_W_HI = 0, OFF_T_HI = NP * 128, OFF_W_LO = 2 * NP * 128, OFF_T_LO = 3 * NP * 128;
-    static_assert(4 * NP * 128 <= QK_BYTES, "operand overlays fit");
-    // scratch over the dead S0 tile, used before R^T is written there: the raw Gram rows and the
-    // back-substitution rows of deep paths
+    // stage-2 B operand [W;T]: 2 NP rows (W rows above T rows, so one MMA yields O and U together)
+    // of NP fp32 columns, as atoms of 2 NP rows x 128 bytes (32 columns) with the 128-byte swizzle,
+    // once for the hi parts and once for the lo parts; they overlay the stage's dead tiles
+    static constexpr int ATOM = 2 * NP * 128, NATOM = BIG ? 2 : 1;
+    static constexpr int OFF_W_HI = 0, OFF_T_HI = NP * 128;
+    static constexpr int OFF_W_LO = NATOM * ATOM, OFF_T_LO = OFF_W_LO + NP * 128;
+    static constexpr int TILE_BYTES = 2 * NATOM * ATOM;
+    static_assert(TILE_BYTES <= (BIG ? QK_BYTES + S0_BYTES : QK_BYTES), "operand overlays fit");
+    // scratch over the dead tiles: the raw Gram rows (up to 32 nodes: in the S0 tile, beside the B
+    // tiles; 64 nodes: under the B tiles, which are zeroed once the lists are built) and, up to 32
+    // nodes, the back-substitution rows of deep paths
     static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
     static constexpr int XLD = NP + 1;
-    static constexpr int OFF_RAW = OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;
-    // ... and, for trees with a path of more than 8 ancestors, the full-length lists
+    static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;
+    static_assert(OFF_RAW + 2 * NP * RLD * 4 <= OFF_S0 + S0_BYTES, "Gram stash fits");
+    // ... and, for trees with a path of more than 8 ancestors, the full-length lists (64 nodes: in an
+    // area of their own, since the B tiles take both dead tiles)
     static constexpr int OFF_DAP = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 15) / 16 * 16;
     static constexpr int OFF_DPP = OFF_DAP + NP * NP * 4, OFF_DIDX = OFF_DPP + NP * NP * 4;
-    static_assert(OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
+    static_assert(BIG || OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
+    static constexpr int DEEP_BYTES = BIG ? 2 * NP * NP * 4 + NP * NP : 0;
     static constexpr int V_BYTES = NP * D * 2;
     // group-private: path lists of the first 8 ancestors, per-node scalars (double-buffered), and
     // the v rows [NP][128] bf16 of the group's next item (loaded one item ahead)
@@ -108,7 +119,8 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int GP_VS = (GP_SCAL + NP * 16 + 127) / 128 * 128;
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
-    static constexpr int OFF_EINFO = OFF_GP + SLOTS * GP_BYTES;  // (n, first node) of the item in a TMEM block
+    static constexpr int OFF_DEEP = OFF_GP + SLOTS * GP_BYTES;  // 64 nodes: full-length lists of deep trees
+    static constexpr int OFF_EINFO = OFF_DEEP + DEEP_BYTES;      // (n, first node) of the item in a TMEM block
     // fused mode: operands of the commit's rank-P product, K-major without swizzle, K = 8 path nodes:
     // core matrices of 8 rows x 16 bytes, the two K halves COPS_LBO apart
     static constexpr int COPS_LBO = D * 16, COPS_TILE = 2 * COPS_LBO;
@@ -212,6 +224,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
     auto meta_rat = [&](unsigned char *stage) { return reinterpret_cast<float4 *>(stage + C::OFF_META + C::META_RAT); };
     auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
+    // byte offset of element (row, col) of a stage-2 B tile (atoms of 32 columns, 128-byte swizzle)
+    auto tile_off = [](int row, int col) {
+        return (col >> 5) * C::ATOM + row * 128 + (((((col & 31) >> 2)) ^ (row & 7)) << 4) + ((col & 3) << 2);
+    };
 
     if (warp >= C::PROD_WARP0) {
         // ------------------------------------------------------------------ producer warp
@@ -226,8 +242,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // dependent chain  node_offsets -> parent / mask / log-gate / beta  never delays a TMA issue.
         struct Pre {
             int item, b, h, lo, n, bad, flag;
-            unsigned long long mk;
-            float Lv, bv;
+            unsigned long long mk[C::NPL];  // lane l owns nodes l, l + 32
+            float Lv[C::NPL], bv[C::NPL];
             int deep;  // whether any path has more than 8 ancestors
             // fused mode: the previous round's accepted path of this sequence
             int plo, pbad, plen, cnt, pj;
@@ -237,7 +253,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         auto fetch = [&](int kk) {
             Pre p;
             p.item = item_of(kk);
-            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.mk = 0ull, p.Lv = 0.f, p.bv = 0.f;
+            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1;
+#pragma unroll
+            for (int r = 0; r < C::NPL; ++r) p.mk[r] = 0ull, p.Lv[r] = 0.f, p.bv[r] = 0.f;
             p.deep = 0;
             p.plo = 0, p.pbad = 0, p.plen = -1, p.cnt = 0, p.pj = 0, p.pmask = 0ull, p.La = 0.f, p.wj = 0.f;
             if (p.item >= n_items) return p;
@@ -251,14 +269,26 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 p.bad = TREEWY_SEQ_TOO_MANY_NODES;  // another launch's size class: skipped, not flagged
                 p.flag = 0;
             } else {
-                const int par = lane < p.n ? a.parent[p.lo + lane] : -1;
-                if (__any_sync(0xffffffffu, lane < p.n && (par < -1 || par >= lane))) p.bad = TREEWY_SEQ_BAD_PARENT;
+                bool bp = false;
+#pragma unroll
+                for (int r = 0; r < C::NPL; ++r) {
+                    const int i = lane + 32 * r;
+                    const int par = i < p.n ? a.parent[p.lo + i] : -1;
+                    bp |= i < p.n && (par < -1 || par >= i);
+                }
+                if (__any_sync(0xffffffffu, bp)) p.bad = TREEWY_SEQ_BAD_PARENT;
             }
-            const bool on = !p.bad && lane < p.n;  // NP <= 32: one node per lane
-            p.mk = on ? a.anc_mask[p.lo + lane] : 0ull;
-            p.Lv = on ? a.cum_log_gate[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
-            p.bv = on ? a.beta[(size_t)(p.lo + lane) * a.H_v + p.h] : 0.f;
-            p.deep = __any_sync(0xffffffffu, __popc((uint32_t)p.mk & ~(1u << lane)) > 8);
+            bool dp8 = false;
+#pragma unroll
+            for (int r = 0; r < C::NPL; ++r) {
+                const int i = lane + 32 * r;
+                const bool on = !p.bad && i < p.n;
+                p.mk[r] = on ? a.anc_mask[p.lo + i] : 0ull;
+                p.Lv[r] = on ? a.cum_log_gate[(size_t)(p.lo + i) * a.H_v + p.h] : 0.f;
+                p.bv[r] = on ? a.beta[(size_t)(p.lo + i) * a.H_v + p.h] : 0.f;
+                dp8 |= __popcll(p.mk[r] & ~(1ull << i)) > 8;
+            }
+            p.deep = __any_sync(0xffffffffu, dp8);
             if constexpr (FUSED) {
                 p.plo = pv.node_offsets[p.b];
                 const int pn = pv.node_offsets[p.b + 1] - p.plo;
@@ -299,7 +329,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], TREEWY_SEQ_TIMEOUT);
                 break;
             }
-            if (lane < NP) meta_mask(stage)[lane] = p.mk, meta_L(stage)[lane] = p.Lv, meta_beta(stage)[lane] = p.bv;
+#pragma unroll
+            for (int r = 0; r < C::NPL; ++r) {
+                const int i = lane + 32 * r;
+                if (i < NP) meta_mask(stage)[i] = p.mk[r], meta_L(stage)[i] = p.Lv[r], meta_beta(stage)[i] = p.bv[r];
+            }
             if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep;
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
@@ -340,16 +374,21 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 // Path lists of the node this lane owns: index and gate ratio e^{L_i - L_j} of its first
                 // 8 ancestors.  Only the ratios depend on the head; building them here takes the
                 // ffs / exp chain off the consumers' critical path.  (Rolled: code size.)
-                uint32_t m = (uint32_t)p.mk & ~(1u << lane);
-                float *ratp = reinterpret_cast<float *>(meta_rat(stage)) + lane * 4;
-                unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(stage)) + lane * 4;
+                __syncwarp();  // the log-gates of all nodes are in the meta block
+                const float *Lm = meta_L(stage);
+#pragma unroll
+                for (int r = 0; r < C::NPL; ++r) {
+                    const int i = lane + 32 * r;
+                    unsigned long long m = p.mk[r] & ~(1ull << i);
+                    float *ratp = reinterpret_cast<float *>(meta_rat(stage)) + i * 4;
+                    unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(stage)) + i * 4;
 #pragma unroll 1
-                for (int d = 0; d < 8; ++d) {
-                    const int j = m ? __ffs(m) - 1 : 0;
-                    const float Lj = __shfl_sync(0xffffffffu, p.Lv, j);
-                    const float r = m ? __expf(p.Lv - Lj) : 0.f;
-                    if (lane < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = r, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
-                    m &= m - 1;
+                    for (int d = 0; d < 8; ++d) {
+                        const int j = m ? __ffsll((long long)m) - 1 : 0;
+                        const float rt = m ? __expf(p.Lv[r] - Lm[j]) : 0.f;
+                        if (i < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = rt, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
+                        m &= m - 1;
+                    }
                 }
             }
             __syncwarp();
@@ -580,7 +619,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     for (int q = 0; q < 3 * (NP / 8); ++q) {
                         const int p = q / (NP / 8), ks = q % (NP / 8);
                         const uint32_t ra = tr + (p == 1 ? C::TM_RLO : C::TM_RHI) + ks * 8;
-                        const uint32_t wt = base + (p == 2 ? C::OFF_W_LO : C::OFF_W_HI) + ks * 32;
+                        const uint32_t wt = base + (p == 2 ? C::OFF_W_LO : C::OFF_W_HI) + (ks >> 2) * C::ATOM + (ks & 3) * 32;
                         ptx::umma_tf32_ts(tb, ra, ptx::umma_desc_k_sw128(wt), idesc, 1u);
                     }
                     ptx::umma_commit(&mma2_done[buf]);
@@ -631,9 +670,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
                 // second item of a pair: same tree, same [Q;K] rows; the Gram entries are in registers
                 const bool reuse_gram = pair_mode && (kk & 1) && !deep;
-                // zero the T / W operand tiles (they overlay the dead [Q;K] tile)
-                for (int q = tg; q < 4 * NP * 128 / 16; q += C::G_THREADS)
-                    reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
+                // zero the stage-2 B tiles (they overlay the dead [Q;K] tile; with 64 nodes they also cover
+                // the Gram stash and are zeroed further down, once the lists are built)
+                if constexpr (!C::BIG) {
+                    for (int q = tg; q < C::TILE_BYTES / 16; q += C::G_THREADS)
+                        reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
+                }
                 // the rows of the Gram block (row owner = lane)
                 if (gram_reader && !reuse_gram) {
                     const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;
@@ -679,14 +721,18 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         val.z = scale * rt.z * gram4[q].z, val.w = scale * rt.w * gram4[q].w;
                         (kind ? Ap4 : Pp4)[hf * NP + i] = val;
                     }
-                } else if (tg < 2 * NP) {  // full-length lists, in the scratch over the dead S0 tile
-                    float *Ap = reinterpret_cast<float *>(stage + C::OFF_DAP);
-                    float *Pp = reinterpret_cast<float *>(stage + C::OFF_DPP);
-                    unsigned char *idx = stage + C::OFF_DIDX;
-                    uint32_t m = valid ? (uint32_t)meta_mask(stage)[i] & ~(1u << i) : 0u;
+                } else if (tg < 2 * NP) {  // full-length lists, in scratch memory
+                    if constexpr (C::BIG) {  // one area for both slots: the previous item's solve must be over
+                        if (kk >= 1) ptx::mbar_wait(&lists_free[(kk - 1) & 1], ((kk - 1) >> 1) & 1);
+                    }
+                    unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;
+                    float *Ap = reinterpret_cast<float *>(dl);
+                    float *Pp = reinterpret_cast<float *>(dl + NP * NP * 4);
+                    unsigned char *idx = dl + 2 * NP * NP * 4;
+                    unsigned long long m = valid ? meta_mask(stage)[i] & ~(1ull << i) : 0ull;
 #pragma unroll 1
                     for (int d = 0; m; ++d) {
-                        const int j = __ffs(m) - 1;
+                        const int j = __ffsll((long long)m) - 1;
                         m &= m - 1;
                         const float val = scale * __expf(Li - Lm[j]) * row[j];
                         const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
@@ -698,6 +744,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     const float gi = __expf(Li);
                     if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
                     scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
+                }
+                if constexpr (C::BIG) {  // the stash is dead: the B tiles take its place
+                    ptx::named_sync(1, C::G_THREADS);
+                    for (int q = tg; q < C::TILE_BYTES / 16; q += C::G_THREADS)
+                        reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
                 }
                 ptx::fence_proxy_async();  // the zero fill is read by the tensor core
             } else {
@@ -756,11 +807,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int n = meta_nlo(stage)[0];  // (the Gram warps read the meta block before they signalled)
             if (n > 0 && tt < 2 * NP && i < n) {
                 const bool deep = meta_nlo(stage)[2] != 0;
-                const float *Ap = reinterpret_cast<const float *>(stage + C::OFF_DAP);
-                const float *Pp = reinterpret_cast<const float *>(stage + C::OFF_DPP);
-                const unsigned char *idx = stage + C::OFF_DIDX;
+                const unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;  // full-length lists
+                const float *Ap = reinterpret_cast<const float *>(dl);
+                const float *Pp = reinterpret_cast<const float *>(dl + NP * NP * 4);
+                const unsigned char *idx = dl + 2 * NP * NP * 4;
                 float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
-                const int dp = __popc((uint32_t)meta_mask(stage)[i]) - 1;  // ancestors of node i
+                const int dp = __popcll(meta_mask(stage)[i]) - 1;  // ancestors of node i
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
@@ -804,9 +856,29 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         for (int e = 8; e >= 0; --e) {
                             const int col = jf[e];
                             const float hi = ptx::tf32_hi(x[e]);
-                            const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
+                            const int off = tile_off(i, col);
                             *reinterpret_cast<float *>(Mhi + off) = hi;
                             *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
+                        }
+                    } else if constexpr (C::BIG) {  // deep paths: x_e is kept in the hi tile at its final column
+                        *reinterpret_cast<float *>(Mhi + tile_off(i, i)) = top;
+#pragma unroll 1
+                        for (int e = dp - 1; e >= 0; --e) {
+                            const int col_e = ((e >> 2) * NP) * 4 + (e & 3);
+                            float acc = wrow ? Pp[col_e + i * 4] : 0.f;
+#pragma unroll 1
+                            for (int f = e + 1; f <= dp; ++f) {
+                                const int jf = (f == dp) ? i : idx[((f >> 2) * NP + i) * 4 + (f & 3)];
+                                acc = fmaf(-*reinterpret_cast<const float *>(Mhi + tile_off(i, jf)), Ap[col_e + jf * 4], acc);
+                            }
+                            *reinterpret_cast<float *>(Mhi + tile_off(i, idx[((e >> 2) * NP + i) * 4 + (e & 3)])) = acc;
+                        }
+#pragma unroll 1
+                        for (int e = 0; e <= dp; ++e) {
+                            const int off = tile_off(i, (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)]);
+                            const float val = *reinterpret_cast<const float *>(Mhi + off), hi = ptx::tf32_hi(val);
+                            *reinterpret_cast<float *>(Mhi + off) = hi;
+                            *reinterpret_cast<float *>(Mlo + off) = val - hi;
                         }
                     } else {  // deep paths: the same recurrence through shared memory
                         float *x = xr + (wrow ? i : NP + i) * C::XLD;
@@ -826,7 +898,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         for (int e = 0; e <= dp; ++e) {
                             const int col = (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)];
                             const float val = x[e], hi = ptx::tf32_hi(val);
-                            const int off = i * 128 + (((col >> 2) ^ (i & 7)) << 4) + ((col & 3) << 2);
+                            const int off = tile_off(i, col);
                             *reinterpret_cast<float *>(Mhi + off) = hi;
                             *reinterpret_cast<float *>(Mlo + off) = val - hi;
                         }
@@ -1014,7 +1086,8 @@ cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, c
     if (e != cudaSuccess || a.max_nodes <= 32) return e;
     VerifyArgs large = a;
     large.cls_lo = 32, large.cls_hi = a.max_nodes;
-    return launch_verify_sm100_tc64(large, T, od, stream);
+    return od == TREEWY_F32 ? launch_vt<64, float, false>(large, none, T, stream)
+                            : launch_vt<64, __nv_bfloat16, false>(large, none, T, stream);
 }
 
 // commit of the previous round + verify of this one, one kernel; this round's trees have <= 32 nodes
