@@ -60,7 +60,6 @@ cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, c
 // commit of the previous round fused into verify (trees of up to 32 nodes in the new round)
 cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv, int T, treewy_dtype_t od,
                                        cudaStream_t stream);
-cudaError_t launch_verify_sm100_tc64(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream);
 cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
 cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream);  // bf16 state
 
