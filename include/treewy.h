@@ -102,6 +102,14 @@ treewy_status_t treewy_tree_prepare(const treewy_tree_t *tree, const float *alph
                                     int32_t *seq_status, void *cuda_stream);
 
 /*
+ * The same with the gates given as logarithms, log_alpha [T,H_v] fp32 <= 0, which is how Gated
+ * DeltaNet layers produce them (Eq. 1's alpha_t = exp(g_t)): cum_log_gate is the plain sum of
+ * log_alpha along the root path, no logf is taken.  Everything else as treewy_tree_prepare.
+ */
+treewy_status_t treewy_tree_prepare_log(const treewy_tree_t *tree, const float *log_alpha,
+                                        int32_t *seq_status, void *cuda_stream);
+
+/*
  * Verify (Section 3, Eq. 2 and the read-out "from that same solve").
  *   S0   [B,H_v,128,128]  io_dtype, read only
  *   q,k  [T,H_qk,128]     io_dtype;  v [T,H_v,128] io_dtype;  beta [T,H_v] fp32

@@ -59,6 +59,8 @@ def load_library(path: str | None = None):
     vp, i32 = ctypes.c_void_p, ctypes.c_int32
     lib.treewy_tree_prepare.argtypes = [ctypes.POINTER(TreeStruct), vp, vp, vp]
     lib.treewy_tree_prepare.restype = ctypes.c_int
+    lib.treewy_tree_prepare_log.argtypes = [ctypes.POINTER(TreeStruct), vp, vp, vp]
+    lib.treewy_tree_prepare_log.restype = ctypes.c_int
     verify_args = [vp, vp, vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int,
                    vp, vp, vp, vp]
     lib.treewy_verify.argtypes = verify_args
@@ -142,6 +144,15 @@ def treewy_tree_prepare(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tenso
     ts = tree.struct()
     _check("treewy_tree_prepare",
            lib.treewy_tree_prepare(ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream)))
+
+
+def treewy_tree_prepare_log(tree: Tree, log_alpha: torch.Tensor, seq_status: torch.Tensor | None = None,
+                            stream=None) -> None:
+    """As treewy_tree_prepare, with the gates given as logarithms (log alpha <= 0)."""
+    lib = load_library()
+    ts = tree.struct()
+    _check("treewy_tree_prepare_log",
+           lib.treewy_tree_prepare_log(ctypes.byref(ts), _p(log_alpha), _p(seq_status), _stream(stream)))
 
 
 def treewy_verify(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,

@@ -65,18 +65,30 @@ treewy_status_t verify_common(bool force_generic, const void *S0, const void *q,
 
 extern "C" {
 
-treewy_status_t treewy_tree_prepare(const treewy_tree_t *tree, const float *alpha,
-                                    int32_t *seq_status, void *cuda_stream)
+static treewy_status_t prepare_common(const treewy_tree_t *tree, const float *gates, bool gates_are_logs,
+                                      int32_t *seq_status, void *cuda_stream)
 {
     int max_nodes = 0;
     treewy_status_t st = check_tree(tree, true, &max_nodes);
     if (st != TREEWY_OK) return st;
     if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
     if (tree->B == 0) return TREEWY_OK;
-    if (tree->T > 0 && bad_ptr(alpha)) return TREEWY_ERR_INVALID_ARG;
-    cudaError_t e =
-        launch_prepare(*tree, max_nodes, alpha, seq_status, static_cast<cudaStream_t>(cuda_stream));
+    if (tree->T > 0 && bad_ptr(gates)) return TREEWY_ERR_INVALID_ARG;
+    cudaError_t e = launch_prepare(*tree, max_nodes, gates, gates_are_logs, seq_status,
+                                   static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_tree_prepare(const treewy_tree_t *tree, const float *alpha,
+                                    int32_t *seq_status, void *cuda_stream)
+{
+    return prepare_common(tree, alpha, false, seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_tree_prepare_log(const treewy_tree_t *tree, const float *log_alpha,
+                                        int32_t *seq_status, void *cuda_stream)
+{
+    return prepare_common(tree, log_alpha, true, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_verify(const void *S0, const void *q, const void *k, const void *v,

@@ -17,7 +17,7 @@ constexpr int PREP_THREADS = 128;
 constexpr int PREP_HCHUNK = 16;  // value heads per CTA
 
 __global__ void __launch_bounds__(PREP_THREADS)
-prepare_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_offsets,
+prepare_kernel(int B, int H_v, int max_nodes, int gates_are_logs, const int32_t *__restrict__ node_offsets,
                const int32_t *__restrict__ parent, const float *__restrict__ alpha,
                int32_t *__restrict__ depth, uint64_t *__restrict__ anc_mask,
                float *__restrict__ cum_log_gate, uint8_t *__restrict__ level_order,
@@ -55,7 +55,8 @@ prepare_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_o
         const int hc = min(PREP_HCHUNK, H_v - h0);
         for (int e = threadIdx.x; e < n * hc; e += PREP_THREADS) {
             const int i = e / hc, h = e - i * hc;
-            s_log[i * PREP_HCHUNK + h] = logf(alpha[(size_t)(lo + i) * H_v + h0 + h]);
+            const float gate = alpha[(size_t)(lo + i) * H_v + h0 + h];
+            s_log[i * PREP_HCHUNK + h] = gates_are_logs ? gate : logf(gate);
         }
         __syncthreads();  // log table and the tree walk are complete
         for (int e = threadIdx.x; e < n * hc; e += PREP_THREADS) {
@@ -85,12 +86,12 @@ prepare_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_o
     }
 }
 
-cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha,
+cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha, bool gates_are_logs,
                            int32_t *seq_status, cudaStream_t stream)
 {
     if (t.B == 0) return cudaSuccess;
     const dim3 grid(t.B, (t.H_v + PREP_HCHUNK - 1) / PREP_HCHUNK);
-    prepare_kernel<<<grid, PREP_THREADS, 0, stream>>>(t.B, t.H_v, max_nodes, t.node_offsets,
+    prepare_kernel<<<grid, PREP_THREADS, 0, stream>>>(t.B, t.H_v, max_nodes, gates_are_logs ? 1 : 0, t.node_offsets,
                                                      t.parent, alpha, t.depth, t.anc_mask,
                                                      t.cum_log_gate, t.level_order, seq_status);
     return cudaGetLastError();

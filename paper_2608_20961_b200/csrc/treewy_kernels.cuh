@@ -51,7 +51,7 @@ struct CommitArgs {
     int T;
 };
 
-cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha,
+cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha, bool gates_are_logs,
                            int32_t *seq_status, cudaStream_t stream);
 cudaError_t launch_verify_generic(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od,
                                   cudaStream_t stream);

@@ -188,3 +188,27 @@ def test_malformed_sequences_in_the_tensor_core_solve(oracle):
     np.testing.assert_allclose(gpu["O"][:4].double().numpy(), ref.O, atol=1e-4)
     assert torch.all(gpu["O"][off[1]:off[2]] == gpu["canary"])
     assert torch.all(gpu["U"][off[3]:off[4]] == gpu["canary"])
+
+
+def test_prepare_from_log_gates(oracle):
+    """Gates given as logarithms: the tree outputs are those of the oracle run on exp(log alpha), the
+    cumulative log-gate is the plain sum along the root path, and verify on top of it matches."""
+    from paper_2608_20961_b200 import binding as tw
+    w = wl.make_workload(5, B=4, H_v=4, seed=7)
+    g = torch.log(w.alpha.double()).float()                      # what a GDN layer would hand over
+    w.alpha = torch.exp(g.double()).float()
+    tree_ref = oracle.prepare(w.node_offsets.numpy(), w.parent.numpy(), np.exp(g.double().numpy()))
+    dev = torch.device("cuda:0")
+    tree = tw.Tree.empty(w.node_offsets.to(dev), w.parent.to(dev), w.H_v, w.max_nodes)
+    status = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    tw.treewy_tree_prepare_log(tree, g.to(dev), status)
+    torch.cuda.synchronize()
+    assert not status.any()
+    np.testing.assert_array_equal(tree.depth.cpu().numpy(), tree_ref.depth)
+    np.testing.assert_array_equal(tree.anc_mask.cpu().numpy().view(np.uint64), tree_ref.anc_mask)
+    np.testing.assert_array_equal(tree.level_order.cpu().numpy(), tree_ref.level_order)
+    np.testing.assert_allclose(tree.cum_log_gate.cpu().numpy(), tree_ref.cum_log_gate, rtol=0, atol=1e-5)
+    lin = tw.Tree.empty(w.node_offsets.to(dev), w.parent.to(dev), w.H_v, w.max_nodes)
+    tw.treewy_tree_prepare(lin, w.alpha.to(dev), status)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(tree.cum_log_gate.cpu().numpy(), lin.cum_log_gate.cpu().numpy(), rtol=0, atol=2e-6)
