@@ -64,7 +64,8 @@ enum {
     TREEWY_SEQ_BAD_PARENT = 1,     /* some parent[i] >= i or < -1 */
     TREEWY_SEQ_TOO_MANY_NODES = 2, /* N_b outside 1..max_nodes */
     TREEWY_SEQ_BAD_ACCEPTED = 4,   /* accepted[b] outside -1..N_b-1 */
-    TREEWY_SEQ_TIMEOUT = 8         /* a bounded wait inside a kernel gave up */
+    TREEWY_SEQ_TIMEOUT = 8,        /* a bounded wait inside a kernel gave up */
+    TREEWY_SEQ_BAD_STATE = 16      /* state_index[b] outside 0..n_states-1 (block-pool calls) */
 };
 
 /*
@@ -151,6 +152,28 @@ treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void 
 treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
                               int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
                               float *S_out_f32, int32_t *seq_status, void *cuda_stream);
+
+/*
+ * Block-pool addressing of the states (the paper keeps one state block per sequence and layer in
+ * the serving engine's block pool, Section 4): sequence b's state is
+ * states[state_index[b]], a [H_v,128,128] block of a pool of n_states blocks.  treewy_verify_pool
+ * and treewy_commit_pool are treewy_verify and treewy_commit (without the fp32 copy) on such a
+ * view; an index outside 0..n_states-1 flags TREEWY_SEQ_BAD_STATE and skips the sequence.  Two
+ * sequences of one call must not share a block.
+ */
+typedef struct {
+    void *states;               /* [n_states,H_v,128,128] io_dtype, device */
+    const int32_t *state_index; /* [B] device */
+    int32_t n_states;
+} treewy_state_pool_t;
+
+treewy_status_t treewy_verify_pool(const treewy_state_pool_t *pool, const void *q, const void *k, const void *v,
+                                   const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                                   treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,
+                                   int32_t *seq_status, void *cuda_stream);
+treewy_status_t treewy_commit_pool(const treewy_state_pool_t *pool, const float *U, const void *k,
+                                   const treewy_tree_t *tree, int32_t H_qk, const int32_t *accepted,
+                                   treewy_dtype_t io_dtype, int32_t *seq_status, void *cuda_stream);
 
 /*
  * Commit of the previous round fused into the verify of this round (Section 3, Eq. 3 then Eq. 2;

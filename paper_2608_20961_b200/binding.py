@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libtreewy.so")
 
 TREEWY_OK, TREEWY_ERR_INVALID_ARG, TREEWY_ERR_UNSUPPORTED, TREEWY_ERR_CUDA = 0, 1, 2, 3
 TREEWY_F32, TREEWY_BF16 = 0, 1
-SEQ_BAD_PARENT, SEQ_TOO_MANY_NODES, SEQ_BAD_ACCEPTED, SEQ_TIMEOUT = 1, 2, 4, 8
+SEQ_BAD_PARENT, SEQ_TOO_MANY_NODES, SEQ_BAD_ACCEPTED, SEQ_TIMEOUT, SEQ_BAD_STATE = 1, 2, 4, 8, 16
 D = 128
 MAX_NODES = 64
 
@@ -34,6 +34,11 @@ class TreeStruct(ctypes.Structure):
         ("depth", ctypes.c_void_p), ("anc_mask", ctypes.c_void_p),
         ("cum_log_gate", ctypes.c_void_p), ("level_order", ctypes.c_void_p),
     ]
+
+
+class PoolStruct(ctypes.Structure):
+    """Mirror of ``treewy_state_pool_t``."""
+    _fields_ = [("states", ctypes.c_void_p), ("state_index", ctypes.c_void_p), ("n_states", ctypes.c_int32)]
 
 
 class TreewyError(RuntimeError):
@@ -61,6 +66,12 @@ def load_library(path: str | None = None):
     lib.treewy_tree_prepare.restype = ctypes.c_int
     lib.treewy_tree_prepare_log.argtypes = [ctypes.POINTER(TreeStruct), vp, vp, vp]
     lib.treewy_tree_prepare_log.restype = ctypes.c_int
+    lib.treewy_verify_pool.argtypes = [ctypes.POINTER(PoolStruct), vp, vp, vp, vp, ctypes.POINTER(TreeStruct), i32,
+                                       ctypes.c_int, ctypes.c_int, vp, vp, vp, vp]
+    lib.treewy_verify_pool.restype = ctypes.c_int
+    lib.treewy_commit_pool.argtypes = [ctypes.POINTER(PoolStruct), vp, vp, ctypes.POINTER(TreeStruct), i32, vp,
+                                       ctypes.c_int, vp, vp]
+    lib.treewy_commit_pool.restype = ctypes.c_int
     verify_args = [vp, vp, vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int,
                    vp, vp, vp, vp]
     lib.treewy_verify.argtypes = verify_args
@@ -153,6 +164,31 @@ def treewy_tree_prepare_log(tree: Tree, log_alpha: torch.Tensor, seq_status: tor
     ts = tree.struct()
     _check("treewy_tree_prepare_log",
            lib.treewy_tree_prepare_log(ctypes.byref(ts), _p(log_alpha), _p(seq_status), _stream(stream)))
+
+
+def _pool(states: torch.Tensor, state_index: torch.Tensor) -> PoolStruct:
+    assert state_index.dtype == torch.int32
+    return PoolStruct(states.data_ptr(), state_index.data_ptr(), int(states.shape[0]))
+
+
+def treewy_verify_pool(states, state_index, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor,
+                       U: torch.Tensor, seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_verify with sequence b's state at states[state_index[b]] (block-pool addressing)."""
+    lib = load_library()
+    ts, ps = tree.struct(), _pool(states, state_index)
+    _check("treewy_verify_pool",
+           lib.treewy_verify_pool(ctypes.byref(ps), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), H_qk,
+                                  _DTYPES[states.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream)))
+
+
+def treewy_commit_pool(states, state_index, U, k, tree: Tree, H_qk: int, accepted: torch.Tensor,
+                       seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_commit, in place, with sequence b's state at states[state_index[b]]."""
+    lib = load_library()
+    ts, ps = tree.struct(), _pool(states, state_index)
+    _check("treewy_commit_pool",
+           lib.treewy_commit_pool(ctypes.byref(ps), _p(U), _p(k), ctypes.byref(ts), H_qk, _p(accepted),
+                                  _DTYPES[states.dtype], _p(seq_status), _stream(stream)))
 
 
 def treewy_verify(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,

@@ -28,11 +28,28 @@ treewy_status_t check_tree(const treewy_tree_t *t, bool need_outputs, int *max_n
     return TREEWY_OK;
 }
 
-treewy_status_t verify_common(bool force_generic, const void *S0, const void *q, const void *k,
+// A state view: either the plain [B,H_v,128,128] array of the classic calls (index NULL) or a block pool.
+struct StateView {
+    void *states;
+    const int32_t *index;
+    int n_states;
+};
+inline StateView plain_view(const void *S0, int B) { return {const_cast<void *>(S0), nullptr, B}; }
+treewy_status_t check_pool(const treewy_state_pool_t *pool, StateView *out)
+{
+    if (!pool) return TREEWY_ERR_INVALID_ARG;
+    if (pool->n_states < 0) return TREEWY_ERR_INVALID_ARG;
+    if (pool->n_states > 0 && (bad_ptr(pool->states) || bad_ptr(pool->state_index))) return TREEWY_ERR_INVALID_ARG;
+    *out = {pool->states, pool->state_index, pool->n_states};
+    return TREEWY_OK;
+}
+
+treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, const void *k,
                               const void *v, const float *beta, const treewy_tree_t *tree,
                               int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype,
                               void *O, float *U, int32_t *seq_status, void *cuda_stream)
 {
+    const void *S0 = sv.states;
     int max_nodes = 0;
     treewy_status_t st = check_tree(tree, true, &max_nodes);
     if (st != TREEWY_OK) return st;
@@ -51,6 +68,7 @@ treewy_status_t verify_common(bool force_generic, const void *S0, const void *q,
     a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.state_index = sv.index, a.n_states = sv.n_states;
     a.cls_lo = 0, a.cls_hi = max_nodes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
@@ -96,8 +114,8 @@ treewy_status_t treewy_verify(const void *S0, const void *q, const void *k, cons
                               treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,
                               int32_t *seq_status, void *cuda_stream)
 {
-    return verify_common(false, S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status,
-                         cuda_stream);
+    return verify_common(false, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
+                         U, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void *k, const void *v,
@@ -105,14 +123,15 @@ treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void 
                                       treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
                                       float *U, int32_t *seq_status, void *cuda_stream)
 {
-    return verify_common(true, S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status,
-                         cuda_stream);
+    return verify_common(true, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
+                         U, seq_status, cuda_stream);
 }
 
-treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
-                              int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
-                              float *S_out_f32, int32_t *seq_status, void *cuda_stream)
+static treewy_status_t commit_common(StateView sv, const float *U, const void *k, const treewy_tree_t *tree,
+                                     int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
+                                     float *S_out_f32, int32_t *seq_status, void *cuda_stream)
 {
+    void *S0 = sv.states;
     int max_nodes = 0;
     treewy_status_t st = check_tree(tree, true, &max_nodes);
     if (st != TREEWY_OK) return st;
@@ -131,8 +150,38 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
     a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     a.snap_out = nullptr, a.T = tree->T;
+    a.state_index = sv.index, a.n_states = sv.n_states;
     cudaError_t e = launch_commit(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
+                              int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
+                              float *S_out_f32, int32_t *seq_status, void *cuda_stream)
+{
+    return commit_common(plain_view(S0, tree ? tree->B : 0), U, k, tree, H_qk, accepted, io_dtype, S_out_f32,
+                         seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_verify_pool(const treewy_state_pool_t *pool, const void *q, const void *k, const void *v,
+                                   const float *beta, const treewy_tree_t *tree, int32_t H_qk,
+                                   treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,
+                                   int32_t *seq_status, void *cuda_stream)
+{
+    StateView sv;
+    treewy_status_t st = check_pool(pool, &sv);
+    if (st != TREEWY_OK) return st;
+    return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_commit_pool(const treewy_state_pool_t *pool, const float *U, const void *k,
+                                   const treewy_tree_t *tree, int32_t H_qk, const int32_t *accepted,
+                                   treewy_dtype_t io_dtype, int32_t *seq_status, void *cuda_stream)
+{
+    StateView sv;
+    treewy_status_t st = check_pool(pool, &sv);
+    if (st != TREEWY_OK) return st;
+    return commit_common(sv, U, k, tree, H_qk, accepted, io_dtype, nullptr, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *k, const treewy_tree_t *tree,
@@ -155,6 +204,7 @@ treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *
     a.accepted = nullptr, a.S_out_f32 = nullptr, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     a.snap_out = Snap, a.T = tree->T;
+    a.state_index = nullptr, a.n_states = tree->B;
     cudaError_t e = launch_commit_pipe(a, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
@@ -192,6 +242,7 @@ treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *
     a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.state_index = nullptr, a.n_states = tree->B;
     a.cls_lo = 0, a.cls_hi = max_nodes;
     PrevRound pv;
     pv.U = U_prev, pv.k = k_prev;

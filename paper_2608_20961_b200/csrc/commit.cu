@@ -69,7 +69,8 @@ __global__ void __launch_bounds__(CM_THREADS) commit_kernel(CommitArgs a)
     const int n = a.node_offsets[b + 1] - lo;
     const int acc_node = a.accepted[b];
 
-    T *tile = static_cast<T *>(a.S0) + ((size_t)b * a.H_v + h) * D * D + (size_t)slab * ROWS * D;
+    const int slot = state_slot(a.state_index, a.n_states, b);
+    T *tile = static_cast<T *>(a.S0) + ((size_t)(slot < 0 ? 0 : slot) * a.H_v + h) * D * D + (size_t)slab * ROWS * D;
     float *tile32 =
         a.S_out_f32 ? a.S_out_f32 + ((size_t)b * a.H_v + h) * D * D + (size_t)slab * ROWS * D : nullptr;
 
@@ -77,6 +78,7 @@ __global__ void __launch_bounds__(CM_THREADS) commit_kernel(CommitArgs a)
     __syncthreads();
     int bad = validate_sequence(a.parent, lo, n, a.max_nodes, &s_bad);
     if (!bad && (acc_node < -1 || acc_node >= n)) bad = TREEWY_SEQ_BAD_ACCEPTED;
+    if (slot < 0) bad = TREEWY_SEQ_BAD_STATE;
     if (bad) {
         if (tid == 0 && blockIdx.x == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
         return;

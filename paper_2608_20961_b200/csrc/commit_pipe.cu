@@ -44,6 +44,7 @@ struct __align__(128) CommitStage {
     int plen;                 // path length; -1 = nothing to do for this item
     int store_tile;           // 1: tile goes back to memory (accepted >= 0)
     int b, h;                 // sequence and value head of the item
+    int tile_index;           // its state tile: (state slot) * H_v + h
 };
 
 struct CommitPipeSmem {
@@ -96,8 +97,11 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             const int n = a.node_offsets[b + 1] - lo;
             const int acc = a.snap_out ? item / a.H_v - lo : a.accepted[b];
 
+            const int slot = state_slot(a.state_index, a.n_states, b);
             int bad = 0;
-            if (n < 1 || n > a.max_nodes) {
+            if (slot < 0) {
+                bad = TREEWY_SEQ_BAD_STATE;
+            } else if (n < 1 || n > a.max_nodes) {
                 bad = TREEWY_SEQ_TOO_MANY_NODES;
             } else {
                 int bp = 0;
@@ -133,7 +137,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             if (lane == 0) {
                 g.mask = mask, g.La = La, g.ga = expf(La), g.plen = plen;
                 g.store_tile = (acc >= 0);
-                g.b = b, g.h = h;
+                g.b = b, g.h = h, g.tile_index = (slot < 0 ? 0 : slot) * a.H_v + h;
             }
             __syncwarp();
             if (!work) {
@@ -142,7 +146,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             }
             if (lane == 0) {
                 ptx::mbar_arrive_expect_tx(&sm.full[s], CP_TILE_BYTES + cnt * (D * 2 + D * 4));
-                ptx::bulk_g2s(g.tile, S0 + ((size_t)b * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
+                ptx::bulk_g2s(g.tile, S0 + ((size_t)slot * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
             }
             __syncwarp();
             if (lane < cnt) {
@@ -242,8 +246,9 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         ptx::named_sync(1, CP_CONSUMERS);  // every consumer is done with this stage
         if (tid == 0) {
             if (plen >= 0 && store_tile) {
-                __nv_bfloat16 *dst = a.snap_out ? static_cast<__nv_bfloat16 *>(a.snap_out) : S0;
-                ptx::bulk_s2g(dst + (size_t)item * D * D, g.tile, CP_TILE_BYTES);
+                __nv_bfloat16 *dst = a.snap_out ? static_cast<__nv_bfloat16 *>(a.snap_out) + (size_t)item * D * D
+                                                : S0 + (size_t)g.tile_index * D * D;
+                ptx::bulk_s2g(dst, g.tile, CP_TILE_BYTES);
                 ptx::bulk_commit_group();
                 if (pending >= 0) {
                     ptx::bulk_wait_group_read<1>();  // the previous store has left its stage

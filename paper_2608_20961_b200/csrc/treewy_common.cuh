@@ -61,6 +61,14 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
+// state slot of sequence b (block-pool addressing), or -1 when the index is out of range
+__device__ __forceinline__ int state_slot(const int32_t *state_index, int n_states, int b)
+{
+    if (!state_index) return b;
+    const int s = state_index[b];
+    return (s >= 0 && s < n_states) ? s : -1;
+}
+
 __device__ __forceinline__ int nth_set_bit(unsigned long long m, int p)
 {
 #pragma unroll 1

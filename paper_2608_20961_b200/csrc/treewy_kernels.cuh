@@ -20,6 +20,9 @@ struct VerifyArgs {
     float *U;
     int32_t *seq_status;
     int B, H_v, H_qk, max_nodes;
+    // block-pool addressing: sequence b's state is states[state_index[b]] of n_states (NULL: state b of B)
+    const int32_t *state_index;
+    int n_states;
     // size class of this launch: sequences with cls_lo < N_b <= cls_hi are processed, the others are
     // left to the launch of their class (N_b outside 1..max_nodes is flagged where cls_lo == 0)
     int cls_lo, cls_hi;
@@ -49,6 +52,8 @@ struct CommitArgs {
     int B, H_v, H_qk, max_nodes;
     void *snap_out;  // snapshot mode when not NULL: [T, H_v, 128, 128] states, one per node
     int T;
+    const int32_t *state_index;  // as in VerifyArgs
+    int n_states;
 };
 
 cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha, bool gates_are_logs,

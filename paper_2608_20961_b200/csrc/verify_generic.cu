@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(VG_THREADS) verify_generic_kernel(VerifyArgs a
 
     if (c == 0) s_bad = 0;
     __syncthreads();
-    const int bad = validate_sequence(a.parent, lo, n, nmax, &s_bad);
+    const int slot = state_slot(a.state_index, a.n_states, b);
+    const int bad = slot < 0 ? TREEWY_SEQ_BAD_STATE : validate_sequence(a.parent, lo, n, nmax, &s_bad);
     if (bad) {
         if (c == 0 && h == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
         return;
@@ -77,7 +78,7 @@ __global__ void __launch_bounds__(VG_THREADS) verify_generic_kernel(VerifyArgs a
     // row c of S0[b,h] into registers
     float s[D];
     {
-        const TIn *srow = static_cast<const TIn *>(a.S0) + (((size_t)b * a.H_v + h) * D + c) * D;
+        const TIn *srow = static_cast<const TIn *>(a.S0) + (((size_t)slot * a.H_v + h) * D + c) * D;
         load_row128(srow, s);
     }
     __syncthreads();

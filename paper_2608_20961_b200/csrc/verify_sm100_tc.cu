@@ -242,6 +242,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // dependent chain  node_offsets -> parent / mask / log-gate / beta  never delays a TMA issue.
         struct Pre {
             int item, b, h, lo, n, bad, flag;
+            int srow;  // state tile of the item: (state slot) * H_v + h
             unsigned long long mk[C::NPL];  // lane l owns nodes l, l + 32
             float Lv[C::NPL], bv[C::NPL];
             int deep;  // whether any path has more than 8 ancestors
@@ -253,7 +254,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         auto fetch = [&](int kk) {
             Pre p;
             p.item = item_of(kk);
-            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1;
+            p.b = 0, p.h = 0, p.lo = 0, p.n = 0, p.bad = 0, p.flag = 1, p.srow = 0;
 #pragma unroll
             for (int r = 0; r < C::NPL; ++r) p.mk[r] = 0ull, p.Lv[r] = 0.f, p.bv[r] = 0.f;
             p.deep = 0;
@@ -262,7 +263,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             p.b = p.item / a.H_v, p.h = p.item - p.b * a.H_v;
             p.lo = a.node_offsets[p.b];
             p.n = a.node_offsets[p.b + 1] - p.lo;
-            if (p.n < 1 || p.n > a.max_nodes) {
+            const int slot = state_slot(a.state_index, a.n_states, p.b);
+            p.srow = (slot < 0 ? 0 : slot) * a.H_v + p.h;
+            if (slot < 0) {
+                p.bad = TREEWY_SEQ_BAD_STATE;
+                p.flag = a.cls_lo == 0;
+            } else if (p.n < 1 || p.n > a.max_nodes) {
                 p.bad = TREEWY_SEQ_TOO_MANY_NODES;
                 p.flag = a.cls_lo == 0;
             } else if (p.n <= a.cls_lo || p.n > a.cls_hi || p.n > NP) {
@@ -293,7 +299,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 p.plo = pv.node_offsets[p.b];
                 const int pn = pv.node_offsets[p.b + 1] - p.plo;
                 const int acc = pv.accepted[p.b];
-                if (pn < 1 || pn > pv.max_nodes) {
+                if (slot < 0) {
+                    p.pbad = TREEWY_SEQ_BAD_STATE;  // no state to commit into
+                } else if (pn < 1 || pn > pv.max_nodes) {
                     p.pbad = TREEWY_SEQ_TOO_MANY_NODES;
                 } else {
                     int bp = 0;
@@ -334,7 +342,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const int i = lane + 32 * r;
                 if (i < NP) meta_mask(stage)[i] = p.mk[r], meta_L(stage)[i] = p.Lv[r], meta_beta(stage)[i] = p.bv[r];
             }
-            if (lane == 0) meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep;
+            if (lane == 0)
+                meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep,
+                meta_nlo(stage)[3] = p.srow;
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
@@ -349,8 +359,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (tx != 0) {
                     const int hq = p.h / group;
                     if (need_tile) {
-                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.item * D, &full[s]);
-                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.item * D, &full[s]);
+                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.srow * D, &full[s]);
+                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.srow * D, &full[s]);
                     }
                     if (!p.bad) {
                         ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
@@ -556,8 +566,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if constexpr (FUSED) {
                 // the new state goes back to global memory while verification proceeds from this copy
                 if (!gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
-                    ptx::tma_store_2d(&tmS0, 0, item * D, stage + C::OFF_S0);
-                    ptx::tma_store_2d(&tmS0, 64, item * D, stage + C::OFF_S0 + C::S0_HALF);
+                    const int srow = meta_nlo(stage)[3];
+                    ptx::tma_store_2d(&tmS0, 0, srow * D, stage + C::OFF_S0);
+                    ptx::tma_store_2d(&tmS0, 64, srow * D, stage + C::OFF_S0 + C::S0_HALF);
                     ptx::bulk_commit_group();
                     stored = true;
                 }
@@ -1040,7 +1051,8 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     using C = VtCfg<NP, FUSED>;
     const long long n_items = (long long)a.B * a.H_v;
     VerifyMaps m;
-    if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_items, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
+    const long long n_tiles = a.state_index ? (long long)a.n_states * a.H_v : n_items;
+    if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_tiles, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
