@@ -45,6 +45,8 @@
 // raised, and the CTA still reaches the common exit where tensor memory is freed.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 #include "treewy_common.cuh"
@@ -160,6 +162,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                        const __grid_constant__ CUtensorMap tmV)
 {
     using C = VtCfg<NP, FUSED>;
+    // ancestor masks of this round's trees as the kernel handles them: 32 bits (cheaper) up to 32 nodes
+    using mask_t = typename std::conditional<(NP > 32), unsigned long long, uint32_t>::type;
+    auto m_ffs = [](mask_t m) { return (NP > 32 ? __ffsll((long long)m) : __ffs((int)m)) - 1; };
+    auto m_popc = [](mask_t m) { return NP > 32 ? __popcll(m) : __popc((uint32_t)m); };
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + C::OFF_BAR);
@@ -226,7 +232,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
     // byte offset of element (row, col) of a stage-2 B tile (atoms of 32 columns, 128-byte swizzle)
     auto tile_off = [](int row, int col) {
-        return (col >> 5) * C::ATOM + row * 128 + (((((col & 31) >> 2)) ^ (row & 7)) << 4) + ((col & 3) << 2);
+        return (C::NATOM > 1 ? (col >> 5) * C::ATOM : 0) + row * 128 + (((((col & 31) >> 2)) ^ (row & 7)) << 4) +
+               ((col & 3) << 2);
     };
 
     if (warp >= C::PROD_WARP0) {
@@ -292,7 +299,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 p.mk[r] = on ? a.anc_mask[p.lo + i] : 0ull;
                 p.Lv[r] = on ? a.cum_log_gate[(size_t)(p.lo + i) * a.H_v + p.h] : 0.f;
                 p.bv[r] = on ? a.beta[(size_t)(p.lo + i) * a.H_v + p.h] : 0.f;
-                dp8 |= __popcll(p.mk[r] & ~(1ull << i)) > 8;
+                dp8 |= m_popc((mask_t)p.mk[r] & ~((mask_t)1 << i)) > 8;
             }
             p.deep = __any_sync(0xffffffffu, dp8);
             if constexpr (FUSED) {
@@ -389,12 +396,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
 #pragma unroll
                 for (int r = 0; r < C::NPL; ++r) {
                     const int i = lane + 32 * r;
-                    unsigned long long m = p.mk[r] & ~(1ull << i);
+                    mask_t m = (mask_t)p.mk[r] & ~((mask_t)1 << i);
                     float *ratp = reinterpret_cast<float *>(meta_rat(stage)) + i * 4;
                     unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(stage)) + i * 4;
 #pragma unroll 1
                     for (int d = 0; d < 8; ++d) {
-                        const int j = m ? __ffsll((long long)m) - 1 : 0;
+                        const int j = m ? m_ffs(m) : 0;
                         const float rt = m ? __expf(p.Lv[r] - Lm[j]) : 0.f;
                         if (i < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = rt, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
                         m &= m - 1;
@@ -740,10 +747,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     float *Ap = reinterpret_cast<float *>(dl);
                     float *Pp = reinterpret_cast<float *>(dl + NP * NP * 4);
                     unsigned char *idx = dl + 2 * NP * NP * 4;
-                    unsigned long long m = valid ? meta_mask(stage)[i] & ~(1ull << i) : 0ull;
+                    mask_t m = valid ? (mask_t)meta_mask(stage)[i] & ~((mask_t)1 << i) : (mask_t)0;
 #pragma unroll 1
                     for (int d = 0; m; ++d) {
-                        const int j = __ffsll((long long)m) - 1;
+                        const int j = m_ffs(m);
                         m &= m - 1;
                         const float val = scale * __expf(Li - Lm[j]) * row[j];
                         const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
@@ -823,7 +830,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const float *Pp = reinterpret_cast<const float *>(dl + NP * NP * 4);
                 const unsigned char *idx = dl + 2 * NP * NP * 4;
                 float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
-                const int dp = __popcll(meta_mask(stage)[i]) - 1;  // ancestors of node i
+                const int dp = m_popc((mask_t)meta_mask(stage)[i]) - 1;  // ancestors of node i
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
