@@ -199,6 +199,12 @@ treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *
                                      const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
                                      int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
                                      float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream);
+/* The same on a block pool of states (see treewy_state_pool_t). */
+treewy_status_t treewy_commit_verify_pool(const treewy_state_pool_t *pool, const float *U_prev, const void *k_prev,
+                                     const treewy_tree_t *tree_prev, const int32_t *accepted_prev, const void *q,
+                                     const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
+                                     int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                     float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream);
 
 /*
  * Full-state snapshotting, the scheme the method replaces (Section 2, "Speculative verification:

@@ -84,6 +84,10 @@ def load_library(path: str | None = None):
     lib.treewy_commit_verify.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), vp, vp, vp, vp, vp,
                                          ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.treewy_commit_verify.restype = ctypes.c_int
+    lib.treewy_commit_verify_pool.argtypes = [ctypes.POINTER(PoolStruct), vp, vp, ctypes.POINTER(TreeStruct), vp, vp,
+                                              vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int,
+                                              vp, vp, i32, vp, vp]
+    lib.treewy_commit_verify_pool.restype = ctypes.c_int
     lib.treewy_snapshot_all.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, vp, vp, vp]
     lib.treewy_snapshot_all.restype = ctypes.c_int
     lib.treewy_status_string.argtypes = [ctypes.c_int]
@@ -225,6 +229,19 @@ def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, 
                                     _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
                                     _DTYPES[O.dtype], _p(O), _p(U), int(bool(single_kernel)), _p(seq_status),
                                     _stream(stream)))
+
+
+def treewy_commit_verify_pool(states, state_index, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta,
+                              tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor, single_kernel: bool = False,
+                              seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_commit_verify with sequence b's state at states[state_index[b]]."""
+    lib = load_library()
+    tp, ts, ps = tree_prev.struct(), tree.struct(), _pool(states, state_index)
+    _check("treewy_commit_verify_pool",
+           lib.treewy_commit_verify_pool(ctypes.byref(ps), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev),
+                                         _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+                                         _DTYPES[states.dtype], _DTYPES[O.dtype], _p(O), _p(U),
+                                         int(bool(single_kernel)), _p(seq_status), _stream(stream)))
 
 
 def treewy_snapshot_all(S0, U, k, tree: Tree, H_qk: int, Snap: torch.Tensor,

@@ -209,12 +209,14 @@ treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 
-treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *k_prev,
-                                     const treewy_tree_t *tree_prev, const int32_t *accepted_prev, const void *q,
-                                     const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
-                                     int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
-                                     float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream)
+static treewy_status_t commit_verify_common(StateView sv, const float *U_prev, const void *k_prev,
+                                            const treewy_tree_t *tree_prev, const int32_t *accepted_prev,
+                                            const void *q, const void *k, const void *v, const float *beta,
+                                            const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                            treewy_dtype_t o_dtype, void *O, float *U, int32_t single_kernel,
+                                            int32_t *seq_status, void *cuda_stream)
 {
+    void *S0 = sv.states;
     int max_prev = 0, max_nodes = 0;
     treewy_status_t st = check_tree(tree_prev, true, &max_prev);
     if (st != TREEWY_OK) return st;
@@ -223,10 +225,10 @@ treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *
     if (tree_prev->B != tree->B || tree_prev->H_v != tree->H_v) return TREEWY_ERR_INVALID_ARG;
     const bool fusable = single_kernel != 0 && io_dtype == TREEWY_BF16 && max_nodes <= 32 && tree->B > 0 && tree->T > 0 && tree_prev->T > 0;
     if (!fusable) {  // same result from the two stand-alone kernels
-        st = treewy_commit(S0, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
+        st = commit_common(sv, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
                            cuda_stream);
         if (st != TREEWY_OK) return st;
-        return treewy_verify(S0, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
+        return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
     }
     if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
     if (bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
@@ -242,7 +244,7 @@ treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *
     a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
-    a.state_index = nullptr, a.n_states = tree->B;
+    a.state_index = sv.index, a.n_states = sv.n_states;
     a.cls_lo = 0, a.cls_hi = max_nodes;
     PrevRound pv;
     pv.U = U_prev, pv.k = k_prev;
@@ -251,6 +253,30 @@ treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *
     pv.accepted = accepted_prev, pv.max_nodes = max_prev;
     cudaError_t e = launch_commit_verify_sm100(a, pv, tree->T, o_dtype, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_commit_verify(void *S0, const float *U_prev, const void *k_prev,
+                                     const treewy_tree_t *tree_prev, const int32_t *accepted_prev, const void *q,
+                                     const void *k, const void *v, const float *beta, const treewy_tree_t *tree,
+                                     int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O,
+                                     float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream)
+{
+    return commit_verify_common(plain_view(S0, tree ? tree->B : 0), U_prev, k_prev, tree_prev, accepted_prev, q, k, v,
+                                beta, tree, H_qk, io_dtype, o_dtype, O, U, single_kernel, seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_commit_verify_pool(const treewy_state_pool_t *pool, const float *U_prev, const void *k_prev,
+                                          const treewy_tree_t *tree_prev, const int32_t *accepted_prev,
+                                          const void *q, const void *k, const void *v, const float *beta,
+                                          const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                          treewy_dtype_t o_dtype, void *O, float *U, int32_t single_kernel,
+                                          int32_t *seq_status, void *cuda_stream)
+{
+    StateView sv;
+    treewy_status_t st = check_pool(pool, &sv);
+    if (st != TREEWY_OK) return st;
+    return commit_verify_common(sv, U_prev, k_prev, tree_prev, accepted_prev, q, k, v, beta, tree, H_qk, io_dtype,
+                                o_dtype, O, U, single_kernel, seq_status, cuda_stream);
 }
 
 const char *treewy_status_string(treewy_status_t status)
