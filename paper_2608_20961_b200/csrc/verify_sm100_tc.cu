@@ -129,7 +129,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int OFF_CA_HI = (OFF_EINFO + TBUF * 8 + 127) / 128 * 128;
     static constexpr int OFF_CA_LO = OFF_CA_HI + COPS_TILE, OFF_CB = OFF_CA_LO + COPS_TILE;
     static constexpr int OFF_BAR = FUSED ? OFF_CB + COPS_TILE : OFF_EINFO + TBUF * 8;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 4 * SLOTS + 1) * 8 + 16 + 1024;
+    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the group
     // turns it, in its own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
@@ -179,7 +179,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *v_free = v_ready + C::SLOTS;             // R^T warps -> fetching thread: v rows copied to registers
     uint64_t *lists_ready = v_free + C::SLOTS;         // Gram warps -> solver / R^T warps: lists and scalars written
     uint64_t *lists_free = lists_ready + C::SLOTS;     // solver + R^T warps -> Gram warps: the slot may be rewritten
-    uint64_t *upd_done = lists_free + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
+    uint64_t *scal_ready = lists_free + C::SLOTS;      // Gram warps -> R^T warps: per-node scalars written
+    uint64_t *upd_done = scal_ready + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
     uint64_t *cmma_done = upd_done + C::STAGES;        // fused mode: the commit's rank-P product has finished
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(cmma_done + 1);
     int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
@@ -210,6 +211,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&v_free[g], C::R_THREADS / 32);
             ptx::mbar_init(&lists_ready[g], C::G_THREADS / 32);
             ptx::mbar_init(&lists_free[g], (C::R_THREADS + C::T_THREADS) / 32);
+            ptx::mbar_init(&scal_ready[g], C::G_THREADS / 32);
         }
         for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32);
         ptx::mbar_init(cmma_done, 1);
@@ -722,6 +724,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const float bi = meta_beta(stage)[i];
                 const float scale = kind ? bi : 1.f;
                 const float *row = raw + (kind ? NP + i : i) * C::RLD;
+                // the per-node scalars first: the R^T warps need nothing else from here
+                if (tg < NP && valid) {
+                    const float gi = __expf(Li);
+                    if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
+                    scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
+                }
+                ptx::mbar_arrive_warp(&scal_ready[L]);
                 if (!deep) {
                     // the producer left indices and gate ratios of the first 8 ancestors: four Gram
                     // entries are scaled at a time, no dependent chain
@@ -758,11 +767,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         else Pp[at] = val, idx[at] = (unsigned char)j;
                     }
                 }
-                if (tg < NP && valid) {
-                    const float gi = __expf(Li);
-                    if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
-                    scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
-                }
                 if constexpr (C::BIG) {  // the stash is dead: the B tiles take its place
                     ptx::named_sync(1, C::G_THREADS);
                     for (int q = tg; q < C::TILE_BYTES / 16; q += C::G_THREADS)
@@ -771,8 +775,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 ptx::fence_proxy_async();  // the zero fill is read by the tensor core
             } else {
                 ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
+                ptx::mbar_arrive_warp(&scal_ready[L]);
             }
-            ptx::mbar_arrive_warp(&lists_ready[L]);  // lists, scalars and the zero fill are in place
+            ptx::mbar_arrive_warp(&lists_ready[L]);  // lists and the zero fill are in place
         }
     } else if (warp >= C::T_WARP0 && warp < C::R_WARP0) {
         // ------------------------------------------------------------------ solver warps
@@ -953,9 +958,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;                 // SQ | SK
             const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;            // D2 | -
-            // The Gram warps signal after they have seen stage 1 complete, read the Gram block out and
-            // recorded the item's size: one wait covers all three.
-            if (!ptx::mbar_wait(&lists_ready[L], (kk >> 1) & 1)) break;
+            // The Gram warps signal the scalars after they have seen stage 1 complete, read the Gram block
+            // out and recorded the item's size: one wait covers all of it.
+            if (!ptx::mbar_wait(&scal_ready[L], (kk >> 1) & 1)) break;
             ptx::tc_fence_after_sync();
             const int n = einfo[buf].x;
             ptx::mbar_wait(&v_ready[L], (kk >> 1) & 1);
