@@ -67,9 +67,12 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int TBUF = BIG ? 2 : FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
     static constexpr int RBUF = BIG ? 2 : FUSED ? 2 : 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
     // every phase of an item has its own warps, and every role walks all items in order
-    static constexpr int G_THREADS = BIG ? 128 : 64, T_THREADS = BIG ? 128 : 64, R_THREADS = 128, E_THREADS = 128;
+    // (64 nodes: two R^T groups, each taking half of the columns of every item)
+    static constexpr int R_GROUPS = BIG ? 2 : 1;
+    static constexpr int G_THREADS = BIG ? 128 : 64, T_THREADS = BIG ? 128 : 64, R_THREADS = 128 * R_GROUPS;
+    static constexpr int E_THREADS = 128;
     static constexpr int G_WARP0 = 0, T_WARP0 = G_THREADS / 32, R_WARP0 = T_WARP0 + T_THREADS / 32;
-    static constexpr int E_WARP0 = R_WARP0 + 4;  // Gram (when 4 warps) / R / E: warp % 4 = TMEM lane quarter
+    static constexpr int E_WARP0 = R_WARP0 + R_THREADS / 32;  // Gram (when 4 warps) / R / E: warp % 4 = TMEM lane quarter
     static constexpr int COMMIT_WARP0 = E_WARP0 + 4;
     static constexpr int MMA1_WARP = COMMIT_WARP0 + CGROUP / 32;
     static constexpr int MMA1B_WARP = MMA1_WARP + 1;  // the Gram chain of stage 1 has its own issuing warp
@@ -945,7 +948,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // Thread c = TMEM lane c = row c of d_v.  Row c of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j),
         // goes back to tensor memory as hi / lo (the A operand of stage 2); g_j (S0 q_j) in place and
         // zeros over S0 k_j are what stage 2 accumulates o_j and u_j on.
-        const int t = tid - C::R_WARP0 * 32;
+        const int t = (tid - C::R_WARP0 * 32) & 127;
+        const int c_lo = ((tid - C::R_WARP0 * 32) >> 7) * (NP / C::R_GROUPS), c_hi = c_lo + NP / C::R_GROUPS;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
@@ -966,7 +970,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_wait(&v_ready[L], (kk >> 1) & 1);
             if (n > 0) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < NP; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
+                for (int c0 = c_lo; c0 < c_hi; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
                     uint32_t hi[8], lo[8];
                     if (c0 < n) {
                         uint32_t sk[8], sq[8];
