@@ -721,7 +721,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
                 if (!reuse_gram) ptx::named_sync(1, C::G_THREADS);
                 // the slot's previous lists and scalars must have been read
-                ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
+                if (!ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1)) break;  // (a role has given up)
                 const bool valid = i < n;
                 const float Li = Lm[i];
                 const float bi = meta_beta(stage)[i];
@@ -753,7 +753,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
                 } else if (tg < 2 * NP) {  // full-length lists, in scratch memory
                     if constexpr (C::BIG) {  // one area for both slots: the previous item's solve must be over
-                        if (kk >= 1) ptx::mbar_wait(&lists_free[(kk - 1) & 1], ((kk - 1) >> 1) & 1);
+                        if (kk >= 1 && !ptx::mbar_wait(&lists_free[(kk - 1) & 1], ((kk - 1) >> 1) & 1)) break;
                     }
                     unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;
                     float *Ap = reinterpret_cast<float *>(dl);
@@ -777,7 +777,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
                 ptx::fence_proxy_async();  // the zero fill is read by the tensor core
             } else {
-                ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1);
+                if (!ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1)) break;
                 ptx::mbar_arrive_warp(&scal_ready[L]);
             }
             ptx::mbar_arrive_warp(&lists_ready[L]);  // lists and the zero fill are in place
@@ -967,7 +967,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (!ptx::mbar_wait(&scal_ready[L], (kk >> 1) & 1)) break;
             ptx::tc_fence_after_sync();
             const int n = einfo[buf].x;
-            ptx::mbar_wait(&v_ready[L], (kk >> 1) & 1);
+            if (!ptx::mbar_wait(&v_ready[L], (kk >> 1) & 1)) break;
             if (n > 0) {
 #pragma unroll 1
                 for (int c0 = c_lo; c0 < c_hi; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
