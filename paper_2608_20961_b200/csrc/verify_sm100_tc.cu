@@ -80,7 +80,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
     static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 96 + 32 * STAGES;
     // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
-    // (the v rows arrive later, into the dead S0 tile)
+    // (the v rows go to the slots below, two items ahead)
     static constexpr int QK_HALF = 2 * NP * 128;
     static constexpr int QK_BYTES = 2 * QK_HALF;
     static constexpr int S0_HALF = D * 128;
@@ -118,8 +118,8 @@ template <int NP, bool FUSED> struct VtCfg {
     static_assert(BIG || OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
     static constexpr int DEEP_BYTES = BIG ? 2 * NP * NP * 4 + NP * NP : 0;
     static constexpr int V_BYTES = NP * D * 2;
-    // group-private: path lists of the first 8 ancestors, per-node scalars (double-buffered), and
-    // the v rows [NP][128] bf16 of the group's next item (loaded one item ahead)
+    // a slot (consecutive items alternate between the two): path lists of the first 8 ancestors,
+    // per-node scalars, and the item's v rows [NP][128] bf16
     static constexpr int GP_AP = 0, GP_PP = 2 * NP * 16, GP_SCAL = 4 * NP * 16;
     static constexpr int GP_VS = (GP_SCAL + NP * 16 + 127) / 128 * 128;
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
@@ -134,11 +134,11 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int OFF_BAR = FUSED ? OFF_CB + COPS_TILE : OFF_EINFO + TBUF * 8;
     static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
-    // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the group
-    // turns it, in its own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
-    // epilogue frees it.  A block of the second takes the Gram block D2 from stage 1; the group
-    // reads it out, writes R^T (hi) over it and R^T (lo) behind it, stage 2 takes both as its A
-    // operand, and its completion frees the block (long before the epilogue runs).
+    // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the R^T warps
+    // turn it, in their own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
+    // epilogue frees it.  A block of the second takes the Gram block D2 from stage 1; the Gram warps
+    // read it out, the R^T warps write R^T (hi) over it and R^T (lo) behind it, stage 2 takes both as
+    // its A operand, and its completion frees the block (long before the epilogue runs).
     static constexpr int TM_COLS = 2 * NP;
     static constexpr int TM_DO = 0, TM_DU = NP;
     static constexpr int TM_R0 = TBUF * TM_COLS;  // second ring
