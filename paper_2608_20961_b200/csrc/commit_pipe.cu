@@ -66,7 +66,9 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         }
         ptx::fence_barrier_init();
     }
+    grid_dependency_wait();  // the kernel before this one on the stream has finished: global memory may be read
     __syncthreads();
+    grid_dependency_trigger();
 
     __nv_bfloat16 *S0 = static_cast<__nv_bfloat16 *>(a.S0);
     const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(a.k);
@@ -281,8 +283,7 @@ cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream)
     e = cudaFuncSetAttribute(commit_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const int grid = (int)(n_items < sms ? n_items : sms);
-    commit_pipe_kernel<<<grid, CP_THREADS, smem, stream>>>(a, (int)n_items);
-    return cudaGetLastError();
+    return launch_dependent(commit_pipe_kernel, dim3(grid), dim3(CP_THREADS), smem, stream, a, (int)n_items);
 }
 
 }  // namespace treewy

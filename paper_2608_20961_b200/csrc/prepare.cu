@@ -31,6 +31,8 @@ prepare_kernel(int B, int H_v, int max_nodes, int gates_are_logs, const int32_t 
 
     const int b = blockIdx.x;
     const int h0 = blockIdx.y * PREP_HCHUNK;
+    grid_dependency_wait();
+    grid_dependency_trigger();
     if (b >= B) return;
     const int lo = node_offsets[b];
     const int n = node_offsets[b + 1] - lo;
@@ -91,10 +93,9 @@ cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *a
 {
     if (t.B == 0) return cudaSuccess;
     const dim3 grid(t.B, (t.H_v + PREP_HCHUNK - 1) / PREP_HCHUNK);
-    prepare_kernel<<<grid, PREP_THREADS, 0, stream>>>(t.B, t.H_v, max_nodes, gates_are_logs ? 1 : 0, t.node_offsets,
-                                                     t.parent, alpha, t.depth, t.anc_mask,
-                                                     t.cum_log_gate, t.level_order, seq_status);
-    return cudaGetLastError();
+    return launch_dependent(prepare_kernel, grid, dim3(PREP_THREADS), 0, stream, t.B, t.H_v, max_nodes,
+                            gates_are_logs ? 1 : 0, t.node_offsets, t.parent, alpha, t.depth, t.anc_mask,
+                            t.cum_log_gate, t.level_order, seq_status);
 }
 
 }  // namespace treewy

@@ -13,6 +13,28 @@ namespace treewy {
 constexpr int D = TREEWY_D;
 constexpr int MAXN = TREEWY_MAX_NODES;
 
+// Programmatic dependent launch: every kernel of the library is launched so that it may become
+// resident while the kernel before it on the stream is still running (its launch latency and its
+// prologue then overlap that kernel's tail).  grid_dependency_wait() returns once the preceding
+// kernel has finished and its writes are visible: a kernel calls it before its first access to
+// global memory, whatever the buffer, since the library cannot know what the kernel before it wrote.
+// grid_dependency_trigger() lets the kernel after this one become resident as resources free up.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 

@@ -225,7 +225,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         ptx::tmem_relinquish();
         ptx::tc_fence_before_sync();
     }
+    grid_dependency_wait();  // the kernel before this one on the stream has finished: global memory may be read
     __syncthreads();
+    grid_dependency_trigger();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -1079,9 +1081,8 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     if (e != cudaSuccess) return e;
     const long long units = (a.H_v / a.H_qk) % 2 == 0 ? n_items / 2 : n_items;  // the kernel takes heads in pairs
     const int grid = (int)(units < sms ? units : sms);
-    verify_sm100_tc_kernel<NP, TOut, FUSED><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(a, pv, (int)n_items, m.S0,
-                                                                                         m.Q, m.K, m.V);
-    return cudaGetLastError();
+    return launch_dependent(verify_sm100_tc_kernel<NP, TOut, FUSED>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream,
+                            a, pv, (int)n_items, m.S0, m.Q, m.K, m.V);
 }
 
 template <bool FUSED>
