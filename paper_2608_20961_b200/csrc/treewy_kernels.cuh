@@ -65,6 +65,12 @@ cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, c
 // commit of the previous round fused into verify (trees of up to 32 nodes in the new round)
 cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv, int T, treewy_dtype_t od,
                                        cudaStream_t stream);
+// bf16 inputs, trees of up to SMALL_MAX_NODES nodes (chains of a few drafts above all): one small CTA
+// per (sequence, head), no role pipeline; pv != NULL commits the previous round first (fused mode,
+// previous trees of up to SMALL_MAX_NODES nodes as well)
+constexpr int SMALL_MAX_NODES = 8;
+cudaError_t launch_verify_small(const VerifyArgs &a, const PrevRound *pv, int T, treewy_dtype_t od,
+                                cudaStream_t stream);
 cudaError_t launch_commit(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);
 cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream);  // bf16 state
 

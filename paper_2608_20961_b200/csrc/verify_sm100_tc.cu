@@ -1097,11 +1097,13 @@ cudaError_t launch_small(const VerifyArgs &a, const PrevRound &pv, int T, treewy
 
 }  // namespace
 
-// bf16 inputs.  Sequences of up to 32 nodes take the kernel above, larger ones the 64-node variant;
-// a batch that may hold both (max_nodes > 32) gets one launch per size class.
+// bf16 inputs.  Batches of trees of up to 8 nodes take the small-tree kernel.  Otherwise sequences of
+// up to 32 nodes take the kernel above, larger ones its 64-node instance; a batch that may hold both
+// (max_nodes > 32) gets one launch per size class.
 cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, cudaStream_t stream)
 {
     if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
+    if (a.max_nodes <= SMALL_MAX_NODES) return launch_verify_small(a, nullptr, T, od, stream);
     const PrevRound none = {};
     VerifyArgs small = a;
     small.cls_lo = 0, small.cls_hi = a.max_nodes < 32 ? a.max_nodes : 32;
@@ -1125,6 +1127,7 @@ cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv,
 {
     VerifyArgs small = a;
     small.cls_lo = 0, small.cls_hi = a.max_nodes;
+    if (a.max_nodes <= SMALL_MAX_NODES && pv.max_nodes <= SMALL_MAX_NODES) return launch_verify_small(small, &pv, T, od, stream);
     return launch_small<true>(small, pv, T, od, stream);
 }
 
