@@ -380,7 +380,10 @@ def run_ours(args, rank: int, size: int, local: int):
                    "max_nodes": w.max_nodes, "seed": w.seed,
                    "l2": l2_note,
                    "parallelism": f"replicas x{size}, no collective"},
-        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 3 * args.steps,
+        "clocks": clocks.summary(), "e2e": e2e,
+        # prepare + verify + commit; a bf16 batch whose trees may exceed 32 nodes verifies in two launches
+        # (one per size class)
+        "gpu_launches": (4 if w.io_dtype == torch.bfloat16 and w.max_nodes > 32 else 3) * args.steps,
         "roofline": roofline,
         "step_roofline": {"bytes": pb.total, "tensor_flops": pb.tensor_flops, "roof_ms": roof_ms,
                           "frac": roof_ms / ms_per_step, "peak_source": f"of {which}"},

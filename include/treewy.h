@@ -189,7 +189,10 @@ treewy_status_t treewy_commit_pool(const treewy_state_pool_t *pool, const float 
  * again): it moves 23 % fewer bytes.  Its rank-P update runs on the tensor cores with every fp32
  * factor split into two tf32 parts (2^-22 relative), so a few elements of the stored bf16 state may
  * differ from the two-kernel result by one rounding step; status words and the set of rows written
- * are identical.
+ * are identical.  When both rounds' trees have at most 8 nodes (max_nodes of both trees; the chain of
+ * a few drafts the paper's Section 4 runs in production), a kernel of its own does the round with the
+ * update in fp32 in the stand-alone commit's operation order: the stored state is then bit-identical
+ * to the two-kernel result.
  * tree_prev / tree must describe the same B sequences and H_v heads; U_prev [T_prev,H_v,128] fp32
  * and k_prev [T_prev,H_qk,128] are the previous round's verify output and keys, accepted_prev [B]
  * its accepted nodes (-1 = nothing to commit for that sequence).  U_prev and U must not overlap.
