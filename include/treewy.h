@@ -210,6 +210,27 @@ treewy_status_t treewy_commit_verify_pool(const treewy_state_pool_t *pool, const
                                      float *U, int32_t single_kernel, int32_t *seq_status, void *cuda_stream);
 
 /*
+ * 16-bit pseudo-values (Section 3, "Verifying a draft": the stored pseudo-value matrix is what makes
+ * the method's footprint 128 times smaller per node than a state; that ratio holds for U in a 16-bit
+ * type beside a 16-bit state).  treewy_verify_half_u is treewy_verify with U written as IEEE fp16
+ * [T,H_v,128]: every u is formed in fp32 exactly as in treewy_verify and rounded once (RNE) on the
+ * store; O is computed from the unrounded values and is bit-identical to treewy_verify's.
+ * treewy_commit_half_u is treewy_commit reading such a U (widened to fp32, fp32 accumulation, one
+ * rounding of the state): the committed state differs from the fp32-U result by the rounding of U,
+ * at most 2.3e-3 of the state's rms in any element and 2.2e-4 in relative Frobenius norm on the
+ * benchmark workloads (fp16 keeps 11 significant bits; a bf16 U would alone break the parity gate of
+ * the state).  Arguments, layouts, status bits and error behaviour are those of
+ * treewy_verify / treewy_commit; U16 must be 16-byte aligned.  The fused and pool calls take fp32 U.
+ */
+treewy_status_t treewy_verify_half_u(const void *S0, const void *q, const void *k, const void *v, const float *beta,
+                                     const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                     treewy_dtype_t o_dtype, void *O, void *U16, int32_t *seq_status,
+                                     void *cuda_stream);
+treewy_status_t treewy_commit_half_u(void *S0, const void *U16, const void *k, const treewy_tree_t *tree,
+                                     int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
+                                     float *S_out_f32, int32_t *seq_status, void *cuda_stream);
+
+/*
  * Full-state snapshotting, the scheme the method replaces (Section 2, "Speculative verification:
  * where GDN blows up" and "Existing approaches" (i)): materialise the state of EVERY draft node,
  *   Snap[t,h] = g_t S0[b,h] + sum_{j ancestor-or-self of t} (g_t/g_j) u_j k_j^T      (Eq. 3 with a = t)

@@ -81,6 +81,10 @@ def load_library(path: str | None = None):
     lib.treewy_commit.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, vp, ctypes.c_int,
                                   vp, vp, vp]
     lib.treewy_commit.restype = ctypes.c_int
+    lib.treewy_verify_half_u.argtypes = verify_args
+    lib.treewy_verify_half_u.restype = ctypes.c_int
+    lib.treewy_commit_half_u.argtypes = lib.treewy_commit.argtypes
+    lib.treewy_commit_half_u.restype = ctypes.c_int
     lib.treewy_commit_verify.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), vp, vp, vp, vp, vp,
                                          ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.treewy_commit_verify.restype = ctypes.c_int
@@ -215,6 +219,29 @@ def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Te
     _check("treewy_commit",
            lib.treewy_commit(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
                              _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+
+
+def treewy_verify_half_u(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U16: torch.Tensor,
+                         seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_verify with the pseudo-values written as fp16."""
+    lib = load_library()
+    ts = tree.struct()
+    assert U16.dtype == torch.float16 and q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
+    _check("treewy_verify_half_u",
+           lib.treewy_verify_half_u(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+                                    _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U16), _p(seq_status),
+                                    _stream(stream)))
+
+
+def treewy_commit_half_u(S0, U16, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
+                         seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_commit reading fp16 pseudo-values."""
+    lib = load_library()
+    ts = tree.struct()
+    assert U16.dtype == torch.float16
+    _check("treewy_commit_half_u",
+           lib.treewy_commit_half_u(_p(S0), _p(U16), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                                    _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
 
 
 def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta, tree: Tree,

@@ -47,7 +47,7 @@ treewy_status_t check_pool(const treewy_state_pool_t *pool, StateView *out)
 treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, const void *k,
                               const void *v, const float *beta, const treewy_tree_t *tree,
                               int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype,
-                              void *O, float *U, int32_t *seq_status, void *cuda_stream)
+                              void *O, void *U, bool u_half, int32_t *seq_status, void *cuda_stream)
 {
     const void *S0 = sv.states;
     int max_nodes = 0;
@@ -66,7 +66,7 @@ treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, c
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.depth = tree->depth, a.level_order = tree->level_order;
-    a.O = O, a.U = U, a.seq_status = seq_status;
+    a.O = O, a.U = U, a.u_half = u_half ? 1 : 0, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     a.state_index = sv.index, a.n_states = sv.n_states;
     a.cls_lo = 0, a.cls_hi = max_nodes;
@@ -115,7 +115,7 @@ treewy_status_t treewy_verify(const void *S0, const void *q, const void *k, cons
                               int32_t *seq_status, void *cuda_stream)
 {
     return verify_common(false, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
-                         U, seq_status, cuda_stream);
+                         U, false, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void *k, const void *v,
@@ -124,10 +124,10 @@ treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void 
                                       float *U, int32_t *seq_status, void *cuda_stream)
 {
     return verify_common(true, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
-                         U, seq_status, cuda_stream);
+                         U, false, seq_status, cuda_stream);
 }
 
-static treewy_status_t commit_common(StateView sv, const float *U, const void *k, const treewy_tree_t *tree,
+static treewy_status_t commit_common(StateView sv, const void *U, bool u_half, const void *k, const treewy_tree_t *tree,
                                      int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
                                      float *S_out_f32, int32_t *seq_status, void *cuda_stream)
 {
@@ -144,7 +144,7 @@ static treewy_status_t commit_common(StateView sv, const float *U, const void *k
     if (tree->T > 0 && (bad_ptr(U) || bad_ptr(k))) return TREEWY_ERR_INVALID_ARG;
 
     CommitArgs a;
-    a.S0 = S0, a.U = U, a.k = k;
+    a.S0 = S0, a.U = U, a.u_half = u_half ? 1 : 0, a.k = k;
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
@@ -159,7 +159,23 @@ treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const tre
                               int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
                               float *S_out_f32, int32_t *seq_status, void *cuda_stream)
 {
-    return commit_common(plain_view(S0, tree ? tree->B : 0), U, k, tree, H_qk, accepted, io_dtype, S_out_f32,
+    return commit_common(plain_view(S0, tree ? tree->B : 0), U, false, k, tree, H_qk, accepted, io_dtype, S_out_f32,
+                         seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_verify_half_u(const void *S0, const void *q, const void *k, const void *v, const float *beta,
+                                  const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                  treewy_dtype_t o_dtype, void *O, void *U16, int32_t *seq_status, void *cuda_stream)
+{
+    return verify_common(false, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
+                         U16, true, seq_status, cuda_stream);
+}
+
+treewy_status_t treewy_commit_half_u(void *S0, const void *U16, const void *k, const treewy_tree_t *tree, int32_t H_qk,
+                                  const int32_t *accepted, treewy_dtype_t io_dtype, float *S_out_f32,
+                                  int32_t *seq_status, void *cuda_stream)
+{
+    return commit_common(plain_view(S0, tree ? tree->B : 0), U16, true, k, tree, H_qk, accepted, io_dtype, S_out_f32,
                          seq_status, cuda_stream);
 }
 
@@ -171,7 +187,7 @@ treewy_status_t treewy_verify_pool(const treewy_state_pool_t *pool, const void *
     StateView sv;
     treewy_status_t st = check_pool(pool, &sv);
     if (st != TREEWY_OK) return st;
-    return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
+    return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, false, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_commit_pool(const treewy_state_pool_t *pool, const float *U, const void *k,
@@ -181,7 +197,7 @@ treewy_status_t treewy_commit_pool(const treewy_state_pool_t *pool, const float 
     StateView sv;
     treewy_status_t st = check_pool(pool, &sv);
     if (st != TREEWY_OK) return st;
-    return commit_common(sv, U, k, tree, H_qk, accepted, io_dtype, nullptr, seq_status, cuda_stream);
+    return commit_common(sv, U, false, k, tree, H_qk, accepted, io_dtype, nullptr, seq_status, cuda_stream);
 }
 
 treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *k, const treewy_tree_t *tree,
@@ -198,7 +214,7 @@ treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *
     if (bad_ptr(S0) || bad_ptr(U) || bad_ptr(k) || bad_ptr(Snap)) return TREEWY_ERR_INVALID_ARG;
 
     CommitArgs a;
-    a.S0 = const_cast<void *>(S0), a.U = U, a.k = k;
+    a.S0 = const_cast<void *>(S0), a.U = U, a.u_half = 0, a.k = k;
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.accepted = nullptr, a.S_out_f32 = nullptr, a.seq_status = seq_status;
@@ -225,10 +241,10 @@ static treewy_status_t commit_verify_common(StateView sv, const float *U_prev, c
     if (tree_prev->B != tree->B || tree_prev->H_v != tree->H_v) return TREEWY_ERR_INVALID_ARG;
     const bool fusable = single_kernel != 0 && io_dtype == TREEWY_BF16 && max_nodes <= 32 && tree->B > 0 && tree->T > 0 && tree_prev->T > 0;
     if (!fusable) {  // same result from the two stand-alone kernels
-        st = commit_common(sv, U_prev, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
+        st = commit_common(sv, U_prev, false, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
                            cuda_stream);
         if (st != TREEWY_OK) return st;
-        return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, seq_status, cuda_stream);
+        return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, false, seq_status, cuda_stream);
     }
     if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
     if (bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
@@ -242,7 +258,7 @@ static treewy_status_t commit_verify_common(StateView sv, const float *U_prev, c
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.depth = tree->depth, a.level_order = tree->level_order;
-    a.O = O, a.U = U, a.seq_status = seq_status;
+    a.O = O, a.U = U, a.u_half = 0, a.seq_status = seq_status;
     a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
     a.state_index = sv.index, a.n_states = sv.n_states;
     a.cls_lo = 0, a.cls_hi = max_nodes;

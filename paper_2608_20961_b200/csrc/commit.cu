@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(CM_THREADS) commit_kernel(CommitArgs a)
             if (tid < D)
                 kw[cnt][tid] = w * to_f32(kg[((size_t)(lo + j) * a.H_qk + hq) * D + tid]);
             else if (tid - D < ROWS)
-                uu[cnt][tid - D] = a.U[((size_t)(lo + j) * a.H_v + h) * D + slab * ROWS + tid - D];
+                uu[cnt][tid - D] = load_u(a.U, ((size_t)(lo + j) * a.H_v + h) * D + slab * ROWS + tid - D, a.u_half);
         }
         rest = m;
         __syncthreads();

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
     grid_dependency_trigger();
 
     __nv_bfloat16 *S0 = static_cast<__nv_bfloat16 *>(a.S0);
+    const uint32_t ub = a.u_half ? 2u : 4u;  // bytes of a U element
     const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(a.k);
     const int group = a.H_v / a.H_qk;
 
@@ -147,14 +148,14 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 continue;
             }
             if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(&sm.full[s], CP_TILE_BYTES + cnt * (D * 2 + D * 4));
+                ptx::mbar_arrive_expect_tx(&sm.full[s], CP_TILE_BYTES + cnt * (D * 2 + D * ub));
                 ptx::bulk_g2s(g.tile, S0 + ((size_t)slot * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
             }
             __syncwarp();
             if (lane < cnt) {
                 ptx::bulk_g2s(g.krow[lane], kg + ((size_t)(lo + j) * a.H_qk + h / group) * D, D * 2,
                               &sm.full[s]);
-                ptx::bulk_g2s(g.urow[lane], a.U + ((size_t)(lo + j) * a.H_v + h) * D, D * 4,
+                ptx::bulk_g2s(g.urow[lane], static_cast<const char *>(a.U) + ((size_t)(lo + j) * a.H_v + h) * D * ub, D * ub,
                               &sm.full[s]);
             }
         }
@@ -197,7 +198,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 for (int e = 0; e < 8; ++e) kf[e] *= w;
 #pragma unroll
                 for (int it = 0; it < 8; ++it) {
-                    const float u = g.urow[p][r0 + 16 * it];
+                    const float u = a.u_half ? __half2float(reinterpret_cast<const __half *>(g.urow[p])[r0 + 16 * it])
+                                             : g.urow[p][r0 + 16 * it];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
                 }
@@ -216,10 +218,10 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                            kf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) kf[e] *= w;
-                    const float *ur = a.U + ((size_t)(lo + j) * a.H_v + h) * D;
+                    const size_t ur = ((size_t)(lo + j) * a.H_v + h) * D;
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
-                        const float u = ur[r0 + 16 * it];
+                        const float u = load_u(a.U, ur + r0 + 16 * it, a.u_half);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc[it][e] = fmaf(u, kf[e], acc[it][e]);
                     }

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -43,6 +44,17 @@ template <> __device__ __forceinline__ float from_f32<float>(float x) { return x
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x)
 {
     return __float2bfloat16_rn(x);
+}
+
+// Element idx of a pseudo-value array U, which the caller keeps in fp32 or (u_half) in fp16.
+__device__ __forceinline__ float load_u(const void *U, size_t idx, int u_half)
+{
+    return u_half ? __half2float(static_cast<const __half *>(U)[idx]) : static_cast<const float *>(U)[idx];
+}
+__device__ __forceinline__ void store_u(void *U, size_t idx, float x, int u_half)
+{
+    if (u_half) static_cast<__half *>(U)[idx] = __float2half_rn(x);
+    else static_cast<float *>(U)[idx] = x;
 }
 
 // Two packed bf16 (low = first element) -> two floats.  bf16 -> fp32 is a 16-bit shift.
@@ -113,6 +125,13 @@ __device__ __forceinline__ void st_global_if(float *p, float v, bool on)
 __device__ __forceinline__ void st_global_if(__nv_bfloat16 *p, float v, bool on)
 {
     const unsigned short b = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.b16 [%0], %1;\n\t}" ::"l"(p), "h"(b),
+                 "r"((int)on));
+}
+
+__device__ __forceinline__ void st_global_if(__half *p, float v, bool on)
+{
+    const unsigned short b = __half_as_ushort(__float2half_rn(v));
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t@q st.global.b16 [%0], %1;\n\t}" ::"l"(p), "h"(b),
                  "r"((int)on));
 }

@@ -17,7 +17,8 @@ struct VerifyArgs {
     const int32_t *depth;
     const uint8_t *level_order;
     void *O;
-    float *U;
+    void *U;     // fp32, or fp16 when u_half
+    int u_half;
     int32_t *seq_status;
     int B, H_v, H_qk, max_nodes;
     // block-pool addressing: sequence b's state is states[state_index[b]] of n_states (NULL: state b of B)
@@ -41,7 +42,8 @@ struct PrevRound {
 
 struct CommitArgs {
     void *S0;
-    const float *U;
+    const void *U;  // fp32, or fp16 when u_half
+    int u_half;
     const void *k;
     const int32_t *node_offsets, *parent;
     const uint64_t *anc_mask;

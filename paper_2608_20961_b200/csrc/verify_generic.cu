@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(VG_THREADS) verify_generic_kernel(VerifyArgs a
         }
         o = fmaf(Ps[i * nmax + i], u, o);
         us[i * D + c] = u;  // read back only by this thread: no barrier needed
-        a.U[orow] = u;
+        store_u(a.U, orow, u, a.u_half);
         Og[orow] = from_f32<TOut>(o);
     }
 }

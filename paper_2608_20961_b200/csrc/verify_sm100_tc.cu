@@ -1030,8 +1030,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int2 info = einfo[buf];
             const int n = info.x, lo = info.y;
             if (n > 0) {
-                float *Ub = a.U + ((size_t)lo * a.H_v + h) * D + t;
-                TOut *Ob = Og + ((size_t)lo * a.H_v + h) * D + t;
+                const size_t row0 = ((size_t)lo * a.H_v + h) * D + t;
+                float *Ub = static_cast<float *>(a.U) + row0;
+                __half *Uh = static_cast<__half *>(a.U) + row0;  // (the caller keeps U in fp16)
+                TOut *Ob = Og + row0;
 #pragma unroll 1
                 for (int c0 = 0; c0 < n; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
                     uint32_t du[8], dout[8];
@@ -1039,12 +1041,17 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     ptx::tmem_ld8(tm + C::TM_DO + c0, dout);
                     ptx::tmem_wait_ld();
                     float *Uc = Ub + (size_t)c0 * rs;
+                    __half *Uhc = Uh + (size_t)c0 * rs;
                     TOut *Oc = Ob + (size_t)c0 * rs;
+                    if (a.u_half) {
 #pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) {
-                        st_global_if(Uc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
-                        st_global_if(Oc + jj * rs, __uint_as_float(dout[jj]), c0 + jj < n);
+                        for (int jj = 0; jj < 8; ++jj) st_global_if(Uhc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) st_global_if(Uc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
                     }
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) st_global_if(Oc + jj * rs, __uint_as_float(dout[jj]), c0 + jj < n);
                 }
             }
             ptx::tc_fence_before_sync();

@@ -433,7 +433,7 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                 }
                 ptx::tc_fence_before_sync();
                 float u[VS_N];
-                float *Ug = a.U + ((size_t)lo * a.H_v + h) * D + t;
+                const size_t urow = ((size_t)lo * a.H_v + h) * D + t;
                 TOut *Og = static_cast<TOut *>(a.O) + ((size_t)lo * a.H_v + h) * D + t;
                 const size_t rs = (size_t)a.H_v * D;
 #pragma unroll
@@ -447,7 +447,7 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                         u[j] = x;
 #pragma unroll
                         for (int i = 0; i <= j; ++i) o = fmaf(Pm[j * VS_N + i], u[i], o);
-                        Ug[j * rs] = x;
+                        store_u(a.U, urow + j * rs, x, a.u_half);
                         store_out(Og + j * rs, o);
                     }
                 }
