@@ -7,28 +7,31 @@
 // phases of one item are too short to be worth a warp role each (the kernel for larger trees hands
 // an item from role to role seven times).  Here an item stays with ONE group of 128 threads from its
 // first byte to its last, three groups per CTA work on three consecutive items side by side, and
-// producer warps (one per stage of a five-stage ring) keep the tiles coming two items ahead.
+// producer warps (one per stage of a four-stage ring) keep the tiles coming.
 //
-//   producer warp of stage s: validates the item, writes its scalars into the stage, and issues the
-//     copies: state tile and q / k rows by TMA (64-column halves, 128-byte swizzle) and -- fused
-//     mode -- the accepted path's k and u rows of the previous round by bulk copy;
+//   producer warp of stage s: validates the item, writes its scalars into the stage's meta block, and
+//     issues the copies: state tile, q / k rows (64-column halves, 128-byte swizzle) and v rows by
+//     TMA and -- fused mode -- the accepted path's k and u rows of the previous round by bulk copy;
 //   group, per item:
 //   * fused mode applies Eq. 3 to the tile in shared memory,
 //     S[r][c] = g_a S[r][c] + sum_p u_p[r] (w_p k_p[c]), in the operation order of the commit
 //     kernels (the stored state is bit-identical to theirs), rounds it to bf16 in place and sends
 //     it back with a TMA store;
-//   * S0 [Q;K]^T is ONE accumulation chain of eight tcgen05.mma (M = 128 state rows, N = 16 = 8 q
-//     rows + 8 k rows, K = 16 each) from the two tiles as they lie in shared memory; the 128 x 16
-//     result sits in tensor memory with lane r = row r of the state, so thread r reads its S0 q_j
-//     and S0 k_j with one tcgen05.ld and owns element r of every r_j, u_j, o_j from there on;
-//   * while the tensor core works, the 128 threads take the 2 x 8 x 8 Gram dot products k_j.k_i,
-//     q_j.k_i and turn them into A and P (Eq. 2); then every thread solves its own column of
-//     (I + A) U = R by forward substitution in registers and reads out o_j.
+//   * S0 [Q;K]^T (M = 128 state rows, N = 16 = 8 q rows + 8 k rows, K = 128) and the Gram block
+//     [Q;K] [Q;K]^T are sixteen tcgen05.mma from the tiles as they lie in shared memory, issued by
+//     four threads into four accumulators each; the stage goes back to its producer as soon as the
+//     tensor core has read it;
+//   * sixteen lanes turn the Gram rows into A and P (Eq. 2); the 128 x 16 state product sits in
+//     tensor memory with lane r = row r of the state, so thread r reads its S0 q_j and S0 k_j with
+//     tcgen05.ld, solves its own column of (I + A) U = R by forward substitution in registers and
+//     reads out o_j.
 //
-// (Two earlier shapes, for the record.  S0 products with fp32 FMAs, thread r against row r: bound by
+// (Earlier shapes, for the record.  S0 products with fp32 FMAs, thread r against row r: bound by
 // the 128 bytes per clock that shared memory delivers to registers -- every thread re-reads every
 // q / k vector -- at 2.8 us per tile and SM.  One CTA per item, four resident per SM: a chain of
-// dependent latencies of 6 us per item that four CTAs do not hide.)
+// dependent latencies of 6 us per item that four CTAs do not hide.  Gram dot products on CUDA cores:
+// 25 of 128 lanes busy for 2 k cycles, behind the MMA issue in the issuing warp.  Five stages and
+// 544 threads: 96 registers per thread and the Eq. 3 pass spilled.)
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 #include "treewy_common.cuh"
@@ -41,7 +44,7 @@ namespace {
 constexpr int VS_N = SMALL_MAX_NODES;
 constexpr int VS_HALF = D * 128;            // bytes of one 64-column half of the state tile
 constexpr int VS_QK_HALF = 2 * VS_N * 128;  // ... of the [Q;K] tile: 8 q rows, then 8 k rows
-constexpr uint32_t VS_TMEM_COLS = 512;      // per group: four accumulators of 16 columns for S0 [Q;K]^T, four for the Gram block
+constexpr uint32_t VS_TMEM_COLS = 512;      // per group 128: four accumulators of 16 columns for S0 [Q;K]^T, four for the Gram block
 static_assert(VS_N == 8, "the thread maps below are written for 8 nodes");
 
 // what a stage says about its item (written by the producer warp)
@@ -71,7 +74,7 @@ template <bool FUSED> struct VsCfg {
     static constexpr int STAGE_BYTES = (OFF_UP + (FUSED ? VS_N * D * 4 : 0) + 1023) / 1024 * 1024;
     static constexpr int OFF_META = STAGES * STAGE_BYTES;  // per stage: what the producer says about the item
     static constexpr int META_BYTES = ((int)sizeof(VsMeta) + 15) / 16 * 16;
-    static constexpr int OFF_GRP = OFF_META + STAGES * META_BYTES;  // per group: A and P, 8 x 8 floats each
+    static constexpr int OFF_GRP = OFF_META + STAGES * META_BYTES;  // per group: what the read-out needs
     static constexpr int GRP_BYTES = (2 * VS_N * VS_N + 3 * VS_N) * 4;  // A, P, g_j, beta_j g_j, beta_j
     static constexpr int OFF_BAR = OFF_GRP + GROUPS * GRP_BYTES;
     static constexpr int SMEM_BYTES = OFF_BAR + (2 * STAGES + GROUPS) * 8 + 16 + 1024;
