@@ -148,3 +148,15 @@ def test_small_kernel_on_a_state_pool():
     assert not st.any() and list(stp) == [0] * 7 + [tw.SEQ_BAD_STATE]
     assert torch.equal(O[:off[7]], Op[:off[7]]) and torch.equal(U[:off[7]], Up[:off[7]])
     assert torch.all(Up[off[7]:] == 3.0)
+
+
+def test_fused_small_round_at_the_chain_workloads_full_size():
+    """The chain configuration as the benchmark runs it (64 sequences x 32 heads, hint 5): the fused
+    round stores the same bits as commit followed by verify."""
+    w1 = wl.make_workload(1, seed=81)
+    w2 = wl.make_workload(1, seed=82)
+    two = _two_rounds(w1, w2, False, 5, 5)
+    one = _two_rounds(w1, w2, True, 5, 5)
+    for x, y, name in zip(two, one, ("S", "O", "U", "status")):
+        assert torch.equal(x, y), name
+    assert not one[3].any()
