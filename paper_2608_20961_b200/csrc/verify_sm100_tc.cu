@@ -132,7 +132,11 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int OFF_CA_HI = (OFF_EINFO + TBUF * 8 + 127) / 128 * 128;
     static constexpr int OFF_CA_LO = OFF_CA_HI + COPS_TILE, OFF_CB = OFF_CA_LO + COPS_TILE;
     static constexpr int OFF_BAR = FUSED ? OFF_CB + COPS_TILE : OFF_EINFO + TBUF * 8;
-    static constexpr int SMEM_BYTES = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16 + 1024;
+    // work list of a launch that takes one size class of a mixed batch: the CTA's units of that class
+    // (up to CT_CAP of them; a longer list is walked whole), then 32 warp counts
+    static constexpr int CT_CAP = 1024;
+    static constexpr int OFF_CTAB = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16;
+    static constexpr int SMEM_BYTES = OFF_CTAB + CT_CAP * 2 + 32 * 4 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the R^T warps
     // turn it, in their own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
@@ -158,7 +162,10 @@ struct PathMeta {
 };
 static_assert(sizeof(PathMeta) <= 128, "path meta block");
 
-template <int NP, typename TOut, bool FUSED>
+// (CLASS: the launch takes one size class of a mixed batch and walks a compacted work list; TU: the
+// type U is stored in, float or __half.  Both are template parameters because the code they add
+// costs the other launches instruction-cache hits: 2 % of the headline kernel's time for either.)
+template <int NP, typename TOut, bool FUSED, bool CLASS, typename TU>
 __global__ void __launch_bounds__(VtCfg<NP, FUSED>::THREADS, 1)
 verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_constant__ CUtensorMap tmS0,
                        const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -193,8 +200,22 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     // share a q/k head, a CTA takes the heads two by two: both items of a pair have the same tree
     // and the same [Q;K] rows, so the second reuses the first one's Gram entries.
     const bool pair_mode = ((a.H_v / a.H_qk) & 1) == 0;
+    // The CTA's units (items, or pairs of them) are blockIdx.x, blockIdx.x + gridDim.x, ...: K of them.
+    // A launch that takes one size class of a mixed batch walks only the units of its class (ctab).
+    const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
+    int K = ((pair_mode ? n_items / 2 : n_items) - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const bool compact = CLASS && K <= C::CT_CAP;
     auto item_of = [&](int kk) {
-        return pair_mode ? 2 * ((int)blockIdx.x + (kk >> 1) * (int)gridDim.x) + (kk & 1) : (int)blockIdx.x + kk * (int)gridDim.x;
+        if constexpr (CLASS) {
+            int ku = pair_mode ? kk >> 1 : kk;
+            if (ku >= K) return n_items;
+            if (compact) ku = ctab[ku];
+            const int unit = (int)blockIdx.x + ku * (int)gridDim.x;
+            return pair_mode ? 2 * unit + (kk & 1) : unit;
+        } else {
+            return pair_mode ? 2 * ((int)blockIdx.x + (kk >> 1) * (int)gridDim.x) + (kk & 1)
+                             : (int)blockIdx.x + kk * (int)gridDim.x;
+        }
     };
 
     if (tid == 0) {
@@ -230,6 +251,39 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     grid_dependency_trigger();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (CLASS && compact) {
+        // Every role would otherwise hand every unit of the other classes through the whole pipeline
+        // just to drop it (a third of the time of a ragged batch).  All threads: one unit each per
+        // round, kept units numbered by warp ballots and a prefix over the warps' counts.
+        uint16_t *tab = reinterpret_cast<uint16_t *>(smem + C::OFF_CTAB);
+        int *wcount = reinterpret_cast<int *>(smem + C::OFF_CTAB + C::CT_CAP * 2);
+        const int K_all = K;
+        int kept = 0;
+        for (int base = 0; base < K_all; base += C::THREADS) {
+            const int ku = base + tid;
+            bool keep = false;
+            if (ku < K_all) {
+                const int unit = (int)blockIdx.x + ku * (int)gridDim.x;
+                const int b = (pair_mode ? 2 * unit : unit) / a.H_v;
+                const int n = a.node_offsets[b + 1] - a.node_offsets[b];
+                // another class's well-formed sequence goes; whatever has to be flagged stays
+                keep = !(n >= 1 && n <= a.max_nodes && (n <= a.cls_lo || n > a.cls_hi || n > NP)) ||
+                       (a.cls_lo == 0 && state_slot(a.state_index, a.n_states, b) < 0);
+            }
+            const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) wcount[warp] = __popc(bal);
+            __syncthreads();
+            int before = 0, total = 0;
+            for (int w2 = 0; w2 < C::THREADS / 32; ++w2) {
+                const int c = wcount[w2];
+                before += w2 < warp ? c : 0, total += c;
+            }
+            if (keep) tab[kept + before + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)ku;
+            kept += total;
+            __syncthreads();
+        }
+        K = kept;
+    }
 
     auto meta_mask = [&](unsigned char *stage) { return reinterpret_cast<unsigned long long *>(stage + C::OFF_META); };
     auto meta_L = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 8); };
@@ -1031,8 +1085,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int n = info.x, lo = info.y;
             if (n > 0) {
                 const size_t row0 = ((size_t)lo * a.H_v + h) * D + t;
-                float *Ub = static_cast<float *>(a.U) + row0;
-                __half *Uh = static_cast<__half *>(a.U) + row0;  // (the caller keeps U in fp16)
+                TU *Ub = static_cast<TU *>(a.U) + row0;
                 TOut *Ob = Og + row0;
 #pragma unroll 1
                 for (int c0 = 0; c0 < n; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
@@ -1040,18 +1093,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     ptx::tmem_ld8(tm + C::TM_DU + c0, du);
                     ptx::tmem_ld8(tm + C::TM_DO + c0, dout);
                     ptx::tmem_wait_ld();
-                    float *Uc = Ub + (size_t)c0 * rs;
-                    __half *Uhc = Uh + (size_t)c0 * rs;
+                    TU *Uc = Ub + (size_t)c0 * rs;
                     TOut *Oc = Ob + (size_t)c0 * rs;
-                    if (a.u_half) {
 #pragma unroll
-                        for (int jj = 0; jj < 8; ++jj) st_global_if(Uhc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
-                    } else {
-#pragma unroll
-                        for (int jj = 0; jj < 8; ++jj) st_global_if(Uc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
+                    for (int jj = 0; jj < 8; ++jj) {
+                        st_global_if(Uc + jj * rs, __uint_as_float(du[jj]), c0 + jj < n);
+                        st_global_if(Oc + jj * rs, __uint_as_float(dout[jj]), c0 + jj < n);
                     }
-#pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) st_global_if(Oc + jj * rs, __uint_as_float(dout[jj]), c0 + jj < n);
                 }
             }
             ptx::tc_fence_before_sync();
@@ -1083,13 +1131,24 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(verify_sm100_tc_kernel<NP, TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
     const long long units = (a.H_v / a.H_qk) % 2 == 0 ? n_items / 2 : n_items;  // the kernel takes heads in pairs
     const int grid = (int)(units < sms ? units : sms);
-    return launch_dependent(verify_sm100_tc_kernel<NP, TOut, FUSED>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream,
-                            a, pv, (int)n_items, m.S0, m.Q, m.K, m.V);
+    auto go = [&](auto kernel) {
+        cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        if (e2 != cudaSuccess) return e2;
+        return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a, pv, (int)n_items, m.S0, m.Q,
+                                m.K, m.V);
+    };
+    if constexpr (FUSED) {
+        return go(verify_sm100_tc_kernel<NP, TOut, true, false, float>);  // (the fused round takes fp32 U)
+    } else {
+        const bool cls = a.cls_lo > 0 || a.cls_hi < a.max_nodes;  // one size class of a mixed batch
+        if (a.u_half)
+            return cls ? go(verify_sm100_tc_kernel<NP, TOut, false, true, __half>)
+                       : go(verify_sm100_tc_kernel<NP, TOut, false, false, __half>);
+        return cls ? go(verify_sm100_tc_kernel<NP, TOut, false, true, float>)
+                   : go(verify_sm100_tc_kernel<NP, TOut, false, false, float>);
+    }
 }
 
 template <bool FUSED>
