@@ -241,6 +241,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         ptx::mbar_init(cmma_done, 1);
         ptx::fence_barrier_init();
     }
+    if (tid == 32) {  // (the descriptors are kernel parameters: fetched while the kernel before this one still runs)
+        ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ);
+        ptx::prefetch_tmap(&tmK), ptx::prefetch_tmap(&tmV);
+    }
     if (warp == C::MMA1_WARP) {
         ptx::tmem_alloc(tmem_slot, VT_TMEM_COLS);
         ptx::tmem_relinquish();
@@ -301,10 +305,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // ------------------------------------------------------------------ producer warp
         const int s = warp - C::PROD_WARP0;
         unsigned char *stage = smem + s * C::STAGE_BYTES;
-        if (lane == 0) {
-            ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ);
-            ptx::prefetch_tmap(&tmK);
-        }
         const int group = a.H_v / a.H_qk;
         // Node scalars of an item: validated and loaded one round ahead (software pipeline), so the
         // dependent chain  node_offsets -> parent / mask / log-gate / beta  never delays a TMA issue.
@@ -866,7 +866,6 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                              &v_ready[kx & 1]);
         };
         if (v_thread) {
-            ptx::prefetch_tmap(&tmV);
             fetch_v(0, first_node(0));
             fetch_v(1, first_node(1));
         }

@@ -112,6 +112,10 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
         for (int s = 0; s < C::STAGES; ++s) reinterpret_cast<VsMeta *>(smem + C::OFF_META + s * C::META_BYTES)->item = -1;
         ptx::fence_barrier_init();
     }
+    if (tid == 32) {  // (the descriptors are kernel parameters: fetched while the kernel before this one still runs)
+        ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ);
+        ptx::prefetch_tmap(&tmK), ptx::prefetch_tmap(&tmV);
+    }
     if (warp == 0) {
         ptx::tmem_alloc(tmem_slot, VS_TMEM_COLS);
         ptx::tmem_relinquish();
@@ -128,7 +132,6 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
         // ------------------------------------------------------------------ producer warp of stage s
         const int s = warp - C::PROD_WARP0;
         unsigned char *stage = smem + s * C::STAGE_BYTES;
-        if (lane == 0) ptx::prefetch_tmap(&tmS0), ptx::prefetch_tmap(&tmQ), ptx::prefetch_tmap(&tmK), ptx::prefetch_tmap(&tmV);
         // An item's scalars are validated and loaded one round ahead, so the dependent chain
         // node_offsets -> parent / mask / log-gate / beta never delays the issue of a copy.
         struct Pre {
