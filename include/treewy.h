@@ -77,7 +77,8 @@ typedef struct {
     int32_t T;                   /* packed nodes, = node_offsets[B] */
     int32_t H_v;                 /* value heads */
     int32_t max_nodes;           /* host-known upper bound on N_b, 1..64; 0 means 64.  Only
-                                    sizes launches; a longer sequence is flagged, not run */
+                                    sizes launches (a tight bound picks the faster kernel: up to
+                                    8, 16, 32 or 64 nodes); a longer sequence is flagged, not run */
     const int32_t *node_offsets; /* [B+1] device, node_offsets[0] = 0 */
     const int32_t *parent;       /* [T]   device, local parent index or -1 */
     int32_t *depth;              /* [T]   device, out: 0 for parent = -1, else depth[parent]+1 */
