@@ -160,3 +160,47 @@ def test_fused_small_round_at_the_chain_workloads_full_size():
     for x, y, name in zip(two, one, ("S", "O", "U", "status")):
         assert torch.equal(x, y), name
     assert not one[3].any()
+
+
+def test_fused_small_round_on_a_state_pool():
+    """commit(r) + verify(r+1) of chains with the states scattered in a pool: bit for bit the plain call."""
+    from paper_2608_20961_b200 import binding as tw
+    dev = torch.device("cuda:0")
+    w1 = wl.make_workload(1, B=6, H_v=4, seed=91)
+    w2 = wl.make_workload(1, B=6, H_v=4, seed=92)
+    n_states = 9
+    perm = torch.randperm(n_states, generator=torch.Generator().manual_seed(3))[: w1.B].to(torch.int32)
+    d = lambda t: t.to(dev)
+
+    def run(pool):
+        status = torch.zeros(w1.B, dtype=torch.int32, device=dev)
+        t1 = tw.Tree.empty(d(w1.node_offsets), d(w1.parent), w1.H_v, 5)
+        t2 = tw.Tree.empty(d(w2.node_offsets), d(w2.parent), w2.H_v, 5)
+        O1 = torch.empty((w1.T, w1.H_v, 128), dtype=torch.bfloat16, device=dev)
+        U1 = torch.empty((w1.T, w1.H_v, 128), dtype=torch.float32, device=dev)
+        O2 = torch.full((w2.T, w2.H_v, 128), 2.0, dtype=torch.bfloat16, device=dev)
+        U2 = torch.full((w2.T, w2.H_v, 128), 2.0, dtype=torch.float32, device=dev)
+        tw.treewy_tree_prepare(t1, d(w1.alpha), status)
+        tw.treewy_tree_prepare(t2, d(w2.alpha), status)
+        if pool:
+            S = torch.full((n_states,) + tuple(w1.S0.shape[1:]), 0.25, dtype=w1.S0.dtype, device=dev)
+            idx = perm.to(dev)
+            S[idx.long()] = d(w1.S0)
+            tw.treewy_verify_pool(S, idx, d(w1.q), d(w1.k), d(w1.v), d(w1.beta), t1, w1.H_qk, O1, U1, status)
+            tw.treewy_commit_verify_pool(S, idx, U1, d(w1.k), t1, d(w1.accepted), d(w2.q), d(w2.k), d(w2.v),
+                                         d(w2.beta), t2, w2.H_qk, O2, U2, True, status)
+            torch.cuda.synchronize()
+            assert torch.all(S[sorted(set(range(n_states)) - set(perm.tolist()))] == 0.25)
+            S = S[idx.long()]
+        else:
+            S = d(w1.S0).clone()
+            tw.treewy_verify(S, d(w1.q), d(w1.k), d(w1.v), d(w1.beta), t1, w1.H_qk, O1, U1, status)
+            tw.treewy_commit_verify(S, U1, d(w1.k), t1, d(w1.accepted), d(w2.q), d(w2.k), d(w2.v), d(w2.beta), t2,
+                                    w2.H_qk, O2, U2, True, status)
+            torch.cuda.synchronize()
+        return S.cpu(), O2.cpu(), U2.cpu(), status.cpu()
+
+    a, b = run(False), run(True)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    assert not a[3].any() and not torch.equal(a[0], w1.S0)
