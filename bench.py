@@ -135,16 +135,18 @@ class LayerSet:
         self.status = torch.zeros(w.B, dtype=torch.int32, device=dev)
         self.tree = tw.Tree.empty(self.off, self.par, w.H_v, w.max_nodes)
 
+    # (trees of more than 64 nodes go through the wide-tree calls)
     def prepare(self):
-        self.tw.treewy_tree_prepare(self.tree, self.alpha, self.status)
+        fn = self.tw.treewy_tree_prepare_wide if self.w.max_nodes > 64 else self.tw.treewy_tree_prepare
+        fn(self.tree, self.alpha, self.status)
 
     def verify(self):
-        self.tw.treewy_verify(self.S0, self.q, self.k, self.v, self.beta, self.tree, self.w.H_qk,
-                              self.O, self.U, self.status)
+        fn = self.tw.treewy_verify_wide if self.w.max_nodes > 64 else self.tw.treewy_verify
+        fn(self.S0, self.q, self.k, self.v, self.beta, self.tree, self.w.H_qk, self.O, self.U, self.status)
 
     def commit(self):
-        self.tw.treewy_commit(self.S0, self.U, self.k, self.tree, self.w.H_qk, self.acc, None,
-                              self.status)
+        fn = self.tw.treewy_commit_wide if self.w.max_nodes > 64 else self.tw.treewy_commit
+        fn(self.S0, self.U, self.k, self.tree, self.w.H_qk, self.acc, None, self.status)
 
     def verify_half(self):
         """verify with the pseudo-values kept in fp16 (own buffer)."""
@@ -191,6 +193,7 @@ def time_oracle(w: wl.Workload, n_seq: int, min_seconds: float = 10.0):
     min_seconds have passed; returns (units/s, seconds, passes, sub-batch, threads)."""
     from oracle import treewy_oracle
     treewy_oracle.build()
+    treewy_oracle.set_max_nodes(max(64, w.max_nodes))   # (64 unless the workload has wider trees)
     sub = w.select_sequences(range(min(n_seq, w.B)))
     args = oracle_inputs(sub)
     passes, t0 = 0, time.perf_counter()
@@ -354,7 +357,7 @@ def run_ours(args, rank: int, size: int, local: int):
 
     # the three calls with U kept in fp16 (treewy_verify_half_u / treewy_commit_half_u): same step shape
     half_u = None
-    if w.io_dtype == torch.bfloat16:
+    if w.io_dtype == torch.bfloat16 and w.max_nodes <= 64:
         for s_ in sets:
             s_.verify_half()
         for i in range(max(args.warmup, 3)):
@@ -380,7 +383,7 @@ def run_ours(args, rank: int, size: int, local: int):
     # the scheme the method replaces, measured on the same inputs: every node's state written out
     storeall = None
     snap_bytes = w.T * w.H_v * 128 * 128 * w.S0.element_size()
-    if w.io_dtype == torch.bfloat16 and snap_bytes < 40e9 and not args.no_snapshot_compare:
+    if w.io_dtype == torch.bfloat16 and w.max_nodes <= 64 and snap_bytes < 40e9 and not args.no_snapshot_compare:
         Snap = torch.empty((w.T, w.H_v, 128, 128), dtype=w.io_dtype, device=dev)
         s0 = sets[0]
         for _ in range(2):

@@ -49,6 +49,7 @@ extern "C" {
 
 #define TREEWY_D 128         /* d_k = d_v */
 #define TREEWY_MAX_NODES 64  /* nodes per sequence (one 64-bit ancestor mask per node) */
+#define TREEWY_MAX_NODES_WIDE 128 /* ... for the *_wide calls, which use no masks */
 
 typedef enum {
     TREEWY_OK = 0,
@@ -230,6 +231,26 @@ treewy_status_t treewy_verify_half_u(const void *S0, const void *q, const void *
 treewy_status_t treewy_commit_half_u(void *S0, const void *U16, const void *k, const treewy_tree_t *tree,
                                      int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
                                      float *S_out_f32, int32_t *seq_status, void *cuda_stream);
+
+/*
+ * Wide draft trees: 65 to TREEWY_MAX_NODES_WIDE nodes per sequence (the draft window is a serving
+ * parameter, Section 4; Eq. 2 and Eq. 3 hold for any N).  The three calls below are
+ * treewy_tree_prepare / treewy_verify / treewy_commit for such batches (smaller trees are accepted
+ * too): the same arguments, layouts, status bits and error behaviour, with these differences:
+ *   - tree->max_nodes may be up to TREEWY_MAX_NODES_WIDE (0 means that);
+ *   - tree->anc_mask is neither written nor read and may be NULL (a root path is walked through the
+ *     parent array instead); depth, cum_log_gate and level_order are written as usual;
+ *   - plain fp32 SIMT kernels, one CTA per (sequence, value head): correct for any tree, an order of
+ *     magnitude slower per node than the main calls; no block-pool, fused or fp16-U variant.
+ */
+treewy_status_t treewy_tree_prepare_wide(const treewy_tree_t *tree, const float *alpha, int32_t *seq_status,
+                                         void *cuda_stream);
+treewy_status_t treewy_verify_wide(const void *S0, const void *q, const void *k, const void *v, const float *beta,
+                                   const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                   treewy_dtype_t o_dtype, void *O, float *U, int32_t *seq_status, void *cuda_stream);
+treewy_status_t treewy_commit_wide(void *S0, const float *U, const void *k, const treewy_tree_t *tree, int32_t H_qk,
+                                   const int32_t *accepted, treewy_dtype_t io_dtype, float *S_out_f32,
+                                   int32_t *seq_status, void *cuda_stream);
 
 /*
  * Full-state snapshotting, the scheme the method replaces (Section 2, "Speculative verification:

@@ -44,7 +44,15 @@
 #include <omp.h>
 #endif
 
-#define ORACLE_MAX_NODES 64
+/* Largest tree taken; larger sequences are flagged.  64 matches the library's main calls (one 64-bit
+ * ancestor mask per node); the tests of the library's wide-tree calls raise it to 128.  Nothing in
+ * the arithmetic below depends on it. */
+static int32_t oracle_max_nodes = 64;
+
+void treewy_oracle_set_max_nodes(int32_t n)
+{
+    oracle_max_nodes = n;
+}
 
 /* per-sequence status bits (same meaning as the library's, restated here) */
 #define ORACLE_SEQ_BAD_PARENT 1
@@ -64,7 +72,7 @@ int treewy_oracle_num_threads(void)
 static int check_sequence(const int32_t *node_offsets, const int32_t *parent, int32_t b)
 {
     const int32_t lo = node_offsets[b], n = node_offsets[b + 1] - lo;
-    if (n < 1 || n > ORACLE_MAX_NODES)
+    if (n < 1 || n > oracle_max_nodes)
         return ORACLE_SEQ_TOO_MANY_NODES;
     for (int32_t i = 0; i < n; ++i) {
         const int32_t p = parent[lo + i];
@@ -95,7 +103,8 @@ int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
         for (int32_t i = 0; i < n; ++i) {
             const int32_t p = parent[lo + i];
             depth[lo + i] = (p < 0) ? 0 : depth[lo + p] + 1;
-            anc_mask[lo + i] = ((p < 0) ? 0ull : anc_mask[lo + p]) | (1ull << i);
+            /* (a 64-bit mask holds the first 64 local nodes; bits of later nodes do not exist) */
+            anc_mask[lo + i] = ((p < 0) ? 0ull : anc_mask[lo + p]) | (i < 64 ? (1ull << i) : 0ull);
             for (int32_t h = 0; h < H_v; ++h) {
                 const double up = (p < 0) ? 0.0 : L[(size_t)(lo + p) * H_v + h];
                 L[(size_t)(lo + i) * H_v + h] = up + log(alpha[(size_t)(lo + i) * H_v + h]);
@@ -127,7 +136,7 @@ int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
  *   S_commit [B, H_v, d_v, d_k]   state at the accepted node
  *   Snap     [T, H_v, d_v, d_k]   every node's state (tests only; large)
  *
- * Malformed sequences (bad parent, node count outside 1..64, accepted outside
+ * Malformed sequences (bad parent, node count outside 1..the limit, accepted outside
  * -1..N-1) are skipped: their outputs are left untouched and seq_status[b] gets
  * the reason OR-ed in.
  */

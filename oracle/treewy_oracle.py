@@ -50,6 +50,11 @@ def _load():
     return _lib
 
 
+def set_max_nodes(n: int = 64) -> None:
+    """Largest tree the oracle takes (default 64, the limit of the library's main calls)."""
+    _load().treewy_oracle_set_max_nodes(ctypes.c_int32(int(n)))
+
+
 def num_threads() -> int:
     """Threads the oracle's OpenMP loop uses (OMP_NUM_THREADS or the core count)."""
     return int(_load().treewy_oracle_num_threads())

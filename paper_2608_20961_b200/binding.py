@@ -85,6 +85,12 @@ def load_library(path: str | None = None):
     lib.treewy_verify_half_u.restype = ctypes.c_int
     lib.treewy_commit_half_u.argtypes = lib.treewy_commit.argtypes
     lib.treewy_commit_half_u.restype = ctypes.c_int
+    lib.treewy_tree_prepare_wide.argtypes = [ctypes.POINTER(TreeStruct), vp, vp, vp]
+    lib.treewy_tree_prepare_wide.restype = ctypes.c_int
+    lib.treewy_verify_wide.argtypes = verify_args
+    lib.treewy_verify_wide.restype = ctypes.c_int
+    lib.treewy_commit_wide.argtypes = lib.treewy_commit.argtypes
+    lib.treewy_commit_wide.restype = ctypes.c_int
     lib.treewy_commit_verify.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), vp, vp, vp, vp, vp,
                                          ctypes.POINTER(TreeStruct), i32, ctypes.c_int, ctypes.c_int, vp, vp, i32, vp, vp]
     lib.treewy_commit_verify.restype = ctypes.c_int
@@ -244,6 +250,31 @@ def treewy_commit_half_u(S0, U16, k, tree: Tree, H_qk: int, accepted, S_out_f32:
                                     _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
 
 
+def treewy_tree_prepare_wide(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tensor | None = None, stream=None) -> None:
+    """treewy_tree_prepare for trees of up to 128 nodes (no ancestor masks are written)."""
+    ts = tree.struct()
+    _check("treewy_tree_prepare_wide",
+           load_library().treewy_tree_prepare_wide(ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream)))
+
+
+def treewy_verify_wide(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,
+                       seq_status: torch.Tensor | None = None, stream=None) -> None:
+    ts = tree.struct()
+    assert q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
+    _check("treewy_verify_wide",
+           load_library().treewy_verify_wide(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+                                             _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status),
+                                             _stream(stream)))
+
+
+def treewy_commit_wide(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
+                       seq_status: torch.Tensor | None = None, stream=None) -> None:
+    ts = tree.struct()
+    _check("treewy_commit_wide",
+           load_library().treewy_commit_wide(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+
+
 def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta, tree: Tree,
                          H_qk: int, O: torch.Tensor, U: torch.Tensor, single_kernel: bool = False,
                          seq_status: torch.Tensor | None = None, stream=None) -> None:
@@ -348,10 +379,13 @@ class VerifyCommitLayer:
 
     def _run(self, b: _StepBuffers, T: int, stream=None) -> None:
         tree = self._tree(b, T)
-        treewy_tree_prepare(tree, b.alpha, self.status, stream)
-        treewy_verify(self.S0, b.q, b.k, b.v, b.beta, tree, self.H_qk, b.O, b.U, self.status, stream)
+        wide = self.max_nodes > 64                      # trees of more than 64 nodes: the wide-tree calls
+        (treewy_tree_prepare_wide if wide else treewy_tree_prepare)(tree, b.alpha, self.status, stream)
+        (treewy_verify_wide if wide else treewy_verify)(self.S0, b.q, b.k, b.v, b.beta, tree, self.H_qk, b.O, b.U,
+                                                        self.status, stream)
         b.verified.record(stream)
-        treewy_commit(self.S0, b.U, b.k, tree, self.H_qk, b.accepted, None, self.status, stream)
+        (treewy_commit_wide if wide else treewy_commit)(self.S0, b.U, b.k, tree, self.H_qk, b.accepted, None,
+                                                        self.status, stream)
 
     def step(self, host: dict, O_host: torch.Tensor) -> None:
         """upload -> prepare -> verify -> outputs to host -> commit, all on the current stream."""

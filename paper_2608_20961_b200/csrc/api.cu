@@ -179,6 +179,81 @@ treewy_status_t treewy_commit_half_u(void *S0, const void *U16, const void *k, c
                          seq_status, cuda_stream);
 }
 
+// the caller-filled part of a wide tree (no mask needed)
+static treewy_status_t check_tree_wide(const treewy_tree_t *t, int *max_nodes)
+{
+    if (!t) return TREEWY_ERR_INVALID_ARG;
+    if (t->B < 0 || t->T < 0 || t->H_v < 1 || t->max_nodes < 0) return TREEWY_ERR_INVALID_ARG;
+    if (t->max_nodes > TREEWY_MAX_NODES_WIDE) return TREEWY_ERR_UNSUPPORTED;
+    *max_nodes = t->max_nodes == 0 ? TREEWY_MAX_NODES_WIDE : t->max_nodes;
+    if (t->B == 0) return TREEWY_OK;
+    if (bad_ptr(t->node_offsets)) return TREEWY_ERR_INVALID_ARG;
+    if (t->T > 0 && (bad_ptr(t->parent) || bad_ptr(t->depth) || bad_ptr(t->cum_log_gate) || bad_ptr(t->level_order)))
+        return TREEWY_ERR_INVALID_ARG;
+    return TREEWY_OK;
+}
+
+treewy_status_t treewy_tree_prepare_wide(const treewy_tree_t *tree, const float *alpha, int32_t *seq_status,
+                                         void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree_wide(tree, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0) return TREEWY_OK;
+    if (tree->T > 0 && bad_ptr(alpha)) return TREEWY_ERR_INVALID_ARG;
+    cudaError_t e = launch_prepare_wide(*tree, max_nodes, alpha, seq_status, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_verify_wide(const void *S0, const void *q, const void *k, const void *v, const float *beta,
+                                   const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                                   treewy_dtype_t o_dtype, void *O, float *U, int32_t *seq_status, void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree_wide(tree, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(io_dtype) || bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0 || tree->T == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(q) || bad_ptr(k) || bad_ptr(v) || bad_ptr(beta) || bad_ptr(O) || bad_ptr(U))
+        return TREEWY_ERR_INVALID_ARG;
+    VerifyArgs a = {};
+    a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.cum_log_gate = tree->cum_log_gate, a.depth = tree->depth, a.level_order = tree->level_order;
+    a.O = O, a.U = U, a.u_half = 0, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.n_states = tree->B, a.cls_lo = 0, a.cls_hi = max_nodes;
+    cudaError_t e = launch_verify_wide(a, io_dtype, o_dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t treewy_commit_wide(void *S0, const float *U, const void *k, const treewy_tree_t *tree, int32_t H_qk,
+                                   const int32_t *accepted, treewy_dtype_t io_dtype, float *S_out_f32,
+                                   int32_t *seq_status, void *cuda_stream)
+{
+    int max_nodes = 0;
+    treewy_status_t st = check_tree_wide(tree, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(io_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (S_out_f32 && misaligned(S_out_f32)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(accepted)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->T > 0 && (bad_ptr(U) || bad_ptr(k))) return TREEWY_ERR_INVALID_ARG;
+    CommitArgs a = {};
+    a.S0 = S0, a.U = U, a.u_half = 0, a.k = k;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent, a.cum_log_gate = tree->cum_log_gate;
+    a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.T = tree->T, a.n_states = tree->B;
+    cudaError_t e = launch_commit_wide(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
 treewy_status_t treewy_verify_pool(const treewy_state_pool_t *pool, const void *q, const void *k, const void *v,
                                    const float *beta, const treewy_tree_t *tree, int32_t H_qk,
                                    treewy_dtype_t io_dtype, treewy_dtype_t o_dtype, void *O, float *U,

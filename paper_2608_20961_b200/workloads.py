@@ -187,6 +187,7 @@ _DEFAULTS = {
     3: ("397B-wide64", 128, 64, 64, torch.bfloat16),
     4: ("ragged-stress", 512, 32, 32, torch.bfloat16),
     5: ("widths-3-3-3", 64, 32, 16, torch.bfloat16),
+    6: ("wide128", 64, 32, 32, torch.bfloat16),
 }
 
 
@@ -195,7 +196,8 @@ def make_workload(config_id: int, seed: int | None = None, B: int | None = None,
                   io_dtype: torch.dtype | None = None, prefix_device: str = "cpu",
                   prefix_tokens: int = 256) -> Workload:
     """Workloads 0-4 are the five benchmark configurations; 5 is a paper-shaped extra
-    (``draft_tree_widths = (3,3,3)`` under one root, N = 40).  ``B``, ``H_v``, ``H_qk``
+    (``draft_tree_widths = (3,3,3)`` under one root, N = 40); 6 has trees of 128 nodes (random
+    parents of depth < 10) for the library's wide-tree calls.  ``B``, ``H_v``, ``H_qk``
     shrink a configuration for parity tests without changing its structure."""
     name, B0, Hv0, Hqk0, dt0 = _DEFAULTS[config_id]
     B = B0 if B is None else B
@@ -228,6 +230,8 @@ def make_workload(config_id: int, seed: int | None = None, B: int | None = None,
             trees.append(random_parent_tree(g, n, 8))
         elif config_id == 5:
             trees.append([-1] + [p + 1 for p in widths_tree((3, 3, 3))])
+        elif config_id == 6:
+            trees.append(random_parent_tree(g, 128, 10))
         else:
             raise ValueError(config_id)
     offsets = [0]

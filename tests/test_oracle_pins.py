@@ -323,3 +323,52 @@ def test_malformed_sequences_are_flagged_and_skipped(oracle):
     off = np.array([0, 65], np.int32)
     tr = oracle.prepare(off, np.full(65, -1, np.int32), np.full((65, 1), 0.9))
     assert list(tr.seq_status) == [oracle.SEQ_TOO_MANY_NODES]
+
+
+# ------------------------------------------------------------------ trees of more than 64 nodes
+
+def test_wide_trees_chain_and_closed_form(oracle):
+    """With the node limit raised to 128 (what the tests of the library's wide-tree calls do) the
+    oracle is still the literal recurrence on a chain and the closed form on a tree; a sequence of
+    129 nodes is flagged; the 64-bit masks keep the bits of the first 64 nodes only."""
+    oracle.set_max_nodes(128)
+    try:
+        r = rng(77)
+        n = 100
+        w = draw(r, [[i - 1 for i in range(n)]], 1, 1, 6, 5)
+        w["accepted"][:] = n - 3
+        res = oracle.verify_commit(**w, want_snapshots=True)
+        states, outs = literal_chain(w["S0"][0, 0], w["k"][:, 0], w["v"][:, 0], w["q"][:, 0],
+                                     w["alpha"][:, 0], w["beta"][:, 0])
+        for i in (0, 63, 64, 65, n - 1):
+            np.testing.assert_allclose(res.Snap[i, 0], states[i], rtol=0, atol=1e-12)
+            np.testing.assert_allclose(res.O[i, 0], outs[i], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(res.S_commit[0, 0], states[n - 3], rtol=0, atol=1e-12)
+
+        trees = [random_tree(r, 128), random_tree(r, 70)]
+        w = draw(r, trees, 2, 1, 8, 8)
+        res = oracle.verify_commit(**w)
+        off = w["node_offsets"]
+        for b in range(2):
+            for h in range(2):
+                Ut, O, Sa = closed_form(w, b, h, 2, 1)
+                sl = slice(int(off[b]), int(off[b + 1]))
+                np.testing.assert_allclose(res.U[sl, h], Ut, rtol=0, atol=1e-11)
+                np.testing.assert_allclose(res.O[sl, h], O, rtol=0, atol=1e-11)
+                np.testing.assert_allclose(res.S_commit[b, h], Sa, rtol=0, atol=1e-11)
+        tree = oracle.prepare(w["node_offsets"], w["parent"], w["alpha"])
+        par = w["parent"]
+        for i in (0, 5, 63, 64, 100, 127):                       # depth and log-gate by walking up
+            d, p, acc = 0, int(par[i]), [i]
+            while p >= 0:
+                d, acc, p = d + 1, acc + [p], int(par[p])
+            assert int(tree.depth[i]) == d
+            np.testing.assert_allclose(tree.cum_log_gate[i, 0], sum(np.log(w["alpha"][j, 0]) for j in sorted(acc)),
+                                       rtol=0, atol=1e-12)
+            assert int(tree.anc_mask[i]) == sum(1 << j for j in acc if j < 64)
+
+        w = draw(r, [[i - 1 for i in range(129)]], 1, 1, 4, 4)
+        res = oracle.verify_commit(**w)
+        assert list(res.seq_status) == [2]
+    finally:
+        oracle.set_max_nodes(64)
