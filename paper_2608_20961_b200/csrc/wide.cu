@@ -86,8 +86,16 @@ prepare_wide_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ n
     }
 }
 
-struct WideSmem {
-    alignas(16) float kf[WN][D];   // k rows of the sequence (this head's q/k head), fp32
+__device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)
+{
+    const uint2 x = *reinterpret_cast<const uint2 *>(p);
+    return make_float4(bf16lo(x.x), bf16hi(x.x), bf16lo(x.y), bf16hi(x.y));
+}
+
+template <typename TIn> struct WideSmem {
+    alignas(16) TIn kf[WN][D];     // k rows of the sequence (this head's q/k head), as stored: bf16 rows
+                                   // leave room for two CTAs per SM
     float uf[WN][D];   // pseudo-values computed so far
     alignas(16) float qrow[D];  // q_i of the node being worked on
     float L[WN], beta[WN];
@@ -101,7 +109,7 @@ template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    WideSmem &sm = *reinterpret_cast<WideSmem *>(smem_raw);
+    WideSmem<TIn> &sm = *reinterpret_cast<WideSmem<TIn> *>(smem_raw);
     const int h = blockIdx.x, b = blockIdx.y;
     const int c = threadIdx.x, lane = c & 31, warp = c >> 5;
     const int lo = a.node_offsets[b];
@@ -115,7 +123,7 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
     }
     const int hq = h / (a.H_v / a.H_qk);
     const TIn *qg = static_cast<const TIn *>(a.q), *kg = static_cast<const TIn *>(a.k), *vg = static_cast<const TIn *>(a.v);
-    for (int i = 0; i < n; ++i) sm.kf[i][c] = to_f32(kg[((size_t)(lo + i) * a.H_qk + hq) * D + c]);
+    for (int i = 0; i < n; ++i) sm.kf[i][c] = kg[((size_t)(lo + i) * a.H_qk + hq) * D + c];
     for (int i = c; i < n; i += WT) {
         sm.L[i] = a.cum_log_gate[(size_t)(lo + i) * a.H_v + h];
         sm.beta[i] = a.beta[(size_t)(lo + i) * a.H_v + h];
@@ -152,8 +160,8 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
             float kk = 0.f, qk = 0.f;
 #pragma unroll
             for (int t = 0; t < D / 32; ++t) {
-                const float kj = sm.kf[j][lane + 32 * t];
-                kk = fmaf(kj, sm.kf[i][lane + 32 * t], kk);
+                const float kj = to_f32(sm.kf[j][lane + 32 * t]);
+                kk = fmaf(kj, to_f32(sm.kf[i][lane + 32 * t]), kk);
                 qk = fmaf(kj, sm.qrow[lane + 32 * t], qk);
             }
             kk = warp_sum(kk), qk = warp_sum(qk);
@@ -167,7 +175,7 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
         float sk0 = 0.f, sk1 = 0.f, sq0 = 0.f, sq1 = 0.f;
 #pragma unroll
         for (int d = 0; d < D; d += 4) {
-            const float4 k4 = *reinterpret_cast<const float4 *>(&sm.kf[i][d]);
+            const float4 k4 = load4(&sm.kf[i][d]);
             const float4 q4 = *reinterpret_cast<const float4 *>(&sm.qrow[d]);
             sk0 = fmaf(srow[d], k4.x, sk0), sk1 = fmaf(srow[d + 1], k4.y, sk1);
             sk0 = fmaf(srow[d + 2], k4.z, sk0), sk1 = fmaf(srow[d + 3], k4.w, sk1);
@@ -284,7 +292,7 @@ cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const flo
 
 template <typename TIn, typename TOut> static cudaError_t launch_vw(const VerifyArgs &a, cudaStream_t stream)
 {
-    const int smem = (int)sizeof(WideSmem);
+    const int smem = (int)sizeof(WideSmem<TIn>);
     cudaError_t e = cudaFuncSetAttribute(verify_wide_kernel<TIn, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     verify_wide_kernel<TIn, TOut><<<dim3(a.H_v, a.B), WT, smem, stream>>>(a);
