@@ -64,3 +64,31 @@ def test_unrelated_branches_do_not_change_a_node():
     cut = _run(small)
     torch.testing.assert_close(cut["O"], big["O"][:keep], rtol=0, atol=2e-5)
     torch.testing.assert_close(cut["U"], big["U"][:keep], rtol=0, atol=2e-5)
+
+
+@pytest.mark.parametrize("hint", [8, 32, 64])
+def test_beta_zero_is_pure_decay_on_every_kernel(hint):
+    """beta = 0 switches the delta rule off (the scalar-gate case): every pseudo-value is exactly 0,
+    o_i = g_i S0 q_i, and the committed state is g_a S0.  One tree size per kernel: the small-tree
+    kernel, the role pipeline's 32-node and 64-node instances, and the SIMT kernel beside each."""
+    from tests.test_gpu_parity import _custom
+    g = torch.Generator().manual_seed(hint)
+    trees = [wl.random_parent_tree(g, hint, 6), [i - 1 for i in range(hint)], [-1]]
+    w = _custom(trees, H_v=4, H_qk=2, seed=hint, accepted=[hint - 1, hint // 2, 0])
+    w.beta[:] = 0.0
+    for generic in (False, True):
+        gpu = pu.run_gpu(w, torch.float32, max_nodes=hint, generic=generic)
+        assert not gpu["status"].any()
+        assert not gpu["U"].any(), "u_i = beta_i (...) = 0 exactly"
+        # gates from the library's own prepare, so that only the kernels under test are compared
+        L = torch.from_numpy(gpu["cum_log_gate"]).double()
+        S0, q = w.S0.double(), w.q.double()
+        off = w.node_offsets.tolist()
+        for b in range(w.B):
+            for h in range(w.H_v):
+                rows = slice(off[b], off[b + 1])
+                want = torch.exp(L[rows, h])[:, None] * (q[rows, h // 2] @ S0[b, h].T)
+                torch.testing.assert_close(gpu["O"][rows, h].double(), want, rtol=0, atol=2e-5 * float(want.abs().max()))
+                a = int(w.accepted[b])
+                torch.testing.assert_close(gpu["S32"][b, h].double(), torch.exp(L[off[b] + a, h]) * S0[b, h],
+                                           rtol=1e-6, atol=1e-9)
