@@ -46,3 +46,56 @@ def test_tensor_core_and_simt_kernels_agree_at_full_size():
     scale = float(b["O"].abs().max())
     assert float((a["O"] - b["O"]).abs().max()) <= 1e-5 * scale
     assert float((a["U"] - b["U"]).abs().max()) <= 1e-5 * float(b["U"].abs().max())
+
+
+def test_full_size_half_u_is_the_rounded_u():
+    """Workload 2 at full size through treewy_verify_half_u / treewy_commit_half_u: U16 = RNE(U32) and the
+    same O, bit for bit; the committed state is the commit of the widened values."""
+    from paper_2608_20961_b200 import binding as tw
+    dev = torch.device("cuda:0")
+    w = wl.make_workload(2)
+    d = lambda t: t.to(dev)
+    tree = tw.Tree.empty(d(w.node_offsets), d(w.parent), w.H_v, w.max_nodes)
+    status = torch.zeros(w.B, dtype=torch.int32, device=dev)
+    q, k, v, beta, acc = d(w.q), d(w.k), d(w.v), d(w.beta), d(w.accepted)
+    tw.treewy_tree_prepare(tree, d(w.alpha), status)
+    out = {}
+    for half in (False, True):
+        S = d(w.S0).clone()
+        O = torch.empty((w.T, w.H_v, 128), dtype=torch.bfloat16, device=dev)
+        U = torch.empty((w.T, w.H_v, 128), dtype=torch.float16 if half else torch.float32, device=dev)
+        if half:
+            tw.treewy_verify_half_u(S, q, k, v, beta, tree, w.H_qk, O, U, status)
+            tw.treewy_commit_half_u(S, U, k, tree, w.H_qk, acc, None, status)
+        else:
+            tw.treewy_verify(S, q, k, v, beta, tree, w.H_qk, O, U, status)
+            tw.treewy_commit(S, U.half().float(), k, tree, w.H_qk, acc, None, status)
+        torch.cuda.synchronize()
+        out[half] = (S, O, U)
+    assert not status.any()
+    assert torch.equal(out[True][1], out[False][1])
+    assert torch.equal(out[True][2], out[False][2].half())
+    assert torch.equal(out[True][0], out[False][0])
+
+
+def test_full_size_wide_trees(oracle):
+    """The 128-node workload through the wide-tree calls, sampled sequences against the oracle."""
+    from tests.test_gpu_wide import run_wide
+    w = wl.make_workload(6)
+    gpu = run_wide(w, max_nodes=w.max_nodes)
+    assert not gpu["status"].any()
+    oracle.set_max_nodes(128)
+    try:
+        seqs = [0, 17, w.B - 1]
+        sub = w.select_sequences(seqs)
+        tree_ref, ref = pu.run_oracle(oracle, sub)
+    finally:
+        oracle.set_max_nodes(64)
+    off = w.node_offsets.numpy()
+    rows = np.array([i for b in seqs for i in range(off[b], off[b + 1])], dtype=np.int64)
+    pick = {"depth": gpu["depth"][rows], "anc_mask": tree_ref.anc_mask, "cum_log_gate": gpu["cum_log_gate"][rows],
+            "level_order": gpu["level_order"][rows], "O": gpu["O"][rows], "U": gpu["U"][rows], "S": gpu["S"][seqs],
+            "S32": gpu["S32"][seqs], "status": gpu["status"][seqs]}
+    errs = pu.assert_parity(sub, pick, tree_ref, ref)
+    print(f"workload 6 full size, sequences {seqs}: {errs}")
+    assert torch.isfinite(gpu["O"]).all() and torch.isfinite(gpu["U"]).all()
