@@ -32,6 +32,8 @@
 // dependent latencies of 6 us per item that four CTAs do not hide.  Gram dot products on CUDA cores:
 // 25 of 128 lanes busy for 2 k cycles, behind the MMA issue in the issuing warp.  Five stages and
 // 544 threads: 96 registers per thread and the Eq. 3 pass spilled.)
+#include <type_traits>
+
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 #include "treewy_common.cuh"
@@ -300,43 +302,55 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                     const float *up = reinterpret_cast<const float *>(stage + C::OFF_UP);
                     // (row r0 + 8 it has r & 7 = r0: the chunk sits at the same swizzled place in every row)
                     unsigned char *base = stage + C::OFF_TILE + (cc >> 3) * VS_HALF + r0 * 128 + (((cc & 7) ^ r0) << 4);
+                    // (the round's code is compiled once per path length up to four: a path of one node
+                    // then issues a quarter of the FMAs, not all of them predicated off)
+                    auto pass = [&](auto ptag) {
+                        constexpr int P = decltype(ptag)::value;
 #pragma unroll 1
-                    for (int it = 0; it < 16; it += 2) {
-                        // two rows per round, every load ahead of the stores (which the compiler must
-                        // otherwise assume to alias the u rows)
-                        uint4 *px0 = reinterpret_cast<uint4 *>(base + it * 1024), *px1 = px0 + 64;
-                        const int r = r0 + 8 * it;
-                        float s0v[8], s1v[8], u0[4], u1[4];
-                        widen8(*px0, s0v);
-                        widen8(*px1, s1v);
+                        for (int it = 0; it < 16; it += 2) {
+                            // two rows per round, every load ahead of the stores (which the compiler must
+                            // otherwise assume to alias the u rows)
+                            uint4 *px0 = reinterpret_cast<uint4 *>(base + it * 1024), *px1 = px0 + 64;
+                            const int r = r0 + 8 * it;
+                            float s0v[8], s1v[8], u0[P > 0 ? P : 1], u1[P > 0 ? P : 1];
+                            widen8(*px0, s0v);
+                            widen8(*px1, s1v);
 #pragma unroll
-                        for (int p = 0; p < 4; ++p) u0[p] = p < plen ? up[p * D + r] : 0.f, u1[p] = p < plen ? up[p * D + r + 8] : 0.f;
+                            for (int p = 0; p < P; ++p) u0[p] = up[p * D + r], u1[p] = up[p * D + r + 8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) s0v[e] *= ga, s1v[e] *= ga;
+                            for (int e = 0; e < 8; ++e) s0v[e] *= ga, s1v[e] *= ga;
 #pragma unroll
-                        for (int p = 0; p < 4; ++p) {
-                            if (p < plen) {
+                            for (int p = 0; p < P; ++p) {
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) s0v[e] = fmaf(u0[p], kwr[p][e], s0v[e]), s1v[e] = fmaf(u1[p], kwr[p][e], s1v[e]);
                             }
-                        }
+                            if constexpr (P == 4) {
 #pragma unroll 1
-                        for (int p = 4; p < plen; ++p) {
-                            float kx[8];
-                            widen8(*reinterpret_cast<const uint4 *>(stage + C::OFF_KP + p * D * 2 + cc * 16), kx);
-                            const float w = meta->w[p], ua = up[p * D + r], ub = up[p * D + r + 8];
+                                for (int p = 4; p < plen; ++p) {
+                                    float kx[8];
+                                    widen8(*reinterpret_cast<const uint4 *>(stage + C::OFF_KP + p * D * 2 + cc * 16), kx);
+                                    const float w = meta->w[p], ua = up[p * D + r], ub = up[p * D + r + 8];
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const float kwv = kx[e] * w;
-                                s0v[e] = fmaf(ua, kwv, s0v[e]), s1v[e] = fmaf(ub, kwv, s1v[e]);
+                                    for (int e = 0; e < 8; ++e) {
+                                        const float kwv = kx[e] * w;
+                                        s0v[e] = fmaf(ua, kwv, s0v[e]), s1v[e] = fmaf(ub, kwv, s1v[e]);
+                                    }
+                                }
                             }
+                            uint4 y0, y1;
+                            y0.x = pack_bf16(s0v[0], s0v[1]), y0.y = pack_bf16(s0v[2], s0v[3]);
+                            y0.z = pack_bf16(s0v[4], s0v[5]), y0.w = pack_bf16(s0v[6], s0v[7]);
+                            y1.x = pack_bf16(s1v[0], s1v[1]), y1.y = pack_bf16(s1v[2], s1v[3]);
+                            y1.z = pack_bf16(s1v[4], s1v[5]), y1.w = pack_bf16(s1v[6], s1v[7]);
+                            *px0 = y0, *px1 = y1;
                         }
-                        uint4 y0, y1;
-                        y0.x = pack_bf16(s0v[0], s0v[1]), y0.y = pack_bf16(s0v[2], s0v[3]);
-                        y0.z = pack_bf16(s0v[4], s0v[5]), y0.w = pack_bf16(s0v[6], s0v[7]);
-                        y1.x = pack_bf16(s1v[0], s1v[1]), y1.y = pack_bf16(s1v[2], s1v[3]);
-                        y1.z = pack_bf16(s1v[4], s1v[5]), y1.w = pack_bf16(s1v[6], s1v[7]);
-                        *px0 = y0, *px1 = y1;
+                    };
+                    switch (plen < 4 ? plen : 4) {
+                    case 0: pass(std::integral_constant<int, 0>{}); break;
+                    case 1: pass(std::integral_constant<int, 1>{}); break;
+                    case 2: pass(std::integral_constant<int, 2>{}); break;
+                    case 3: pass(std::integral_constant<int, 3>{}); break;
+                    default: pass(std::integral_constant<int, 4>{}); break;
                     }
                     ptx::fence_proxy_async();  // written by ordinary stores, read by the TMA store and the tensor core
                 }
