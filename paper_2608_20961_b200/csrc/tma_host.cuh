@@ -15,12 +15,17 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 inline EncodeTiledFn tma_encode_fn()
 {
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-        return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(fn);
+    // (looked up once per process: the entry point does not change, and the lookup is a microsecond
+    // on every launch otherwise)
+    static const EncodeTiledFn cached = [] {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(fn);
+    }();
+    return cached;
 }
 
 // bf16 matrix [rows, cols] with `row_bytes` between rows; box = box_cols x box_rows
