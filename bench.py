@@ -13,12 +13,18 @@ follows the rest of the forward pass -- so no kernel is timed on an L2-resident 
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config ID] [--impl reference]
 
+Timing: after W warm-up steps, blocks of exactly K steps are timed back to back with CUDA events on
+the launching stream (at least five blocks, tens of milliseconds in all); `value` and `ms_per_step`
+are the median block, min and max stand beside them.  The other benchmark workloads are timed with
+the same code and reported under `workloads`.
+
 N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange
 step, so there is no data-path collective (weak scaling).
 """
 from __future__ import annotations
 
 import argparse
+import contextlib
 import json
 import os
 import sys
@@ -37,11 +43,14 @@ from paper_2608_20961_b200 import workloads as wl  # noqa: E402
 METRIC = "gdn_tree_verify_commit_node_heads_per_s_per_layer"
 UNIT = "node*heads/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0          # the nominal HBM3e figure the target also names; context, not the denominator
+OTHER_WORKLOADS = (1, 3, 4, 6)    # timed beside the headline workload: 35B-chain5, 397B-wide64, ragged-stress, wide128
 
 # DRAM bytes per launch of the verify kernel on the bench workload: dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture at batch 96 (151.9 MB + 40.3 MB), scaled by 256/96
 # (traffic is linear in the batch).  Writes still dirty in L2 at kernel end are not in it.
-VERIFY_DRAM_TRAFFIC_BYTES = {2: int((151.9e6 + 40.3e6) * 256 / 96)}
+VERIFY_DRAM_TRAFFIC = {2: {"bytes": int((151.9e6 + 40.3e6) * 256 / 96),
+                           "source": "ncu capture at batch 96 scaled by 256/96: profiles/kernels_35B-tree32_b96.md"}}
 
 
 def measured_peaks():
@@ -56,7 +65,7 @@ def measured_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.004):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -120,7 +129,10 @@ def physical_gpu_index(local: int) -> int:
 
 
 class LayerSet:
-    """Device buffers of one GDN layer for one batch of draft trees."""
+    """Device buffers of one GDN layer for one batch of draft trees, and the library calls on them
+    with their arguments marshalled once (``binding.prebound``): a decoding loop calls the library
+    with the same buffers step after step, and on the small workloads the Python work of building
+    structs and pointer objects per call would otherwise be a visible part of the step."""
 
     def __init__(self, w: wl.Workload, dev: torch.device):
         from paper_2608_20961_b200 import binding as tw
@@ -134,38 +146,44 @@ class LayerSet:
         self.U = torch.empty((w.T, w.H_v, 128), dtype=torch.float32, device=dev)
         self.status = torch.zeros(w.B, dtype=torch.int32, device=dev)
         self.tree = tw.Tree.empty(self.off, self.par, w.H_v, w.max_nodes)
+        wide = w.max_nodes > 64          # trees of more than 64 nodes go through the wide-tree calls
+        self.prepare = tw.prebound(tw.treewy_tree_prepare_wide if wide else tw.treewy_tree_prepare,
+                                   self.tree, self.alpha, self.status)
+        self.verify = tw.prebound(tw.treewy_verify_wide if wide else tw.treewy_verify, self.S0, self.q, self.k,
+                                  self.v, self.beta, self.tree, w.H_qk, self.O, self.U, self.status)
+        self.commit = tw.prebound(tw.treewy_commit_wide if wide else tw.treewy_commit, self.S0, self.U, self.k,
+                                  self.tree, w.H_qk, self.acc, None, self.status)
+        self._half = self._fused = None
+        self._flip = 0
 
-    # (trees of more than 64 nodes go through the wide-tree calls)
-    def prepare(self):
-        fn = self.tw.treewy_tree_prepare_wide if self.w.max_nodes > 64 else self.tw.treewy_tree_prepare
-        fn(self.tree, self.alpha, self.status)
-
-    def verify(self):
-        fn = self.tw.treewy_verify_wide if self.w.max_nodes > 64 else self.tw.treewy_verify
-        fn(self.S0, self.q, self.k, self.v, self.beta, self.tree, self.w.H_qk, self.O, self.U, self.status)
-
-    def commit(self):
-        fn = self.tw.treewy_commit_wide if self.w.max_nodes > 64 else self.tw.treewy_commit
-        fn(self.S0, self.U, self.k, self.tree, self.w.H_qk, self.acc, None, self.status)
+    def _half_calls(self):
+        """verify / commit with the pseudo-values kept in fp16 (own buffer)."""
+        if self._half is None:
+            tw, w = self.tw, self.w
+            self.U16 = torch.empty((w.T, w.H_v, 128), dtype=torch.float16, device=self.O.device)
+            self._half = (tw.prebound(tw.treewy_verify_half_u, self.S0, self.q, self.k, self.v, self.beta, self.tree,
+                                      w.H_qk, self.O, self.U16, self.status),
+                          tw.prebound(tw.treewy_commit_half_u, self.S0, self.U16, self.k, self.tree, w.H_qk, self.acc,
+                                      None, self.status))
+        return self._half
 
     def verify_half(self):
-        """verify with the pseudo-values kept in fp16 (own buffer)."""
-        if not hasattr(self, "U16"):
-            self.U16 = torch.empty((self.w.T, self.w.H_v, 128), dtype=torch.float16, device=self.O.device)
-        self.tw.treewy_verify_half_u(self.S0, self.q, self.k, self.v, self.beta, self.tree, self.w.H_qk,
-                                     self.O, self.U16, self.status)
+        self._half_calls()[0]()
 
     def commit_half(self):
-        self.tw.treewy_commit_half_u(self.S0, self.U16, self.k, self.tree, self.w.H_qk, self.acc, None,
-                                     self.status)
+        self._half_calls()[1]()
 
     def commit_verify(self):
         """Commit of the previous round fused into this round's verify (U double-buffered)."""
-        if not hasattr(self, "U2"):
+        if self._fused is None:
+            tw, w = self.tw, self.w
             self.U2 = torch.empty_like(self.U)
-        self.tw.treewy_commit_verify(self.S0, self.U, self.k, self.tree, self.acc, self.q, self.k, self.v,
-                                     self.beta, self.tree, self.w.H_qk, self.O, self.U2, True, self.status)
-        self.U, self.U2 = self.U2, self.U
+            mk = lambda u_prev, u_new: tw.prebound(tw.treewy_commit_verify, self.S0, u_prev, self.k, self.tree,
+                                                   self.acc, self.q, self.k, self.v, self.beta, self.tree, w.H_qk,
+                                                   self.O, u_new, True, self.status)
+            self._fused = (mk(self.U, self.U2), mk(self.U2, self.U))
+        self._fused[self._flip]()
+        self._flip ^= 1
 
 
 def pass_bytes(w: wl.Workload) -> footprint.PassBytes:
@@ -243,49 +261,48 @@ def run_reference(args, rank: int):
     }))
 
 
-def run_ours(args, rank: int, size: int, local: int):
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: libtreewy has no CPU path")
-    dev = torch.device("cuda", local)
-    torch.cuda.set_device(dev)
-    from paper_2608_20961_b200 import binding as tw
-    tw.load_library()
-
-    w = wl.make_workload(args.config, B=args.batch, prefix_device=str(dev))
-    units = w.T * w.H_v
-    pb = pass_bytes(w)
-    sets = [LayerSet(w, dev) for _ in range(2)]
-    for s in sets:                       # every set holds a verified tree before step 0
-        s.prepare(), s.verify()
+def timed_blocks(step, steps: int, dev, stream, start: int = 0, min_total_ms: float = 40.0, sampler=None):
+    """Times blocks of exactly `steps` steps back to back with CUDA events on the launching stream:
+    at least five blocks, more when a block is short, so that the whole timed region lasts tens of
+    milliseconds.  Barrier and device synchronisation on both sides.  Returns the per-block times
+    (ms, this rank) and the index of the next step."""
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    p0, p1 = ev(), ev()
+    p0.record(stream)
+    for i in range(steps):                      # pilot block: sizes the run, not reported
+        step(start + i)
+    p1.record(stream)
     torch.cuda.synchronize(dev)
-
-    def step(i: int):
-        a, b = sets[i % 2], sets[(i + 1) % 2]
-        a.prepare()
-        a.verify()
-        b.commit()
-
-    stream = torch.cuda.current_stream(dev)
-    for i in range(args.warmup):
-        step(i)
-    torch.cuda.synchronize(dev)
+    start += steps
+    pilot = max(p0.elapsed_time(p1), 1e-3)
+    n_blocks = int(min(400, max(5, -(-min_total_ms // pilot))))
+    marks = [ev() for _ in range(n_blocks + 1)]
     replicas.barrier(dev)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(physical_gpu_index(local)) as clocks:
-        e0.record(stream)
-        for i in range(args.steps):
-            step(args.warmup + i)
-        e1.record(stream)
+    torch.cuda.synchronize(dev)
+    ctx = sampler if sampler is not None else contextlib.nullcontext()
+    with ctx:
+        marks[0].record(stream)
+        for blk in range(n_blocks):
+            for i in range(steps):
+                step(start + blk * steps + i)
+            marks[blk + 1].record(stream)
         torch.cuda.synchronize(dev)
     replicas.barrier(dev)
-    ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
-    ms_per_step = ms / args.steps
-    value = size * units * args.steps / (ms * 1e-3)
+    return [marks[i].elapsed_time(marks[i + 1]) for i in range(n_blocks)], start + n_blocks * steps
 
-    # per-kernel durations, separate pass: events around every launch on the launching stream
-    kb = max(3, min(args.steps, 50))
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(kb)]
-    for i in range(kb):
+
+def block_stats(block_ms, steps: int, dev):
+    """Median / min / max over the blocks of the time per step, each the MAX over ranks."""
+    s = sorted(block_ms)
+    med = 0.5 * (s[(len(s) - 1) // 2] + s[len(s) // 2])
+    f = lambda x: replicas.max_over_ranks(x, dev) / steps
+    return {"median": f(med), "min": f(s[0]), "max": f(s[-1]), "blocks": len(s)}
+
+
+def kernel_times(sets, dev, stream, reps: int):
+    """Per-call durations (ms), separate pass: events around every call on the launching stream."""
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+    for i in range(reps):
         a, b = sets[i % 2], sets[(i + 1) % 2]
         ev[i][0].record(stream)
         a.prepare()
@@ -295,19 +312,97 @@ def run_ours(args, rank: int, size: int, local: int):
         b.commit()
         ev[i][3].record(stream)
     torch.cuda.synchronize(dev)
-    kt = [sum(e[j].elapsed_time(e[j + 1]) for e in ev) / kb for j in range(3)]   # ms
-    assert not any(int(s.status.max()) for s in sets), "a sequence was flagged"
+    return [sum(e[j].elapsed_time(e[j + 1]) for e in ev) / reps for j in range(3)]
 
+
+def host_cost_per_call(ls: LayerSet, dev, n: int = 300):
+    """Host time of one enqueue (microseconds): n calls of each entry point through its marshalled
+    C call, no synchronisation inside, wall clock / n.  The queue is drained between the three."""
+    out = {}
+    for name in ("prepare", "verify", "commit"):
+        call = getattr(ls, name)
+        torch.cuda.synchronize(dev)
+        t0 = time.perf_counter()
+        for _ in range(n):
+            call()
+        out[name] = (time.perf_counter() - t0) / n * 1e6
+        torch.cuda.synchronize(dev)
+    return out
+
+
+def n_launches(w: wl.Workload) -> int:
+    """Kernels per prepare + verify + commit step: a bf16 batch whose trees may exceed 32 nodes verifies
+    in two launches (one per size class)."""
+    return 4 if w.io_dtype == torch.bfloat16 and 32 < w.max_nodes <= 64 else 3
+
+
+def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampler=None):
+    """The step (prepare + verify + commit, two layer sets rotated) on one workload: block-median time,
+    per-kernel times, roofline fractions against the measured and the nominal bandwidth."""
+    pb = pass_bytes(w)
+    sets = [LayerSet(w, dev) for _ in range(2)]
+    for s_ in sets:                      # every set holds a verified tree before step 0
+        s_.prepare(), s_.verify()
+    torch.cuda.synchronize(dev)
+
+    def step(i: int):
+        a, b = sets[i % 2], sets[(i + 1) % 2]
+        a.prepare()
+        a.verify()
+        b.commit()
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize(dev)
+    blocks, nxt = timed_blocks(step, steps, dev, stream, start=warmup, sampler=sampler)
+    st = block_stats(blocks, steps, dev)
+    kt = kernel_times(sets, dev, stream, max(3, min(steps, 50)))
+    assert not any(int(s_.status.max()) for s_ in sets), "a sequence was flagged"
     hbm, tf, which = measured_peaks()
-    verify_gbs = pb.verify / (kt[1] * 1e-3) / 1e9
     roof_ms = max(pb.total / (hbm * 1e9), pb.tensor_flops / (tf * 1e12)) * 1e3
+    nominal_ms = pb.total / (NOMINAL_HBM_GBS * 1e9) * 1e3
+    rec = {
+        "ms_per_step": st["median"], "ms_per_step_min": st["min"], "ms_per_step_max": st["max"],
+        "blocks": st["blocks"], "steps_per_block": steps,
+        "kernel_ms": {"prepare": kt[0], "verify": kt[1], "commit": kt[2]},
+        "kernel_gbs": {"prepare": pb.prepare / kt[0] / 1e6, "verify": pb.verify / kt[1] / 1e6,
+                       "commit": pb.commit / kt[2] / 1e6},
+        "step_roofline": {"bytes": pb.total, "tensor_flops": pb.tensor_flops, "roof_ms": roof_ms,
+                          "frac": roof_ms / st["median"], "peak_source": f"of {which}",
+                          "frac_of_nominal_8tbs": nominal_ms / st["median"]},
+        "gpu_launches_per_step": n_launches(w),
+    }
+    return rec, sets, pb, kt
+
+
+def run_ours(args, rank: int, size: int, local: int):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libtreewy has no CPU path")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    from paper_2608_20961_b200 import binding as tw
+    tw.load_library()
+    stream = torch.cuda.current_stream(dev)
+    hbm, tf, which = measured_peaks()
+
+    w = wl.make_workload(args.config, B=args.batch, prefix_device=str(dev))
+    units = w.T * w.H_v
+    clocks = ClockSampler(physical_gpu_index(local))
+    main, sets, pb, kt = measure_workload(w, dev, stream, args.steps, args.warmup, sampler=clocks)
+    ms_per_step = main["ms_per_step"]
+    value = size * units / (ms_per_step * 1e-3)
+
+    verify_gbs = pb.verify / (kt[1] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "treewy_verify", "achieved": verify_gbs, "peak": hbm,
                 "unit": "GB/s", "frac": verify_gbs / hbm, "peak_source": f"of {which}",
-                "traffic": VERIFY_DRAM_TRAFFIC_BYTES.get(args.config),
+                "frac_of_nominal_8tbs": verify_gbs / NOMINAL_HBM_GBS,
+                "traffic": VERIFY_DRAM_TRAFFIC.get(args.config, {}).get("bytes"),
+                "traffic_source": VERIFY_DRAM_TRAFFIC.get(args.config, {}).get("source"),
                 "algorithmic_bytes_per_launch": pb.verify}
 
     # end to end through the user-level API: pinned host inputs in, outputs back, every step;
     # consecutive steps are pipelined over upload / compute / download streams
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ke = max(4, min(args.steps, 20))
     layer = tw.VerifyCommitLayer(sets[0].S0, w.H_qk, w.T, w.max_nodes)
     names = ("q", "k", "v", "alpha", "beta", "parent", "node_offsets", "accepted")
@@ -332,52 +427,46 @@ def run_ours(args, rank: int, size: int, local: int):
     e2e = {"value": size * units * ke / (e2e_ms * 1e-3), "unit": UNIT, "steps": ke,
            "ms_per_step": e2e_ms / ke, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
            "note": "pinned host buffers; upload, kernels and download pipelined over three streams"}
+    del layer, hosts, O_hosts
+
+    def variant(step, warm_first=None):
+        if warm_first is not None:
+            warm_first()
+        for i in range(max(args.warmup, 3)):
+            step(i)
+        torch.cuda.synchronize(dev)
+        blocks, _ = timed_blocks(step, args.steps, dev, stream, start=max(args.warmup, 3), min_total_ms=20.0)
+        return block_stats(blocks, args.steps, dev)
 
     # the same hot path with the commit of round r fused into the verify of round r+1
     # (treewy_commit_verify): step = prepare + commit_verify on one layer set, sets rotated
     fused = None
     if w.io_dtype == torch.bfloat16 and w.max_nodes <= 32:
-        for i in range(max(args.warmup, 3)):
-            sets[i % 2].prepare(), sets[i % 2].commit_verify()
-        torch.cuda.synchronize(dev)
-        replicas.barrier(dev)
-        e0.record(stream)
-        for i in range(args.steps):
-            sets[i % 2].prepare(), sets[i % 2].commit_verify()
-        e1.record(stream)
-        torch.cuda.synchronize(dev)
-        fms = replicas.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+        st = variant(lambda i: (sets[i % 2].prepare(), sets[i % 2].commit_verify()))
         fbytes = pb.total - w.B * w.H_v * 128 * 128 * w.S0.element_size()   # the state is read once
         fused = {"what": "prepare + treewy_commit_verify(single_kernel=1) per step: the previous round's commit "
                          "and this round's verify in one kernel, state read once and written once",
-                 "ms_per_step": fms, "value": size * units / (fms * 1e-3), "unit": UNIT,
+                 "ms_per_step": st["median"], "ms_per_step_min": st["min"], "ms_per_step_max": st["max"],
+                 "value": size * units / (st["median"] * 1e-3), "unit": UNIT,
                  "algorithmic_bytes": fbytes, "roof_ms": fbytes / (hbm * 1e9) * 1e3,
-                 "frac": fbytes / (hbm * 1e9) * 1e3 / fms, "gpu_launches": 2 * args.steps}
+                 "frac": fbytes / (hbm * 1e9) * 1e3 / st["median"],
+                 "frac_of_nominal_8tbs": fbytes / (NOMINAL_HBM_GBS * 1e9) * 1e3 / st["median"],
+                 "gpu_launches_per_step": 2}
         assert not any(int(s_.status.max()) for s_ in sets), "a sequence was flagged"
 
     # the three calls with U kept in fp16 (treewy_verify_half_u / treewy_commit_half_u): same step shape
     half_u = None
     if w.io_dtype == torch.bfloat16 and w.max_nodes <= 64:
-        for s_ in sets:
-            s_.verify_half()
-        for i in range(max(args.warmup, 3)):
-            sets[i % 2].prepare(), sets[i % 2].verify_half(), sets[(i + 1) % 2].commit_half()
-        torch.cuda.synchronize(dev)
-        replicas.barrier(dev)
-        e0.record(stream)
-        for i in range(args.steps):
-            sets[i % 2].prepare(), sets[i % 2].verify_half(), sets[(i + 1) % 2].commit_half()
-        e1.record(stream)
-        torch.cuda.synchronize(dev)
-        hms = replicas.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
+        st = variant(lambda i: (sets[i % 2].prepare(), sets[i % 2].verify_half(), sets[(i + 1) % 2].commit_half()),
+                     warm_first=lambda: [s_.verify_half() for s_ in sets])
         off_, par_ = w.node_offsets.tolist(), w.parent.tolist()
         plen_total = sum(wl.tree_depths(par_[off_[b]:off_[b + 1]])[int(w.accepted[b])] + 1
                          for b in range(w.B) if int(w.accepted[b]) >= 0)   # path rows commit reads, per head
         hbytes = pb.total - 2 * w.T * w.H_v * 128 - 2 * plen_total * w.H_v * 128   # U: 2 bytes instead of 4
         half_u = {"what": "prepare + treewy_verify_half_u + treewy_commit_half_u per step: U stored as fp16",
-                  "ms_per_step": hms, "value": size * units / (hms * 1e-3), "unit": UNIT,
+                  "ms_per_step": st["median"], "value": size * units / (st["median"] * 1e-3), "unit": UNIT,
                   "algorithmic_bytes": hbytes, "roof_ms": hbytes / (hbm * 1e9) * 1e3,
-                  "frac": hbytes / (hbm * 1e9) * 1e3 / hms, "gpu_launches": 3 * args.steps}
+                  "frac": hbytes / (hbm * 1e9) * 1e3 / st["median"], "gpu_launches_per_step": n_launches(w)}
         assert not any(int(s_.status.max()) for s_ in sets), "a sequence was flagged"
 
     # the scheme the method replaces, measured on the same inputs: every node's state written out
@@ -410,6 +499,25 @@ def run_ours(args, rank: int, size: int, local: int):
         l2_note = (f"two layer sets ({set_bytes / 1e6:.0f} MB each, {2 * set_bytes / 1e6:.0f} MB together against a "
                    "126 MB L2) rotated, commit runs one step after its verify: this small configuration is "
                    "partly L2-resident and is not the headline workload")
+    host_us = host_cost_per_call(sets[0], dev)
+    del sets
+    torch.cuda.empty_cache()
+
+    # the other benchmark workloads, same step and timing code (no end-to-end or CPU leg)
+    others = {}
+    if not args.no_other_workloads and args.batch is None:
+        for cid in OTHER_WORKLOADS:
+            if cid == args.config:
+                continue
+            wo = wl.make_workload(cid, prefix_device=str(dev))
+            rec, osets, _, _ = measure_workload(wo, dev, stream, args.steps, args.warmup)
+            rec["value"] = size * wo.T * wo.H_v / (rec["ms_per_step"] * 1e-3)
+            rec["config"] = {"B": wo.B, "H_v": wo.H_v, "H_qk": wo.H_qk, "T": wo.T, "max_nodes": wo.max_nodes}
+            rec["host_us_per_call"] = host_cost_per_call(osets[0], dev)
+            others[wo.name] = rec
+            del osets, wo
+            torch.cuda.empty_cache()
+
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -418,20 +526,22 @@ def run_ours(args, rank: int, size: int, local: int):
         "config": {"workload": w.name, "B": w.B, "H_v": w.H_v, "H_qk": w.H_qk, "T": w.T,
                    "max_nodes": w.max_nodes, "seed": w.seed,
                    "l2": l2_note,
+                   "timing": f"median of {main['blocks']} back-to-back blocks of {args.steps} steps "
+                             "(CUDA events on the launching stream, MAX over ranks)",
                    "parallelism": f"replicas x{size}, no collective"},
+        "ms_per_step_min": main["ms_per_step_min"], "ms_per_step_max": main["ms_per_step_max"],
+        "blocks": main["blocks"],
         "clocks": clocks.summary(), "e2e": e2e,
-        # prepare + verify + commit; a bf16 batch whose trees may exceed 32 nodes verifies in two launches
-        # (one per size class)
-        "gpu_launches": (4 if w.io_dtype == torch.bfloat16 and w.max_nodes > 32 else 3) * args.steps,
+        "gpu_launches": n_launches(w) * args.steps,
         "roofline": roofline,
-        "step_roofline": {"bytes": pb.total, "tensor_flops": pb.tensor_flops, "roof_ms": roof_ms,
-                          "frac": roof_ms / ms_per_step, "peak_source": f"of {which}"},
-        "kernel_ms": {"prepare": kt[0], "verify": kt[1], "commit": kt[2]},
-        "kernel_gbs": {"prepare": pb.prepare / kt[0] / 1e6, "verify": verify_gbs,
-                       "commit": pb.commit / kt[2] / 1e6},
+        "step_roofline": main["step_roofline"],
+        "kernel_ms": main["kernel_ms"],
+        "kernel_gbs": main["kernel_gbs"],
+        "host_us_per_call": host_us,
         "footprint": footprint.footprint_report(w.max_nodes, w.H_v, w.H_qk),
         "snapshot_comparator": storeall,
         "fused_commit_verify": fused, "half_u": half_u,
+        "workloads": others,
     }
     if rank == 0 and size == 1 and not args.no_cpu_baseline:
         v, dt, passes, sub, cores = time_oracle(w, args.cpu_seqs)
@@ -455,6 +565,8 @@ def main():
     ap.add_argument("--ref-seqs", type=int, default=16, help="sequences per reference-arm step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-snapshot-compare", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="time the selected workload only (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank, size, local = replicas.world()

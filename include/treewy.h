@@ -66,7 +66,9 @@ enum {
     TREEWY_SEQ_TOO_MANY_NODES = 2, /* N_b outside 1..max_nodes */
     TREEWY_SEQ_BAD_ACCEPTED = 4,   /* accepted[b] outside -1..N_b-1 */
     TREEWY_SEQ_TIMEOUT = 8,        /* a bounded wait inside a kernel gave up */
-    TREEWY_SEQ_BAD_STATE = 16      /* state_index[b] outside 0..n_states-1 (block-pool calls) */
+    TREEWY_SEQ_BAD_STATE = 16,     /* state_index[b] outside 0..n_states-1 (block-pool calls) */
+    TREEWY_SEQ_BAD_OFFSETS = 32    /* node_offsets[b] .. node_offsets[b+1] is not a range inside 0..T
+                                      (negative, decreasing or past the T packed nodes of the tree) */
 };
 
 /*
@@ -265,6 +267,18 @@ treewy_status_t treewy_commit_wide(void *S0, const float *U, const void *k, cons
 treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *k, const treewy_tree_t *tree,
                                     int32_t H_qk, treewy_dtype_t io_dtype, void *Snap, int32_t *seq_status,
                                     void *cuda_stream);
+
+/*
+ * Test hook (the paper has no counterpart).  Every wait inside the pipelined kernels is bounded by one
+ * deadline per kernel, about two seconds of SM clocks; a kernel whose wait runs out sets
+ * TREEWY_SEQ_TIMEOUT on the sequence it was working on, frees what it holds and returns, and the
+ * stream stays usable.  This call lets a test reach that path on purpose, without a fault:
+ *   wait_cycles  limit of the bounded waits of later launches, in SM clocks (0 restores the default);
+ *   skip_item    the (sequence * H_v + head) item whose loads treewy_verify's kernel for trees of
+ *                9 to 64 nodes never issues, so every role runs into the limit (-1 = none).
+ * Process-wide and not thread-safe: the only state the library keeps; never call it in production.
+ */
+void treewy_debug_inject(int64_t wait_cycles, int32_t skip_item);
 
 /* A short constant string for a status code. */
 const char *treewy_status_string(treewy_status_t status);

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libtreewy.so")
 
 TREEWY_OK, TREEWY_ERR_INVALID_ARG, TREEWY_ERR_UNSUPPORTED, TREEWY_ERR_CUDA = 0, 1, 2, 3
 TREEWY_F32, TREEWY_BF16 = 0, 1
-SEQ_BAD_PARENT, SEQ_TOO_MANY_NODES, SEQ_BAD_ACCEPTED, SEQ_TIMEOUT, SEQ_BAD_STATE = 1, 2, 4, 8, 16
+SEQ_BAD_PARENT, SEQ_TOO_MANY_NODES, SEQ_BAD_ACCEPTED, SEQ_TIMEOUT, SEQ_BAD_STATE, SEQ_BAD_OFFSETS = 1, 2, 4, 8, 16, 32
 D = 128
 MAX_NODES = 64
 
@@ -100,6 +100,8 @@ def load_library(path: str | None = None):
     lib.treewy_commit_verify_pool.restype = ctypes.c_int
     lib.treewy_snapshot_all.argtypes = [vp, vp, vp, ctypes.POINTER(TreeStruct), i32, ctypes.c_int, vp, vp, vp]
     lib.treewy_snapshot_all.restype = ctypes.c_int
+    lib.treewy_debug_inject.argtypes = [ctypes.c_int64, ctypes.c_int32]
+    lib.treewy_debug_inject.restype = None
     lib.treewy_status_string.argtypes = [ctypes.c_int]
     lib.treewy_status_string.restype = ctypes.c_char_p
     lib.treewy_version.restype = ctypes.c_int
@@ -115,6 +117,12 @@ def version() -> int:
     return int(load_library().treewy_version())
 
 
+def treewy_debug_inject(wait_cycles: int = 0, skip_item: int = -1) -> None:
+    """Test hook: limit of the kernels' bounded waits (SM clocks, 0 = default) and the one item whose
+    loads the tree-verify kernel never issues (-1 = none).  Process-wide; tests only."""
+    load_library().treewy_debug_inject(int(wait_cycles), int(skip_item))
+
+
 def _p(t: torch.Tensor | None):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
@@ -128,6 +136,48 @@ def _stream(stream) -> ctypes.c_void_p:
 def _check(fn: str, code: int):
     if code != TREEWY_OK:
         raise TreewyError(fn, code)
+
+
+_recording: list | None = None
+
+
+def _call(name: str, cfunc, *cargs):
+    """Invoke one C entry point with marshalled arguments (or, inside ``prebound``, record it)."""
+    if _recording is not None:
+        _recording.append((name, cfunc, cargs))
+        return
+    _check(name, cfunc(*cargs))
+
+
+class Prebound:
+    """C calls with their arguments already marshalled: calling the object enqueues them again on
+    the stream(s) they were recorded with.  For loops that call the library with the same buffers
+    step after step (a decoding loop over fixed device buffers): the per-call Python work of
+    building structs and pointer objects is done once."""
+
+    def __init__(self, calls, keep):
+        self._calls, self._keep = calls, keep
+
+    def __call__(self) -> None:
+        for name, cfunc, cargs in self._calls:
+            code = cfunc(*cargs)
+            if code != TREEWY_OK:
+                raise TreewyError(name, code)
+
+
+def prebound(fn, *args, **kwargs) -> Prebound:
+    """Marshal ``fn(*args, **kwargs)`` (any function of this module, or a callable that makes several
+    such calls) once and return a ``Prebound`` that replays the C call(s).  Tensors and trees passed in
+    are kept alive by the returned object; the stream is the one current (or passed) at this time."""
+    global _recording
+    assert _recording is None, "prebound() does not nest"
+    _recording = []
+    try:
+        fn(*args, **kwargs)
+        calls = _recording
+    finally:
+        _recording = None
+    return Prebound(calls, (args, kwargs))
 
 
 @dataclass
@@ -167,8 +217,7 @@ def treewy_tree_prepare(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tenso
                         stream=None) -> None:
     lib = load_library()
     ts = tree.struct()
-    _check("treewy_tree_prepare",
-           lib.treewy_tree_prepare(ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream)))
+    _call("treewy_tree_prepare", lib.treewy_tree_prepare, ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream))
 
 
 def treewy_tree_prepare_log(tree: Tree, log_alpha: torch.Tensor, seq_status: torch.Tensor | None = None,
@@ -176,8 +225,7 @@ def treewy_tree_prepare_log(tree: Tree, log_alpha: torch.Tensor, seq_status: tor
     """As treewy_tree_prepare, with the gates given as logarithms (log alpha <= 0)."""
     lib = load_library()
     ts = tree.struct()
-    _check("treewy_tree_prepare_log",
-           lib.treewy_tree_prepare_log(ctypes.byref(ts), _p(log_alpha), _p(seq_status), _stream(stream)))
+    _call("treewy_tree_prepare_log", lib.treewy_tree_prepare_log, ctypes.byref(ts), _p(log_alpha), _p(seq_status), _stream(stream))
 
 
 def _pool(states: torch.Tensor, state_index: torch.Tensor) -> PoolStruct:
@@ -190,9 +238,8 @@ def treewy_verify_pool(states, state_index, q, k, v, beta, tree: Tree, H_qk: int
     """treewy_verify with sequence b's state at states[state_index[b]] (block-pool addressing)."""
     lib = load_library()
     ts, ps = tree.struct(), _pool(states, state_index)
-    _check("treewy_verify_pool",
-           lib.treewy_verify_pool(ctypes.byref(ps), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), H_qk,
-                                  _DTYPES[states.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream)))
+    _call("treewy_verify_pool", lib.treewy_verify_pool, ctypes.byref(ps), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), H_qk,
+                                  _DTYPES[states.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream))
 
 
 def treewy_commit_pool(states, state_index, U, k, tree: Tree, H_qk: int, accepted: torch.Tensor,
@@ -200,9 +247,8 @@ def treewy_commit_pool(states, state_index, U, k, tree: Tree, H_qk: int, accepte
     """treewy_commit, in place, with sequence b's state at states[state_index[b]]."""
     lib = load_library()
     ts, ps = tree.struct(), _pool(states, state_index)
-    _check("treewy_commit_pool",
-           lib.treewy_commit_pool(ctypes.byref(ps), _p(U), _p(k), ctypes.byref(ts), H_qk, _p(accepted),
-                                  _DTYPES[states.dtype], _p(seq_status), _stream(stream)))
+    _call("treewy_commit_pool", lib.treewy_commit_pool, ctypes.byref(ps), _p(U), _p(k), ctypes.byref(ts), H_qk, _p(accepted),
+                                  _DTYPES[states.dtype], _p(seq_status), _stream(stream))
 
 
 def treewy_verify(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,
@@ -212,9 +258,8 @@ def treewy_verify(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: 
     ts = tree.struct()
     fn = lib.treewy_verify_generic if generic else lib.treewy_verify
     assert q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
-    _check("treewy_verify",
-           fn(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
-              _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream)))
+    _call("treewy_verify_generic" if generic else "treewy_verify", fn, _p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+              _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status), _stream(stream))
 
 
 def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
@@ -222,9 +267,8 @@ def treewy_commit(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Te
     """S0 is updated in place; S_out_f32, when given, also receives the unrounded state."""
     lib = load_library()
     ts = tree.struct()
-    _check("treewy_commit",
-           lib.treewy_commit(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
-                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+    _call("treewy_commit", lib.treewy_commit, _p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream))
 
 
 def treewy_verify_half_u(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U16: torch.Tensor,
@@ -233,10 +277,9 @@ def treewy_verify_half_u(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tens
     lib = load_library()
     ts = tree.struct()
     assert U16.dtype == torch.float16 and q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
-    _check("treewy_verify_half_u",
-           lib.treewy_verify_half_u(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+    _call("treewy_verify_half_u", lib.treewy_verify_half_u, _p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
                                     _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U16), _p(seq_status),
-                                    _stream(stream)))
+                                    _stream(stream))
 
 
 def treewy_commit_half_u(S0, U16, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
@@ -245,34 +288,30 @@ def treewy_commit_half_u(S0, U16, k, tree: Tree, H_qk: int, accepted, S_out_f32:
     lib = load_library()
     ts = tree.struct()
     assert U16.dtype == torch.float16
-    _check("treewy_commit_half_u",
-           lib.treewy_commit_half_u(_p(S0), _p(U16), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
-                                    _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+    _call("treewy_commit_half_u", lib.treewy_commit_half_u, _p(S0), _p(U16), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                                    _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream))
 
 
 def treewy_tree_prepare_wide(tree: Tree, alpha: torch.Tensor, seq_status: torch.Tensor | None = None, stream=None) -> None:
     """treewy_tree_prepare for trees of up to 128 nodes (no ancestor masks are written)."""
     ts = tree.struct()
-    _check("treewy_tree_prepare_wide",
-           load_library().treewy_tree_prepare_wide(ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream)))
+    _call("treewy_tree_prepare_wide", load_library().treewy_tree_prepare_wide, ctypes.byref(ts), _p(alpha), _p(seq_status), _stream(stream))
 
 
 def treewy_verify_wide(S0, q, k, v, beta, tree: Tree, H_qk: int, O: torch.Tensor, U: torch.Tensor,
                        seq_status: torch.Tensor | None = None, stream=None) -> None:
     ts = tree.struct()
     assert q.dtype == S0.dtype and k.dtype == S0.dtype and v.dtype == S0.dtype
-    _check("treewy_verify_wide",
-           load_library().treewy_verify_wide(_p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
+    _call("treewy_verify_wide", load_library().treewy_verify_wide, _p(S0), _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
                                              _DTYPES[S0.dtype], _DTYPES[O.dtype], _p(O), _p(U), _p(seq_status),
-                                             _stream(stream)))
+                                             _stream(stream))
 
 
 def treewy_commit_wide(S0, U, k, tree: Tree, H_qk: int, accepted, S_out_f32: torch.Tensor | None = None,
                        seq_status: torch.Tensor | None = None, stream=None) -> None:
     ts = tree.struct()
-    _check("treewy_commit_wide",
-           load_library().treewy_commit_wide(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
-                                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream)))
+    _call("treewy_commit_wide", load_library().treewy_commit_wide, _p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _p(accepted),
+                                             _DTYPES[S0.dtype], _p(S_out_f32), _p(seq_status), _stream(stream))
 
 
 def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta, tree: Tree,
@@ -282,11 +321,10 @@ def treewy_commit_verify(S0, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, 
     kernels, or (single_kernel) the fused kernel that reads and writes the state once."""
     lib = load_library()
     tp, ts = tree_prev.struct(), tree.struct()
-    _check("treewy_commit_verify",
-           lib.treewy_commit_verify(_p(S0), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev), _p(q),
+    _call("treewy_commit_verify", lib.treewy_commit_verify, _p(S0), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev), _p(q),
                                     _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
                                     _DTYPES[O.dtype], _p(O), _p(U), int(bool(single_kernel)), _p(seq_status),
-                                    _stream(stream)))
+                                    _stream(stream))
 
 
 def treewy_commit_verify_pool(states, state_index, U_prev, k_prev, tree_prev: Tree, accepted_prev, q, k, v, beta,
@@ -295,11 +333,10 @@ def treewy_commit_verify_pool(states, state_index, U_prev, k_prev, tree_prev: Tr
     """treewy_commit_verify with sequence b's state at states[state_index[b]]."""
     lib = load_library()
     tp, ts, ps = tree_prev.struct(), tree.struct(), _pool(states, state_index)
-    _check("treewy_commit_verify_pool",
-           lib.treewy_commit_verify_pool(ctypes.byref(ps), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev),
+    _call("treewy_commit_verify_pool", lib.treewy_commit_verify_pool, ctypes.byref(ps), _p(U_prev), _p(k_prev), ctypes.byref(tp), _p(accepted_prev),
                                          _p(q), _p(k), _p(v), _p(beta), ctypes.byref(ts), int(H_qk),
                                          _DTYPES[states.dtype], _DTYPES[O.dtype], _p(O), _p(U),
-                                         int(bool(single_kernel)), _p(seq_status), _stream(stream)))
+                                         int(bool(single_kernel)), _p(seq_status), _stream(stream))
 
 
 def treewy_snapshot_all(S0, U, k, tree: Tree, H_qk: int, Snap: torch.Tensor,
@@ -307,9 +344,8 @@ def treewy_snapshot_all(S0, U, k, tree: Tree, H_qk: int, Snap: torch.Tensor,
     """Every node's state into Snap [T, H_v, 128, 128] (the snapshotting comparator); S0 is read only."""
     lib = load_library()
     ts = tree.struct()
-    _check("treewy_snapshot_all",
-           lib.treewy_snapshot_all(_p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
-                                   _p(Snap), _p(seq_status), _stream(stream)))
+    _call("treewy_snapshot_all", lib.treewy_snapshot_all, _p(S0), _p(U), _p(k), ctypes.byref(ts), int(H_qk), _DTYPES[S0.dtype],
+                                   _p(Snap), _p(seq_status), _stream(stream))
 
 
 # --------------------------------------------------------------------------- user-level step

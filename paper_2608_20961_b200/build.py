@@ -1,18 +1,24 @@
-"""Builds libtreewy.so in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
+"""Builds libtreewy.so in-tree with nvcc for sm_100a (cross-compiles without a GPU).
+
+Every ``csrc/*.cu`` is compiled to an object file of its own (in parallel, and only when it or a
+header changed), then the objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
+OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libtreewy.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -20,28 +26,53 @@ def sources() -> list[str]:
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + \
+def _headers() -> list[str]:
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + \
         glob.glob(os.path.join(PKG, "..", "include", "*.h")) + [os.path.abspath(__file__)]
-    return any(os.path.getmtime(d) > t for d in deps)
+
+
+def _obj(src: str) -> str:
+    return os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+
+
+def _newer(path: str, than: list[str]) -> bool:
+    if not os.path.exists(path):
+        return False
+    t = os.path.getmtime(path)
+    return all(os.path.getmtime(d) <= t for d in than)
+
+
+def is_stale() -> bool:
+    return not _newer(LIB, sources() + _headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
-    if verbose:
-        flags += ["-Xptxas", "-v"]
-    cmd = [nvcc, *flags, *sources(), "-o", LIB]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libtreewy.so")
+    os.makedirs(OBJ, exist_ok=True)
+    flags = NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else [])
+    hdrs = _headers()
+
+    def compile_one(src: str):
+        if not force and _newer(_obj(src), [src] + hdrs):
+            return None
+        return subprocess.run([nvcc, *flags, "-c", src, "-o", _obj(src)], capture_output=True, text=True)
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        results = list(pool.map(compile_one, sources()))
+    failed = False
+    for res in results:
+        if res is not None and (verbose or res.returncode != 0):
+            sys.stderr.write(res.stdout + res.stderr)
+        failed |= res is not None and res.returncode != 0
+    if failed:
+        raise RuntimeError("nvcc failed compiling libtreewy's sources")
+    link = subprocess.run([nvcc, "-shared", "-cudart", "static", *[_obj(s) for s in sources()], "-o", LIB],
+                          capture_output=True, text=True)
+    if link.returncode != 0:
+        sys.stderr.write(link.stdout + link.stderr)
+        raise RuntimeError("linking libtreewy.so failed")
     return LIB
 
 

@@ -4,6 +4,12 @@
 
 using namespace treewy;
 
+treewy::DebugInject &treewy::debug_inject()
+{
+    static DebugInject d;
+    return d;
+}
+
 namespace {
 
 inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
@@ -44,13 +50,17 @@ treewy_status_t check_pool(const treewy_state_pool_t *pool, StateView *out)
     return TREEWY_OK;
 }
 
-treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, const void *k,
-                              const void *v, const float *beta, const treewy_tree_t *tree,
-                              int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype,
-                              void *O, void *U, bool u_half, int32_t *seq_status, void *cuda_stream)
+// Every host-side check of a verify call, and its argument block.  *run is false when the call is
+// valid but has nothing to do (no sequences or no nodes).  Nothing is launched here, so a call made
+// of two kernels can check both halves before it enqueues the first.
+treewy_status_t verify_check(StateView sv, const void *q, const void *k, const void *v, const float *beta,
+                             const treewy_tree_t *tree, int32_t H_qk, treewy_dtype_t io_dtype,
+                             treewy_dtype_t o_dtype, void *O, void *U, bool u_half, int32_t *seq_status,
+                             VerifyArgs *out, bool *run)
 {
     const void *S0 = sv.states;
     int max_nodes = 0;
+    *run = false;
     treewy_status_t st = check_tree(tree, true, &max_nodes);
     if (st != TREEWY_OK) return st;
     if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
@@ -61,21 +71,84 @@ treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, c
         bad_ptr(U))
         return TREEWY_ERR_INVALID_ARG;
 
-    VerifyArgs a;
+    VerifyArgs a = {};
     a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
     a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.u_half = u_half ? 1 : 0, a.seq_status = seq_status;
-    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes, a.T = tree->T;
     a.state_index = sv.index, a.n_states = sv.n_states;
     a.cls_lo = 0, a.cls_hi = max_nodes;
+    a.wait_cycles = debug_inject().wait_cycles, a.skip_item = debug_inject().skip_item;
+    *out = a, *run = true;
+    return TREEWY_OK;
+}
+
+treewy_status_t verify_launch(const VerifyArgs &a, bool force_generic, treewy_dtype_t io_dtype,
+                              treewy_dtype_t o_dtype, void *cuda_stream)
+{
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
     if (io_dtype == TREEWY_BF16 && !force_generic)
-        e = launch_verify_sm100(a, tree->T, o_dtype, stream);
+        e = launch_verify_sm100(a, a.T, o_dtype, stream);
     else
         e = launch_verify_generic(a, io_dtype, o_dtype, stream);
+    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
+}
+
+treewy_status_t verify_common(bool force_generic, StateView sv, const void *q, const void *k,
+                              const void *v, const float *beta, const treewy_tree_t *tree,
+                              int32_t H_qk, treewy_dtype_t io_dtype, treewy_dtype_t o_dtype,
+                              void *O, void *U, bool u_half, int32_t *seq_status, void *cuda_stream)
+{
+    VerifyArgs a;
+    bool run = false;
+    treewy_status_t st = verify_check(sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, u_half, seq_status, &a, &run);
+    if (st != TREEWY_OK || !run) return st;
+    return verify_launch(a, force_generic, io_dtype, o_dtype, cuda_stream);
+}
+
+// The same split for commit.
+treewy_status_t commit_check(StateView sv, const void *U, bool u_half, const void *k, const treewy_tree_t *tree,
+                             int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype, float *S_out_f32,
+                             int32_t *seq_status, CommitArgs *out, bool *run)
+{
+    void *S0 = sv.states;
+    int max_nodes = 0;
+    *run = false;
+    treewy_status_t st = check_tree(tree, true, &max_nodes);
+    if (st != TREEWY_OK) return st;
+    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
+    if (bad_dtype(io_dtype)) return TREEWY_ERR_UNSUPPORTED;
+    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
+    if (S_out_f32 && misaligned(S_out_f32)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->B == 0) return TREEWY_OK;
+    if (bad_ptr(S0) || bad_ptr(accepted)) return TREEWY_ERR_INVALID_ARG;
+    if (tree->T > 0 && (bad_ptr(U) || bad_ptr(k))) return TREEWY_ERR_INVALID_ARG;
+
+    CommitArgs a = {};
+    a.S0 = S0, a.U = U, a.u_half = u_half ? 1 : 0, a.k = k;
+    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
+    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
+    a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
+    a.snap_out = nullptr, a.T = tree->T;
+    a.state_index = sv.index, a.n_states = sv.n_states;
+    a.wait_cycles = debug_inject().wait_cycles;
+    *out = a, *run = true;
+    return TREEWY_OK;
+}
+
+treewy_status_t commit_common(StateView sv, const void *U, bool u_half, const void *k, const treewy_tree_t *tree,
+                              int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype, float *S_out_f32,
+                              int32_t *seq_status, void *cuda_stream)
+{
+    CommitArgs a;
+    bool run = false;
+    treewy_status_t st = commit_check(sv, U, u_half, k, tree, H_qk, accepted, io_dtype, S_out_f32, seq_status, &a, &run);
+    if (st != TREEWY_OK || !run) return st;
+    cudaError_t e = launch_commit(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 
@@ -125,34 +198,6 @@ treewy_status_t treewy_verify_generic(const void *S0, const void *q, const void 
 {
     return verify_common(true, plain_view(S0, tree ? tree->B : 0), q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O,
                          U, false, seq_status, cuda_stream);
-}
-
-static treewy_status_t commit_common(StateView sv, const void *U, bool u_half, const void *k, const treewy_tree_t *tree,
-                                     int32_t H_qk, const int32_t *accepted, treewy_dtype_t io_dtype,
-                                     float *S_out_f32, int32_t *seq_status, void *cuda_stream)
-{
-    void *S0 = sv.states;
-    int max_nodes = 0;
-    treewy_status_t st = check_tree(tree, true, &max_nodes);
-    if (st != TREEWY_OK) return st;
-    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
-    if (bad_dtype(io_dtype)) return TREEWY_ERR_UNSUPPORTED;
-    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
-    if (S_out_f32 && misaligned(S_out_f32)) return TREEWY_ERR_INVALID_ARG;
-    if (tree->B == 0) return TREEWY_OK;
-    if (bad_ptr(S0) || bad_ptr(accepted)) return TREEWY_ERR_INVALID_ARG;
-    if (tree->T > 0 && (bad_ptr(U) || bad_ptr(k))) return TREEWY_ERR_INVALID_ARG;
-
-    CommitArgs a;
-    a.S0 = S0, a.U = U, a.u_half = u_half ? 1 : 0, a.k = k;
-    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
-    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
-    a.accepted = accepted, a.S_out_f32 = S_out_f32, a.seq_status = seq_status;
-    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
-    a.snap_out = nullptr, a.T = tree->T;
-    a.state_index = sv.index, a.n_states = sv.n_states;
-    cudaError_t e = launch_commit(a, io_dtype, static_cast<cudaStream_t>(cuda_stream));
-    return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
 
 treewy_status_t treewy_commit(void *S0, const float *U, const void *k, const treewy_tree_t *tree,
@@ -224,8 +269,8 @@ treewy_status_t treewy_verify_wide(const void *S0, const void *q, const void *k,
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.cum_log_gate = tree->cum_log_gate, a.depth = tree->depth, a.level_order = tree->level_order;
     a.O = O, a.U = U, a.u_half = 0, a.seq_status = seq_status;
-    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
-    a.n_states = tree->B, a.cls_lo = 0, a.cls_hi = max_nodes;
+    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes, a.T = tree->T;
+    a.n_states = tree->B, a.cls_lo = 0, a.cls_hi = max_nodes, a.skip_item = -1;
     cudaError_t e = launch_verify_wide(a, io_dtype, o_dtype, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
@@ -288,7 +333,7 @@ treewy_status_t treewy_snapshot_all(const void *S0, const float *U, const void *
     if (tree->B == 0 || tree->T == 0) return TREEWY_OK;
     if (bad_ptr(S0) || bad_ptr(U) || bad_ptr(k) || bad_ptr(Snap)) return TREEWY_ERR_INVALID_ARG;
 
-    CommitArgs a;
+    CommitArgs a = {};
     a.S0 = const_cast<void *>(S0), a.U = U, a.u_half = 0, a.k = k;
     a.node_offsets = tree->node_offsets, a.parent = tree->parent;
     a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
@@ -307,7 +352,6 @@ static treewy_status_t commit_verify_common(StateView sv, const float *U_prev, c
                                             treewy_dtype_t o_dtype, void *O, float *U, int32_t single_kernel,
                                             int32_t *seq_status, void *cuda_stream)
 {
-    void *S0 = sv.states;
     int max_prev = 0, max_nodes = 0;
     treewy_status_t st = check_tree(tree_prev, true, &max_prev);
     if (st != TREEWY_OK) return st;
@@ -315,33 +359,28 @@ static treewy_status_t commit_verify_common(StateView sv, const float *U_prev, c
     if (st != TREEWY_OK) return st;
     if (tree_prev->B != tree->B || tree_prev->H_v != tree->H_v) return TREEWY_ERR_INVALID_ARG;
     const bool fusable = single_kernel != 0 && io_dtype == TREEWY_BF16 && max_nodes <= 32 && tree->B > 0 && tree->T > 0 && tree_prev->T > 0;
-    if (!fusable) {  // same result from the two stand-alone kernels
-        st = commit_common(sv, U_prev, false, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status,
-                           cuda_stream);
-        if (st != TREEWY_OK) return st;
-        return verify_common(false, sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, false, seq_status, cuda_stream);
-    }
-    if (H_qk < 1 || tree->H_v % H_qk != 0) return TREEWY_ERR_INVALID_ARG;
-    if (bad_dtype(o_dtype)) return TREEWY_ERR_UNSUPPORTED;
-    if (seq_status && misaligned(seq_status)) return TREEWY_ERR_INVALID_ARG;
-    if (bad_ptr(S0) || bad_ptr(U_prev) || bad_ptr(k_prev) || bad_ptr(accepted_prev) || bad_ptr(q) || bad_ptr(k) ||
-        bad_ptr(v) || bad_ptr(beta) || bad_ptr(O) || bad_ptr(U))
-        return TREEWY_ERR_INVALID_ARG;
-
+    // every check of both halves comes before the first launch: a call that is going to fail must not
+    // have committed already
+    CommitArgs ca;
     VerifyArgs a;
-    a.S0 = S0, a.q = q, a.k = k, a.v = v, a.beta = beta;
-    a.node_offsets = tree->node_offsets, a.parent = tree->parent;
-    a.anc_mask = tree->anc_mask, a.cum_log_gate = tree->cum_log_gate;
-    a.depth = tree->depth, a.level_order = tree->level_order;
-    a.O = O, a.U = U, a.u_half = 0, a.seq_status = seq_status;
-    a.B = tree->B, a.H_v = tree->H_v, a.H_qk = H_qk, a.max_nodes = max_nodes;
-    a.state_index = sv.index, a.n_states = sv.n_states;
-    a.cls_lo = 0, a.cls_hi = max_nodes;
+    bool run_commit = false, run_verify = false;
+    st = commit_check(sv, U_prev, false, k_prev, tree_prev, H_qk, accepted_prev, io_dtype, nullptr, seq_status, &ca,
+                      &run_commit);
+    if (st != TREEWY_OK) return st;
+    st = verify_check(sv, q, k, v, beta, tree, H_qk, io_dtype, o_dtype, O, U, false, seq_status, &a, &run_verify);
+    if (st != TREEWY_OK) return st;
+    if (!fusable) {  // same result from the two stand-alone kernels
+        if (run_commit) {
+            cudaError_t e = launch_commit(ca, io_dtype, static_cast<cudaStream_t>(cuda_stream));
+            if (e != cudaSuccess) return TREEWY_ERR_CUDA;
+        }
+        return run_verify ? verify_launch(a, false, io_dtype, o_dtype, cuda_stream) : TREEWY_OK;
+    }
     PrevRound pv;
     pv.U = U_prev, pv.k = k_prev;
     pv.node_offsets = tree_prev->node_offsets, pv.parent = tree_prev->parent;
     pv.anc_mask = tree_prev->anc_mask, pv.cum_log_gate = tree_prev->cum_log_gate;
-    pv.accepted = accepted_prev, pv.max_nodes = max_prev;
+    pv.accepted = accepted_prev, pv.max_nodes = max_prev, pv.T = tree_prev->T;
     cudaError_t e = launch_commit_verify_sm100(a, pv, tree->T, o_dtype, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TREEWY_OK : TREEWY_ERR_CUDA;
 }
@@ -368,6 +407,12 @@ treewy_status_t treewy_commit_verify_pool(const treewy_state_pool_t *pool, const
     if (st != TREEWY_OK) return st;
     return commit_verify_common(sv, U_prev, k_prev, tree_prev, accepted_prev, q, k, v, beta, tree, H_qk, io_dtype,
                                 o_dtype, O, U, single_kernel, seq_status, cuda_stream);
+}
+
+void treewy_debug_inject(int64_t wait_cycles, int32_t skip_item)
+{
+    debug_inject().wait_cycles = wait_cycles > 0 ? wait_cycles : 0;
+    debug_inject().skip_item = skip_item;
 }
 
 const char *treewy_status_string(treewy_status_t status)

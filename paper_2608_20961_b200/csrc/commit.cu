@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(CM_THREADS) commit_kernel(CommitArgs a)
 
     if (tid == 0) s_bad = 0;
     __syncthreads();
-    int bad = validate_sequence(a.parent, lo, n, a.max_nodes, &s_bad);
+    int bad = validate_sequence(a.parent, lo, n, a.T, a.max_nodes, &s_bad);
     if (!bad && (acc_node < -1 || acc_node >= n)) bad = TREEWY_SEQ_BAD_ACCEPTED;
     if (slot < 0) bad = TREEWY_SEQ_BAD_STATE;
     if (bad) {

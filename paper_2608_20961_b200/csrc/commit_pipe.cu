@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         ptx::fence_barrier_init();
     }
     grid_dependency_wait();  // the kernel before this one on the stream has finished: global memory may be read
+    if (tid == 0) ptx::wait_deadline_init(a.wait_cycles);
     __syncthreads();
     grid_dependency_trigger();
 
@@ -104,6 +105,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             int bad = 0;
             if (slot < 0) {
                 bad = TREEWY_SEQ_BAD_STATE;
+            } else if (bad_offsets(lo, n, a.T)) {
+                bad = TREEWY_SEQ_BAD_OFFSETS;
             } else if (n < 1 || n > a.max_nodes) {
                 bad = TREEWY_SEQ_TOO_MANY_NODES;
             } else {
@@ -277,12 +280,10 @@ cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream)
     const long long n_items = (long long)(a.snap_out ? a.T : a.B) * a.H_v;
     if (n_items == 0) return cudaSuccess;
     int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = current_device_sms(&dev, &sms);
     if (e != cudaSuccess) return e;
     const int smem = (int)sizeof(CommitPipeSmem);
-    e = cudaFuncSetAttribute(commit_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = ensure_dynamic_smem(reinterpret_cast<const void *>(commit_pipe_kernel), smem, dev);
     if (e != cudaSuccess) return e;
     const int grid = (int)(n_items < sms ? n_items : sms);
     return launch_dependent(commit_pipe_kernel, dim3(grid), dim3(CP_THREADS), smem, stream, a, (int)n_items);

@@ -17,7 +17,7 @@ constexpr int PREP_THREADS = 128;
 constexpr int PREP_HCHUNK = 16;  // value heads per CTA
 
 __global__ void __launch_bounds__(PREP_THREADS)
-prepare_kernel(int B, int H_v, int max_nodes, int gates_are_logs, const int32_t *__restrict__ node_offsets,
+prepare_kernel(int B, int T, int H_v, int max_nodes, int gates_are_logs, const int32_t *__restrict__ node_offsets,
                const int32_t *__restrict__ parent, const float *__restrict__ alpha,
                int32_t *__restrict__ depth, uint64_t *__restrict__ anc_mask,
                float *__restrict__ cum_log_gate, uint8_t *__restrict__ level_order,
@@ -38,7 +38,7 @@ prepare_kernel(int B, int H_v, int max_nodes, int gates_are_logs, const int32_t 
     const int n = node_offsets[b + 1] - lo;
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
-    const int bad = validate_sequence(parent, lo, n, max_nodes, &s_bad);
+    const int bad = validate_sequence(parent, lo, n, T, max_nodes, &s_bad);
     if (bad) {
         if (threadIdx.x == 0 && blockIdx.y == 0 && seq_status) atomicOr(&seq_status[b], bad);
         return;
@@ -93,7 +93,7 @@ cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *a
 {
     if (t.B == 0) return cudaSuccess;
     const dim3 grid(t.B, (t.H_v + PREP_HCHUNK - 1) / PREP_HCHUNK);
-    return launch_dependent(prepare_kernel, grid, dim3(PREP_THREADS), 0, stream, t.B, t.H_v, max_nodes,
+    return launch_dependent(prepare_kernel, grid, dim3(PREP_THREADS), 0, stream, t.B, t.T, t.H_v, max_nodes,
                             gates_are_logs ? 1 : 0, t.node_offsets, t.parent, alpha, t.depth, t.anc_mask,
                             t.cum_log_gate, t.level_order, seq_status);
 }

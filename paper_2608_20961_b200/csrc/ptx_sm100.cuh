@@ -3,7 +3,7 @@
 // tiled tensor-map forms, never with cluster multicast), the async-proxy fence, and the
 // tcgen05 tensor-core / tensor-memory instructions.
 //
-// Every wait is bounded: a barrier that does not flip within the limit makes the wait
+// Every wait is bounded: a barrier that does not flip before the kernel's deadline makes the wait
 // return false, so a kernel can raise a status bit and leave instead of hanging the GPU.
 #pragma once
 
@@ -63,16 +63,25 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint64_t *bar, uint32_t par
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the phase did not complete within about two seconds of SM clocks,
-// so a kernel can raise a status bit and leave instead of hanging the GPU.
-// (the slow path is kept out of line: the kernels wait in dozens of places and their code has to
-// stay small enough for the instruction cache)
+// Bounded waits.  A kernel sets ONE deadline when it starts (wait_deadline_init, by one thread, ahead of
+// the CTA's first barrier): every wait of every role gives up once the SM's clock has passed it, so a
+// kernel that cannot make progress costs the limit once, not once per waiting role, and returns with
+// a status bit instead of hanging the GPU.  The default limit is about two seconds of SM clocks,
+// three orders of magnitude above the longest kernel the library runs.
+// (The deadline lives in static shared memory and the slow path is kept out of line: the kernels
+// wait in dozens of places and their code has to stay small enough for the instruction cache.)
+constexpr long long WAIT_CYCLES_DEFAULT = 4000000000ll;
+static __shared__ long long s_wait_deadline;
+__device__ __forceinline__ void wait_deadline_init(long long cycles)
+{
+    s_wait_deadline = clock64() + (cycles > 0 ? cycles : WAIT_CYCLES_DEFAULT);
+}
+__device__ __forceinline__ bool wait_deadline_passed() { return clock64() > s_wait_deadline; }
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity)
 {
-    const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
-        if (clock64() - t0 > 4000000000ll) return false;
+        if (wait_deadline_passed()) return false;
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/treewy.h"
 
 namespace treewy {
@@ -34,6 +36,43 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr, cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Host side of a launch, kept off the per-call path: the SM count of a device and the raised dynamic
+// shared-memory limit of a kernel are looked up / set once per device and process (on a batch of a
+// few dozen microseconds of GPU work, three runtime calls per launch are a visible part of the step).
+inline cudaError_t current_device_sms(int *dev, int *sms)
+{
+    static std::atomic<int> cache[64];
+    cudaError_t e = cudaGetDevice(dev);
+    if (e != cudaSuccess) return e;
+    const bool cached = *dev >= 0 && *dev < 64;
+    if (cached && (*sms = cache[*dev].load(std::memory_order_relaxed)) > 0) return cudaSuccess;
+    e = cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, *dev);
+    if (e == cudaSuccess && cached) cache[*dev].store(*sms, std::memory_order_relaxed);
+    return e;
+}
+inline cudaError_t ensure_dynamic_smem(const void *kernel, int bytes, int dev)
+{
+    constexpr int SLOTS = 128;
+    static std::atomic<const void *> fn[SLOTS];
+    static std::atomic<unsigned long long> devs[SLOTS];
+    if (dev >= 0 && dev < 64) {
+        for (int i = 0; i < SLOTS; ++i) {
+            const void *f = fn[i].load(std::memory_order_acquire);
+            if (f == nullptr) {
+                const void *expected = nullptr;
+                if (fn[i].compare_exchange_strong(expected, kernel, std::memory_order_acq_rel)) f = kernel;
+                else f = expected;
+            }
+            if (f != kernel) continue;
+            if ((devs[i].load(std::memory_order_acquire) >> dev) & 1ull) return cudaSuccess;
+            const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e == cudaSuccess) devs[i].fetch_or(1ull << dev, std::memory_order_release);
+            return e;
+        }
+    }
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
@@ -136,12 +175,22 @@ __device__ __forceinline__ void st_global_if(__half *p, float v, bool on)
                  "r"((int)on));
 }
 
-// Status bits of sequence [lo, lo+n): node count in 1..max_nodes, parent[i] in -1..i-1.
+// Whether the packed range [lo, lo + n) of a sequence leaves the T packed nodes the caller declared
+// (a stale or non-monotone node_offsets array): such a sequence is flagged and skipped before any of
+// its rows is addressed.
+__device__ __forceinline__ bool bad_offsets(int lo, int n, int T)
+{
+    return lo < 0 || n < 0 || (long long)lo + n > (long long)T;
+}
+
+// Status bits of sequence [lo, lo+n) of T packed nodes: range inside the packed arrays, node count in
+// 1..max_nodes, parent[i] in -1..i-1.
 // Called by every thread of a CTA with the same arguments; `scratch` is one shared int the
 // caller zeroed before a barrier.  Returns the same value in every thread.
-__device__ __forceinline__ int validate_sequence(const int32_t *__restrict__ parent, int lo, int n,
+__device__ __forceinline__ int validate_sequence(const int32_t *__restrict__ parent, int lo, int n, int T,
                                                  int max_nodes, int *scratch)
 {
+    if (bad_offsets(lo, n, T)) return TREEWY_SEQ_BAD_OFFSETS;
     if (n < 1 || n > max_nodes) return TREEWY_SEQ_TOO_MANY_NODES;
     int bad = 0;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {

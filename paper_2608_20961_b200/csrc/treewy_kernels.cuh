@@ -21,6 +21,9 @@ struct VerifyArgs {
     int u_half;
     int32_t *seq_status;
     int B, H_v, H_qk, max_nodes;
+    int T;  // packed nodes: a sequence whose node range leaves 0..T is flagged and skipped
+    long long wait_cycles;  // limit of the kernel's bounded waits in SM clocks (0: the default, ~2 s)
+    int skip_item;          // test hook (treewy_debug_inject): the item whose loads are never issued, or -1
     // block-pool addressing: sequence b's state is states[state_index[b]] of n_states (NULL: state b of B)
     const int32_t *state_index;
     int n_states;
@@ -38,6 +41,7 @@ struct PrevRound {
     const float *cum_log_gate;
     const int32_t *accepted;
     int max_nodes;
+    int T;  // packed nodes of the previous round's trees
 };
 
 struct CommitArgs {
@@ -54,9 +58,17 @@ struct CommitArgs {
     int B, H_v, H_qk, max_nodes;
     void *snap_out;  // snapshot mode when not NULL: [T, H_v, 128, 128] states, one per node
     int T;
+    long long wait_cycles;  // as in VerifyArgs
     const int32_t *state_index;  // as in VerifyArgs
     int n_states;
 };
+
+// What treewy_debug_inject set (process-wide test hook; all zeros / -1 unless a test called it).
+struct DebugInject {
+    long long wait_cycles = 0;
+    int skip_item = -1;
+};
+DebugInject &debug_inject();
 
 cudaError_t launch_prepare(const treewy_tree_t &t, int max_nodes, const float *alpha, bool gates_are_logs,
                            int32_t *seq_status, cudaStream_t stream);

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(VG_THREADS) verify_generic_kernel(VerifyArgs a
     if (c == 0) s_bad = 0;
     __syncthreads();
     const int slot = state_slot(a.state_index, a.n_states, b);
-    const int bad = slot < 0 ? TREEWY_SEQ_BAD_STATE : validate_sequence(a.parent, lo, n, nmax, &s_bad);
+    const int bad = slot < 0 ? TREEWY_SEQ_BAD_STATE : validate_sequence(a.parent, lo, n, a.T, nmax, &s_bad);
     if (bad) {
         if (c == 0 && h == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
         return;

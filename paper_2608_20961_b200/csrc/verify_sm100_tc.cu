@@ -41,8 +41,9 @@
 // bound (a third of the instruction fetches missed) until the long loops were rolled and the slow
 // path of the waits went out of line.
 //
-// Every mbarrier wait is bounded; on give-up the role leaves its loop, TREEWY_SEQ_TIMEOUT is
-// raised, and the CTA still reaches the common exit where tensor memory is freed.
+// Every mbarrier wait is bounded by one deadline per kernel; once it has passed, every role's next
+// wait fails at once, the role leaves its loop, TREEWY_SEQ_TIMEOUT is raised, and the CTA still
+// reaches the common exit where tensor memory is freed.
 #include <cuda.h>
 
 #include <type_traits>
@@ -251,6 +252,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         ptx::tc_fence_before_sync();
     }
     grid_dependency_wait();  // the kernel before this one on the stream has finished: global memory may be read
+    if (tid == 0) ptx::wait_deadline_init(a.wait_cycles);
     __syncthreads();
     grid_dependency_trigger();
     ptx::tc_fence_after_sync();
@@ -269,9 +271,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (ku < K_all) {
                 const int unit = (int)blockIdx.x + ku * (int)gridDim.x;
                 const int b = (pair_mode ? 2 * unit : unit) / a.H_v;
-                const int n = a.node_offsets[b + 1] - a.node_offsets[b];
+                const int lo = a.node_offsets[b], n = a.node_offsets[b + 1] - lo;
                 // another class's well-formed sequence goes; whatever has to be flagged stays
-                keep = !(n >= 1 && n <= a.max_nodes && (n <= a.cls_lo || n > a.cls_hi || n > NP)) ||
+                keep = !(n >= 1 && n <= a.max_nodes && (n <= a.cls_lo || n > a.cls_hi || n > NP)) || bad_offsets(lo, n, a.T) ||
                        (a.cls_lo == 0 && state_slot(a.state_index, a.n_states, b) < 0);
             }
             const uint32_t bal = __ballot_sync(0xffffffffu, keep);
@@ -336,6 +338,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (slot < 0) {
                 p.bad = TREEWY_SEQ_BAD_STATE;
                 p.flag = a.cls_lo == 0;
+            } else if (bad_offsets(p.lo, p.n, a.T)) {
+                p.bad = TREEWY_SEQ_BAD_OFFSETS;
+                p.flag = a.cls_lo == 0;
             } else if (p.n < 1 || p.n > a.max_nodes) {
                 p.bad = TREEWY_SEQ_TOO_MANY_NODES;
                 p.flag = a.cls_lo == 0;
@@ -369,6 +374,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const int acc = pv.accepted[p.b];
                 if (slot < 0) {
                     p.pbad = TREEWY_SEQ_BAD_STATE;  // no state to commit into
+                } else if (bad_offsets(p.plo, pn, pv.T)) {
+                    p.pbad = TREEWY_SEQ_BAD_OFFSETS;
                 } else if (pn < 1 || pn > pv.max_nodes) {
                     p.pbad = TREEWY_SEQ_TOO_MANY_NODES;
                 } else {
@@ -398,6 +405,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
 #pragma unroll 1
         for (int kk = s;; kk += C::STAGES) {
             if (cur.item >= n_items) break;
+            if (cur.item == a.skip_item) {  // test hook: this item's loads and their arrival never happen
+                cur = fetch(kk + C::STAGES);
+                continue;
+            }
             const Pre p = cur;
             if (p.bad && p.flag && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
             if (FUSED && p.pbad && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.pbad);
@@ -572,6 +583,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     ok = ptx::mbar_wait(cmma_done, rounds & 1);
                     ++rounds;
                     ptx::tc_fence_after_sync();
+                }
+                if (!ok) {  // the product never finished: the tile keeps the old state, nothing is stored
+                    if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
+                    break;
                 }
                 // S[t][:] = g_a S[t][:] + C[t][:], sixteen columns at a time; the next sixteen columns of
                 // C are on their way from tensor memory while the current ones are worked on
@@ -1126,14 +1141,12 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     const long long n_tiles = a.state_index ? (long long)a.n_states * a.H_v : n_items;
     if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_tiles, T, a.H_v, a.H_qk, NP)) return cudaErrorInvalidValue;
     int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = current_device_sms(&dev, &sms);
     if (e != cudaSuccess) return e;
     const long long units = (a.H_v / a.H_qk) % 2 == 0 ? n_items / 2 : n_items;  // the kernel takes heads in pairs
     const int grid = (int)(units < sms ? units : sms);
     auto go = [&](auto kernel) {
-        cudaError_t e2 = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        cudaError_t e2 = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), C::SMEM_BYTES, dev);
         if (e2 != cudaSuccess) return e2;
         return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a, pv, (int)n_items, m.S0, m.Q,
                                 m.K, m.V);

@@ -124,6 +124,7 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
         ptx::tc_fence_before_sync();
     }
     grid_dependency_wait();  // the kernel before this one on the stream has finished: global memory may be read
+    if (tid == 0) ptx::wait_deadline_init(a.wait_cycles);
     __syncthreads();
     grid_dependency_trigger();
     ptx::tc_fence_after_sync();
@@ -156,6 +157,8 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
             p.srow = (slot < 0 ? 0 : slot) * a.H_v + p.h;
             if (slot < 0) {
                 p.bad = TREEWY_SEQ_BAD_STATE, p.flag = a.cls_lo == 0;
+            } else if (bad_offsets(p.lo, p.n, a.T)) {
+                p.bad = TREEWY_SEQ_BAD_OFFSETS, p.flag = a.cls_lo == 0;
             } else if (p.n < 1 || p.n > a.max_nodes) {
                 p.bad = TREEWY_SEQ_TOO_MANY_NODES, p.flag = a.cls_lo == 0;
             } else if (p.n <= a.cls_lo || p.n > a.cls_hi || p.n > VS_N) {
@@ -175,6 +178,8 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                 const int acc = pv.accepted[p.b];
                 if (slot < 0) {
                     p.pbad = TREEWY_SEQ_BAD_STATE;  // no state to commit into
+                } else if (bad_offsets(p.plo, pn, pv.T)) {
+                    p.pbad = TREEWY_SEQ_BAD_OFFSETS;
                 } else if (pn < 1 || pn > pv.max_nodes || pn > VS_N) {
                     p.pbad = TREEWY_SEQ_TOO_MANY_NODES;
                 } else {
@@ -263,9 +268,8 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
             bool ready = true;
             {
                 const volatile int *named = &meta->item;
-                const long long t0 = clock64();
                 while (*named != item) {
-                    if (clock64() - t0 > 4000000000ll) {
+                    if (ptx::wait_deadline_passed()) {
                         ready = false;
                         break;
                     }
@@ -498,12 +502,9 @@ cudaError_t launch_vs(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     if (!make_verify_maps(&m, a.S0, a.q, a.k, a.v, n_tiles, T, a.H_v, a.H_qk, VS_N)) return cudaErrorInvalidValue;
     using C = VsCfg<FUSED>;
     int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    cudaError_t e = current_device_sms(&dev, &sms);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(verify_small_kernel<TOut, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             C::SMEM_BYTES);
+    e = ensure_dynamic_smem(reinterpret_cast<const void *>(verify_small_kernel<TOut, FUSED>), C::SMEM_BYTES, dev);
     if (e != cudaSuccess) return e;
     const int grid = (int)(n_items < sms ? n_items : sms);
     return launch_dependent(verify_small_kernel<TOut, FUSED>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a, pv,

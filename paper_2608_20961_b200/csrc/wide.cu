@@ -26,22 +26,8 @@ namespace {
 constexpr int WN = TREEWY_MAX_NODES_WIDE;
 constexpr int WT = 128;  // threads of a verify / prepare CTA
 
-// status bits of sequence [lo, lo + n): every thread of the CTA calls it with the same arguments
-__device__ __forceinline__ int wide_validate(const int32_t *__restrict__ parent, int lo, int n, int max_nodes, int *scratch)
-{
-    if (n < 1 || n > max_nodes) return TREEWY_SEQ_TOO_MANY_NODES;
-    int bad = 0;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const int p = parent[lo + i];
-        if (p < -1 || p >= i) bad = 1;
-    }
-    if (bad) atomicOr(scratch, TREEWY_SEQ_BAD_PARENT);
-    __syncthreads();
-    return *scratch;
-}
-
 __global__ void __launch_bounds__(WT)
-prepare_wide_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ node_offsets,
+prepare_wide_kernel(int B, int T, int H_v, int max_nodes, const int32_t *__restrict__ node_offsets,
                     const int32_t *__restrict__ parent, const float *__restrict__ alpha, int32_t *__restrict__ depth,
                     float *__restrict__ cum_log_gate, uint8_t *__restrict__ level_order, int32_t *__restrict__ seq_status)
 {
@@ -53,7 +39,7 @@ prepare_wide_kernel(int B, int H_v, int max_nodes, const int32_t *__restrict__ n
     const int n = node_offsets[b + 1] - lo;
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
-    const int bad = wide_validate(parent, lo, n, max_nodes, &s_bad);
+    const int bad = validate_sequence(parent, lo, n, T, max_nodes, &s_bad);
     if (bad) {
         if (threadIdx.x == 0 && seq_status) atomicOr(&seq_status[b], bad);
         return;
@@ -116,7 +102,7 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
     const int n = a.node_offsets[b + 1] - lo;
     if (c == 0) sm.bad = 0;
     __syncthreads();
-    const int bad = wide_validate(a.parent, lo, n, a.max_nodes, &sm.bad);
+    const int bad = validate_sequence(a.parent, lo, n, a.T, a.max_nodes, &sm.bad);
     if (bad) {
         if (c == 0 && h == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
         return;
@@ -214,7 +200,7 @@ template <typename T> __global__ void __launch_bounds__(WC_THREADS) commit_wide_
     const int n = a.node_offsets[b + 1] - lo;
     if (tid == 0) s_bad = 0;
     __syncthreads();
-    int bad = wide_validate(a.parent, lo, n, a.max_nodes, &s_bad);
+    int bad = validate_sequence(a.parent, lo, n, a.T, a.max_nodes, &s_bad);
     const int acc_node = a.accepted[b];
     if (!bad && (acc_node < -1 || acc_node >= n)) bad = TREEWY_SEQ_BAD_ACCEPTED;
     if (bad) {
@@ -285,7 +271,7 @@ cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const flo
                                 cudaStream_t stream)
 {
     if (t.B == 0) return cudaSuccess;
-    prepare_wide_kernel<<<t.B, WT, 0, stream>>>(t.B, t.H_v, max_nodes, t.node_offsets, t.parent, alpha, t.depth,
+    prepare_wide_kernel<<<t.B, WT, 0, stream>>>(t.B, t.T, t.H_v, max_nodes, t.node_offsets, t.parent, alpha, t.depth,
                                                 t.cum_log_gate, t.level_order, seq_status);
     return cudaGetLastError();
 }

@@ -50,15 +50,6 @@ def max_over_ranks(value: float, device: torch.device | None = None) -> float:
     return float(t.item())
 
 
-def sum_over_ranks(value: float, device: torch.device | None = None) -> float:
-    if not dist.is_initialized():
-        return float(value)
-    t = torch.tensor([float(value)], dtype=torch.float64,
-                     device=device if device is not None else "cpu")
-    dist.all_reduce(t, op=dist.ReduceOp.SUM)
-    return float(t.item())
-
-
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

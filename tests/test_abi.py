@@ -95,6 +95,35 @@ def test_argument_errors_are_reported_before_any_launch(tw):
                              None) == tw.TREEWY_OK
 
 
+def test_commit_verify_checks_both_halves_before_it_launches_anything(tw):
+    """The two-kernel form of treewy_commit_verify must not have committed when the verify half is going
+    to be rejected: with no GPU here a launch would show up as TREEWY_ERR_CUDA, a clean rejection as
+    TREEWY_ERR_INVALID_ARG / TREEWY_ERR_UNSUPPORTED."""
+    lib = tw.load_library()
+    vp = ctypes.c_void_p
+    tp, t = _tree(tw), _tree(tw)
+
+    def call(q=vp(A), o_dtype=tw.TREEWY_BF16, O=vp(A), single=0, tree=t, pool=None):
+        args = [vp(A), vp(A), ctypes.byref(tp), vp(A), q, vp(A), vp(A), vp(A), ctypes.byref(tree), 2,
+                tw.TREEWY_BF16, o_dtype, O, vp(A), single, None, None]
+        if pool is not None:
+            return lib.treewy_commit_verify_pool(ctypes.byref(pool), *args)
+        return lib.treewy_commit_verify(vp(A), *args)
+
+    for single in (0, 1):
+        assert call(q=None, single=single) == tw.TREEWY_ERR_INVALID_ARG
+        assert call(O=vp(A + 2), single=single) == tw.TREEWY_ERR_INVALID_ARG
+        assert call(o_dtype=5, single=single) == tw.TREEWY_ERR_UNSUPPORTED
+        assert call(tree=_tree(tw, B=3), single=single) == tw.TREEWY_ERR_INVALID_ARG   # B differs between the rounds
+    pool = tw.PoolStruct(A, A, 4)
+    assert call(q=None, pool=pool) == tw.TREEWY_ERR_INVALID_ARG
+
+
+def test_debug_hook_is_exported_and_resets(tw):
+    tw.treewy_debug_inject(1000, 3)
+    tw.treewy_debug_inject(0, -1)
+
+
 def test_missing_library_fails_loudly(tw, tmp_path):
     with pytest.raises(ImportError):
         tw.load_library(str(tmp_path / "libtreewy.so"))

@@ -1,7 +1,8 @@
-"""The benchmark configurations at FULL size, in the launch configuration bench.py times:
-sampled sequences are compared with the oracle element by element, every node's tree outputs
-are checked through invariants, and every stored state is checked to be the rounding of the
-fp32 state."""
+"""The benchmark configurations at FULL size, in the launch configuration bench.py times: every
+sequence of configurations 1-4 is compared with the oracle element by element (the oracle does a
+whole configuration in a second or two), every node's tree outputs are also checked through
+invariants, and every stored state is checked to be the rounding of the fp32 state.  Only the
+128-node workload of the wide-tree calls is compared on sampled sequences."""
 import numpy as np
 import pytest
 import torch
@@ -18,17 +19,14 @@ def test_full_size_config(oracle, cid):
     gpu = pu.run_gpu(w, torch.float32, max_nodes=w.max_nodes)
     assert not gpu["status"].any()
     pu.assert_tree_invariants(w, gpu)
-    g = np.random.default_rng(cid)
-    seqs = sorted(set([0, w.B - 1] + g.integers(0, w.B, 4).tolist()))
-    if cid == 4:   # make sure every tree size of the ragged mix is sampled
-        sizes = (w.node_offsets[1:] - w.node_offsets[:-1]).tolist()
-        seqs = sorted(set(seqs + [sizes.index(s) for s in (1, 8, 16, 32, 64) if s in sizes]))
-    errs = pu.assert_parity_sampled(oracle, w, gpu, seqs)
-    print(f"config {cid} full size, sequences {seqs}: {errs}")
-    # whole batch: stored state is RNE(fp32 state); finite everywhere; untouched canaries none
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    errs = pu.assert_parity(w, gpu, tree_ref, ref)         # the whole batch, every output
+    print(f"config {cid} full size, all {w.B} sequences: {errs}")
+    # stored state is RNE(fp32 state); finite everywhere; no row of O or U left at its canary value
     assert torch.equal(gpu["S"], gpu["S32"].to(gpu["S"].dtype))
     assert torch.isfinite(gpu["O"]).all() and torch.isfinite(gpu["U"]).all()
     assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any()
+    assert not (gpu["O"] == gpu["canary"]).all(dim=-1).any()
 
 
 def test_full_size_bf16_outputs_match_rounded_fp32_outputs():
