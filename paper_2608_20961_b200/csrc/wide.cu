@@ -91,8 +91,10 @@ template <typename TIn> struct WideSmem {
     int bad;
 };
 
+// (deep_only: the tensor-core kernel takes every sequence whose deepest path has at most
+// WIDE_TC_MAX_DEPTH ancestors; this launch then serves the others and leaves those alone)
 template <typename TIn, typename TOut>
-__global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
+__global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a, int deep_only)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     WideSmem<TIn> &sm = *reinterpret_cast<WideSmem<TIn> *>(smem_raw);
@@ -107,13 +109,20 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
         if (c == 0 && h == 0 && a.seq_status) atomicOr(&a.seq_status[b], bad);
         return;
     }
+    for (int i = c; i < n; i += WT) sm.parent[i] = a.parent[lo + i];
+    if (deep_only) {
+        __syncthreads();
+        int d = 0;
+        if (c < n)
+            for (int p = sm.parent[c]; p >= 0; p = sm.parent[p]) ++d;
+        if (!__syncthreads_or(d > WIDE_TC_MAX_DEPTH)) return;
+    }
     const int hq = h / (a.H_v / a.H_qk);
     const TIn *qg = static_cast<const TIn *>(a.q), *kg = static_cast<const TIn *>(a.k), *vg = static_cast<const TIn *>(a.v);
     for (int i = 0; i < n; ++i) sm.kf[i][c] = kg[((size_t)(lo + i) * a.H_qk + hq) * D + c];
     for (int i = c; i < n; i += WT) {
         sm.L[i] = a.cum_log_gate[(size_t)(lo + i) * a.H_v + h];
         sm.beta[i] = a.beta[(size_t)(lo + i) * a.H_v + h];
-        sm.parent[i] = a.parent[lo + i];
     }
     float srow[D];  // row c of S0
     load_row128(static_cast<const TIn *>(a.S0) + ((size_t)b * a.H_v + h) * D * D + (size_t)c * D, srow);
@@ -276,12 +285,12 @@ cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const flo
     return cudaGetLastError();
 }
 
-template <typename TIn, typename TOut> static cudaError_t launch_vw(const VerifyArgs &a, cudaStream_t stream)
+template <typename TIn, typename TOut> static cudaError_t launch_vw(const VerifyArgs &a, int deep_only, cudaStream_t stream)
 {
     const int smem = (int)sizeof(WideSmem<TIn>);
     cudaError_t e = cudaFuncSetAttribute(verify_wide_kernel<TIn, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    verify_wide_kernel<TIn, TOut><<<dim3(a.H_v, a.B), WT, smem, stream>>>(a);
+    verify_wide_kernel<TIn, TOut><<<dim3(a.H_v, a.B), WT, smem, stream>>>(a, deep_only);
     return cudaGetLastError();
 }
 
@@ -289,8 +298,13 @@ cudaError_t launch_verify_wide(const VerifyArgs &a, treewy_dtype_t io, treewy_dt
 {
     if (a.B == 0 || a.H_v == 0) return cudaSuccess;
     if (io == TREEWY_F32)
-        return od == TREEWY_F32 ? launch_vw<float, float>(a, stream) : launch_vw<float, __nv_bfloat16>(a, stream);
-    return od == TREEWY_F32 ? launch_vw<__nv_bfloat16, float>(a, stream) : launch_vw<__nv_bfloat16, __nv_bfloat16>(a, stream);
+        return od == TREEWY_F32 ? launch_vw<float, float>(a, 0, stream) : launch_vw<float, __nv_bfloat16>(a, 0, stream);
+    // bf16: the tensor-core kernel for every sequence it takes (paths of up to WIDE_TC_MAX_DEPTH ancestors),
+    // the SIMT kernel for the deeper ones
+    cudaError_t e = od == TREEWY_F32 ? launch_vw<__nv_bfloat16, float>(a, 1, stream)
+                                     : launch_vw<__nv_bfloat16, __nv_bfloat16>(a, 1, stream);
+    if (e != cudaSuccess) return e;
+    return launch_verify_wide_tc(a, od, stream);
 }
 
 cudaError_t launch_commit_wide(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream)
