@@ -8,24 +8,31 @@
 // all three accumulated in tensor memory (256 + 128 + 128 = 512 columns: one item at a time).  A node
 // of such a tree has no 64-bit ancestor mask; the producer warp walks the parent array once per item
 // and hands over four-word masks, depths and the level order.  The triangular system itself is solved
-// on the CUDA cores, one thread per element c of d_v and four threads per c:
+// on the CUDA cores:
 //
 //   lists     the thread whose tensor-memory lane holds row i of a Gram block picks node i's ancestors
-//             out of it: A[i][d] = beta_i e^{L_i - L_j} k_i.k_j, P[i][d] = e^{L_i - L_j} q_i.k_j, j the
-//             ancestor of depth d (ancestors in index order are in depth order);
-//   r         r_i[c] = beta_i v_i[c] - beta_i g_i (S0 k_i)[c] into a [node][c] tile of shared memory;
-//   solve     level by level (nodes of one depth do not depend on each other and are shared out over
-//             the four thread groups):  u_i[c] = r_i[c] - sum_d A[i][d] u_{j_d}[c],
-//             o_i[c] = g_i (S0 q_i)[c] + sum_d P[i][d] u_{j_d}[c] + (q_i.k_i) u_i[c];  u_i replaces r_i in
-//             the tile, both leave for global memory at once.
+//             out of it (through a private line of shared memory, so that they can be taken by index):
+//             A[i][d] = beta_i e^{L_i - L_j} k_i.k_j, P[i][d] = e^{L_i - L_j} q_i.k_j, j the ancestor of
+//             depth d (ancestors in index order are in depth order);
+//   r, o0     thread c = tensor-memory lane c = element c of d_v:  r_i[c] = beta_i v_i[c] - beta_i g_i (S0 k_i)[c]
+//             and o0_i[c] = g_i (S0 q_i)[c] into two [node][c] tiles of shared memory; tensor memory is
+//             not needed after this;
+//   solve     level by level (nodes of one depth do not depend on each other): ONE WARP PER NODE, a lane
+//             holding four elements of d_v, so that the coefficients and indices, which are the same for
+//             all 128 elements, are fetched once per node and not once per 32 elements:
+//             u_i = r_i - sum_d A[i][d] u_{j_d},  o_i = o0_i + sum_d P[i][d] u_{j_d} + (q_i.k_i) u_i;
+//             u_i replaces r_i in its tile, both rows leave for global memory as 512 / 256 contiguous bytes.
+//             (A first version gave every node to four warps of 32 elements each: 37 k warp instructions
+//             and 20 k cycles per item in this phase alone.)
 //
 // The lists keep WT_DCAP entries per node, which covers the trees speculative decoding drafts (wide,
 // a handful of levels).  A sequence with a deeper path is left alone here and taken by the SIMT
 // kernel of wide.cu, which the launcher runs beside this one for exactly those sequences.
 //
-// One load stage: the S0 / q / k tiles are free again as soon as the tensor core has read them and the
-// v tile as soon as r is formed, so the next item's loads fly during this item's solve.  Every
-// mbarrier wait is bounded by the kernel's deadline (TREEWY_SEQ_TIMEOUT on give-up).
+// Shared memory holds one item.  The o0 tile lies over the q / k tiles (dead once the tensor core has
+// read them); the S0 tile is free again after the MMAs and the v tile once r is formed, so those two
+// are refilled during the solve and only the next item's q / k rows wait for its end.  Every mbarrier
+// wait is bounded by the kernel's deadline (TREEWY_SEQ_TIMEOUT on give-up).
 #include <cuda.h>
 
 #include <cstddef>
@@ -67,14 +74,22 @@ constexpr int OFF_AP = OFF_U + WN * D * 4;            // (A, P)[node][d]
 constexpr int OFF_IDX = OFF_AP + WN * WT_DCAP * 8;    // ancestor index [node][d]
 constexpr int OFF_PSELF = OFF_IDX + WN * WT_DCAP;     // q_i . k_i
 constexpr int OFF_PAR = OFF_PSELF + WN * 4;           // producer scratch: the sequence's parent array
+constexpr int OFF_O0 = OFF_QK;                        // o0_i = g_i S0 q_i: [node][c] fp32 over the dead q / k tiles
+static_assert(2 * QK_HALF >= WN * D * 4, "the o0 tile fits over the q / k tiles");
 constexpr int META_BYTES = ((int)sizeof(WtMeta) + 15) / 16 * 16;
 constexpr int OFF_META = OFF_PAR + WN * 4;
 static_assert(OFF_META % 16 == 0 && META_BYTES % 16 == 0 && OFF_AP % 8 == 0, "alignment of vector accesses");
 constexpr int OFF_BAR = OFF_META + 2 * META_BYTES;
-constexpr int N_BARS = 10;
+constexpr int N_BARS = 12;
 constexpr int SMEM_BYTES = OFF_BAR + N_BARS * 8 + 16 + 1024;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
-constexpr uint32_t TX_SQK = 2 * QK_HALF + 2 * S0_HALF, TX_V = WN * D * 2;
+constexpr uint32_t TX_QK = 2 * QK_HALF, TX_S0 = 2 * S0_HALF, TX_V = WN * D * 2;
+
+__device__ __forceinline__ void store_o4(float *p, const float4 &o) { *reinterpret_cast<float4 *>(p) = o; }
+__device__ __forceinline__ void store_o4(__nv_bfloat16 *p, const float4 &o)
+{
+    *reinterpret_cast<uint2 *>(p) = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
+}
 
 template <typename TOut>
 __global__ void __launch_bounds__(WT_THREADS, 1)
@@ -85,13 +100,15 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + OFF_BAR);
-    uint64_t *full_sqk = bars, *free_sqk = bars + 1, *full_v = bars + 2, *free_v = bars + 3;
+    uint64_t *full_qk = bars, *free_qk = bars + 1, *full_v = bars + 2, *free_v = bars + 3;
     uint64_t *mma_done = bars + 4, *tmem_free = bars + 5, *meta_full = bars + 6, *meta_free = bars + 8;
+    uint64_t *full_s0 = bars + 10, *free_s0 = bars + 11;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + N_BARS);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        ptx::mbar_init(full_sqk, 1), ptx::mbar_init(free_sqk, 1);
+        ptx::mbar_init(full_qk, 1), ptx::mbar_init(free_qk, WT_CWARPS);
+        ptx::mbar_init(full_s0, 1), ptx::mbar_init(free_s0, 1);
         ptx::mbar_init(full_v, 1), ptx::mbar_init(free_v, WT_CWARPS);
         ptx::mbar_init(mma_done, 1), ptx::mbar_init(tmem_free, WT_CWARPS);
         for (int x = 0; x < 2; ++x) {
@@ -207,21 +224,26 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
             __syncwarp();
             if (run) {
                 const int hq = h / group;
-                // the tiles are free once the tensor core has read them (S0, q, k) / r has been formed (v)
-                if (!ptx::mbar_wait(free_sqk, (np & 1) ^ 1)) break;
+                // S0 is free once the tensor core has read it, v once r has been formed: both early in the
+                // previous item.  The q / k tiles carry that item's o0 tile until its solve has ended.
+                if (!ptx::mbar_wait(free_s0, (np & 1) ^ 1)) break;
                 if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full_sqk, TX_SQK);
-                    ptx::tma_load_2d(smem + OFF_S0, &tmS0, 0, item * D, full_sqk);
-                    ptx::tma_load_2d(smem + OFF_S0 + S0_HALF, &tmS0, 64, item * D, full_sqk);
-                    ptx::tma_load_2d(smem + OFF_QK, &tmQ, hq * D, lo, full_sqk);
-                    ptx::tma_load_2d(smem + OFF_QK + QK_HALF, &tmQ, hq * D + 64, lo, full_sqk);
-                    ptx::tma_load_2d(smem + OFF_QK + WN * 128, &tmK, hq * D, lo, full_sqk);
-                    ptx::tma_load_2d(smem + OFF_QK + QK_HALF + WN * 128, &tmK, hq * D + 64, lo, full_sqk);
+                    ptx::mbar_arrive_expect_tx(full_s0, TX_S0);
+                    ptx::tma_load_2d(smem + OFF_S0, &tmS0, 0, item * D, full_s0);
+                    ptx::tma_load_2d(smem + OFF_S0 + S0_HALF, &tmS0, 64, item * D, full_s0);
                 }
                 if (!ptx::mbar_wait(free_v, (np & 1) ^ 1)) break;
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(full_v, TX_V);
                     ptx::tma_load_2d(smem + OFF_V, &tmV, h * D, lo, full_v);
+                }
+                if (!ptx::mbar_wait(free_qk, (np & 1) ^ 1)) break;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(full_qk, TX_QK);
+                    ptx::tma_load_2d(smem + OFF_QK, &tmQ, hq * D, lo, full_qk);
+                    ptx::tma_load_2d(smem + OFF_QK + QK_HALF, &tmQ, hq * D + 64, lo, full_qk);
+                    ptx::tma_load_2d(smem + OFF_QK + WN * 128, &tmK, hq * D, lo, full_qk);
+                    ptx::tma_load_2d(smem + OFF_QK + QK_HALF + WN * 128, &tmK, hq * D + 64, lo, full_qk);
                 }
                 ++np;
             }
@@ -240,7 +262,8 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
             if (!ptx::mbar_wait(&meta_full[kk & 1], (kk >> 1) & 1)) break;
             const int n = meta_of(kk)->n;
             if (n > 0) {
-                if (!ptx::mbar_wait(full_sqk, np & 1)) break;
+                if (!ptx::mbar_wait(full_s0, np & 1)) break;
+                if (!ptx::mbar_wait(full_qk, np & 1)) break;
                 if (!ptx::mbar_wait(tmem_free, (np & 1) ^ 1)) break;
                 ptx::tc_fence_after_sync();
                 if (lane == 0) {
@@ -255,7 +278,7 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                         ptx::umma_bf16(tmem_base + TM_GQK, dq, dk, idesc2, ks > 0);
                         ptx::umma_bf16(tmem_base + TM_GKK, dk, dk, idesc2, ks > 0);
                     }
-                    ptx::umma_commit(free_sqk);  // the three tiles have been read
+                    ptx::umma_commit(free_s0);  // the tiles have been read (q / k now take the o0 tile)
                     ptx::umma_commit(mma_done);
                 }
                 __syncwarp();
@@ -272,6 +295,7 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
         float2 *AP = reinterpret_cast<float2 *>(smem + OFF_AP);
         unsigned char *IDX = smem + OFF_IDX;
         float *pself = reinterpret_cast<float *>(smem + OFF_PSELF);
+        float *O0 = reinterpret_cast<float *>(smem + OFF_O0);
         const __nv_bfloat16 *Vt = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
         TOut *Og = static_cast<TOut *>(a.O);
         float *Ug = static_cast<float *>(a.U);
@@ -307,6 +331,11 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                 const uint32_t words[2] = {ch ? p2 : p0, ch ? p3 : p1};  // this thread's 64 columns
                 const float Li = m->L[i < n ? i : 0], scale = mat ? m->beta[i < n ? i : 0] : 1.f;
                 int pos = ch ? __popc(p0) + __popc(p1) : 0;
+                // The 32 entries of a chunk go from tensor memory to a private 128-byte line of shared memory
+                // (the tile that later holds r and u is idle now), 16-byte pieces rotated by the lane so that
+                // the stores of a quarter warp fall on different banks; the few ancestors among them are then
+                // picked by index.  (Testing all 32 columns in registers instead cost 900 instructions per thread.)
+                float *line = Ut + tid * 32;
 #pragma unroll
                 for (int cq = 0; cq < 2; ++cq) {
                     const int c0 = 64 * ch + 32 * cq;
@@ -314,28 +343,34 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                         uint32_t g[32];
                         ptx::tmem_ld32(tl + (mat ? TM_GKK : TM_GQK) + c0, g);
                         ptx::tmem_wait_ld();
-                        if (i < n) {
-                            const uint32_t word = words[cq];
 #pragma unroll
-                            for (int cc = 0; cc < 32; ++cc) {
-                                if ((word >> cc) & 1u) {
-                                    const float val = scale * __expf(Li - m->L[c0 + cc]) * __uint_as_float(g[cc]);
-                                    if (mat) {
-                                        AP[i * WT_DCAP + pos].x = val;
-                                    } else {
-                                        AP[i * WT_DCAP + pos].y = val;
-                                        IDX[i * WT_DCAP + pos] = (unsigned char)(c0 + cc);
-                                    }
-                                    ++pos;
+                        for (int q = 0; q < 8; ++q)
+                            *reinterpret_cast<uint4 *>(line + 4 * (q ^ (lane & 7))) =
+                                make_uint4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
+                        auto entry = [&](int cc) { return line[4 * ((cc >> 2) ^ (lane & 7)) + (cc & 3)]; };
+                        if (i < n) {
+                            uint32_t word = words[cq];
+#pragma unroll 1
+                            while (word) {
+                                const int cc = __ffs((int)word) - 1;
+                                word &= word - 1;
+                                const float val = scale * __expf(Li - m->L[c0 + cc]) * entry(cc);
+                                if (mat) {
+                                    AP[i * WT_DCAP + pos].x = val;
+                                } else {
+                                    AP[i * WT_DCAP + pos].y = val;
+                                    IDX[i * WT_DCAP + pos] = (unsigned char)(c0 + cc);
                                 }
-                                if (!mat && c0 + cc == i) pself[i] = __uint_as_float(g[cc]);
+                                ++pos;
                             }
+                            if (!mat && (i >> 5) == (c0 >> 5)) pself[i] = entry(i & 31);  // q_i . k_i
                         }
                     }
                 }
             }
+            ptx::named_sync(1, WT_CONS);  // every line has been read: the tile may take r
             {
-                // ---- r_i[c] for the nodes 32 grp .. 32 grp + 31 of this thread's group
+                // ---- r_i[c] and o0_i[c] for the nodes 32 grp .. 32 grp + 31 of this thread's group
                 if (!ptx::mbar_wait(full_v, np & 1)) {
                     if (tid == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                     break;
@@ -353,41 +388,50 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                             Ut[i * D + c] = fmaf(-m->bg[i], __uint_as_float(sk[jj]), m->beta[i] * v);
                         }
                     }
+                    ptx::tmem_ld32(tl + TM_SQ + i0, sk);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const int i = i0 + jj;
+                        if (i < n) O0[i * D + c] = m->g[i] * __uint_as_float(sk[jj]);
+                    }
                 }
                 ptx::mbar_arrive_warp(free_v);
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive_warp(tmem_free);  // tensor memory has been read out
             }
-            ptx::named_sync(1, WT_CONS);  // lists, q_i . k_i and r are in place
-            // ---- the solve, level by level
+            ptx::named_sync(1, WT_CONS);  // lists, q_i . k_i, r and o0 are in place
+            // ---- the solve, level by level, a warp per node, a lane per four elements of d_v
             const int lo = m->lo, h = m->h, maxd = m->maxd;
-            const size_t row0 = ((size_t)lo * a.H_v + h) * D + c;
+            const size_t row0 = ((size_t)lo * a.H_v + h) * D + 4 * lane;
 #pragma unroll 1
             for (int lv = 0; lv <= maxd; ++lv) {
                 const int p1 = m->lvl[lv + 1];
 #pragma unroll 1
-                for (int p = m->lvl[lv] + grp; p < p1; p += WT_GROUPS) {
+                for (int p = m->lvl[lv] + warp; p < p1; p += WT_CWARPS) {
                     const int i = m->order[p];
-                    const uint32_t sq = ptx::tmem_ld1(tl + TM_SQ + i);
-                    float u = Ut[i * D + c], o = 0.f;
+                    float4 *ui = reinterpret_cast<float4 *>(Ut + i * D) + lane;
+                    float4 u = *ui, o = reinterpret_cast<const float4 *>(O0 + i * D)[lane];
                     const float2 *ap = AP + i * WT_DCAP;
                     const unsigned char *ix = IDX + i * WT_DCAP;
-#pragma unroll 4
+#pragma unroll 2
                     for (int d = 0; d < lv; ++d) {
                         const float2 co = ap[d];
-                        const float uj = Ut[(int)ix[d] * D + c];
-                        u = fmaf(-co.x, uj, u);
-                        o = fmaf(co.y, uj, o);
+                        const float4 uj = reinterpret_cast<const float4 *>(Ut + (int)ix[d] * D)[lane];
+                        u.x = fmaf(-co.x, uj.x, u.x), u.y = fmaf(-co.x, uj.y, u.y);
+                        u.z = fmaf(-co.x, uj.z, u.z), u.w = fmaf(-co.x, uj.w, u.w);
+                        o.x = fmaf(co.y, uj.x, o.x), o.y = fmaf(co.y, uj.y, o.y);
+                        o.z = fmaf(co.y, uj.z, o.z), o.w = fmaf(co.y, uj.w, o.w);
                     }
-                    ptx::tmem_wait_ld();
-                    o = fmaf(m->g[i], __uint_as_float(sq), o);
-                    o = fmaf(pself[i], u, o);
-                    Ut[i * D + c] = u;
-                    Ug[row0 + (size_t)i * rs] = u;
-                    Og[row0 + (size_t)i * rs] = from_f32<TOut>(o);
+                    const float ps = pself[i];
+                    o.x = fmaf(ps, u.x, o.x), o.y = fmaf(ps, u.y, o.y), o.z = fmaf(ps, u.z, o.z), o.w = fmaf(ps, u.w, o.w);
+                    *ui = u;
+                    *reinterpret_cast<float4 *>(Ug + row0 + (size_t)i * rs) = u;
+                    store_o4(Og + row0 + (size_t)i * rs, o);
                 }
-                ptx::named_sync(1, WT_CONS);  // the level's u rows are visible to every group
+                ptx::named_sync(1, WT_CONS);  // the level's u rows are visible to every warp
             }
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive_warp(tmem_free);
+            ptx::mbar_arrive_warp(free_qk);  // the o0 tile has been read: the next item's q / k rows may land
             ptx::mbar_arrive_warp(&meta_free[kk & 1]);
             ++np;
         }
