@@ -36,6 +36,7 @@
 #include <cuda.h>
 
 #include <cstddef>
+#include <type_traits>
 
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
@@ -377,8 +378,9 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                 }
                 const int i0 = 32 * grp;
                 if (i0 < n) {
-                    uint32_t sk[32];
+                    uint32_t sk[32], sq[32];
                     ptx::tmem_ld32(tl + TM_SK + i0, sk);
+                    ptx::tmem_ld32(tl + TM_SQ + i0, sq);
                     ptx::tmem_wait_ld();
 #pragma unroll
                     for (int jj = 0; jj < 32; ++jj) {
@@ -386,14 +388,8 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                         if (i < n) {
                             const float v = __bfloat162float(Vt[i * D + c]);
                             Ut[i * D + c] = fmaf(-m->bg[i], __uint_as_float(sk[jj]), m->beta[i] * v);
+                            O0[i * D + c] = m->g[i] * __uint_as_float(sq[jj]);
                         }
-                    }
-                    ptx::tmem_ld32(tl + TM_SQ + i0, sk);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const int i = i0 + jj;
-                        if (i < n) O0[i * D + c] = m->g[i] * __uint_as_float(sk[jj]);
                     }
                 }
                 ptx::mbar_arrive_warp(free_v);
@@ -407,28 +403,45 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
 #pragma unroll 1
             for (int lv = 0; lv <= maxd; ++lv) {
                 const int p1 = m->lvl[lv + 1];
-#pragma unroll 1
-                for (int p = m->lvl[lv] + warp; p < p1; p += WT_CWARPS) {
-                    const int i = m->order[p];
-                    float4 *ui = reinterpret_cast<float4 *>(Ut + i * D) + lane;
-                    float4 u = *ui, o = reinterpret_cast<const float4 *>(O0 + i * D)[lane];
-                    const float2 *ap = AP + i * WT_DCAP;
-                    const unsigned char *ix = IDX + i * WT_DCAP;
+                // (a node is a chain of dependent shared-memory reads -- order -> lists -> u_j -- so a warp
+                // takes two nodes of the level side by side where the level has them)
+                auto nodes = [&](auto nb_tag, int p) {
+                    constexpr int NB = decltype(nb_tag)::value;
+                    int ii[NB];
+                    float4 u[NB], o[NB];
+#pragma unroll
+                    for (int t = 0; t < NB; ++t) ii[t] = m->order[p + t * WT_CWARPS];
+#pragma unroll
+                    for (int t = 0; t < NB; ++t) {
+                        u[t] = reinterpret_cast<const float4 *>(Ut + ii[t] * D)[lane];
+                        o[t] = reinterpret_cast<const float4 *>(O0 + ii[t] * D)[lane];
+                    }
 #pragma unroll 2
                     for (int d = 0; d < lv; ++d) {
-                        const float2 co = ap[d];
-                        const float4 uj = reinterpret_cast<const float4 *>(Ut + (int)ix[d] * D)[lane];
-                        u.x = fmaf(-co.x, uj.x, u.x), u.y = fmaf(-co.x, uj.y, u.y);
-                        u.z = fmaf(-co.x, uj.z, u.z), u.w = fmaf(-co.x, uj.w, u.w);
-                        o.x = fmaf(co.y, uj.x, o.x), o.y = fmaf(co.y, uj.y, o.y);
-                        o.z = fmaf(co.y, uj.z, o.z), o.w = fmaf(co.y, uj.w, o.w);
+#pragma unroll
+                        for (int t = 0; t < NB; ++t) {
+                            const float2 co = AP[ii[t] * WT_DCAP + d];
+                            const float4 uj = reinterpret_cast<const float4 *>(Ut + (int)IDX[ii[t] * WT_DCAP + d] * D)[lane];
+                            u[t].x = fmaf(-co.x, uj.x, u[t].x), u[t].y = fmaf(-co.x, uj.y, u[t].y);
+                            u[t].z = fmaf(-co.x, uj.z, u[t].z), u[t].w = fmaf(-co.x, uj.w, u[t].w);
+                            o[t].x = fmaf(co.y, uj.x, o[t].x), o[t].y = fmaf(co.y, uj.y, o[t].y);
+                            o[t].z = fmaf(co.y, uj.z, o[t].z), o[t].w = fmaf(co.y, uj.w, o[t].w);
+                        }
                     }
-                    const float ps = pself[i];
-                    o.x = fmaf(ps, u.x, o.x), o.y = fmaf(ps, u.y, o.y), o.z = fmaf(ps, u.z, o.z), o.w = fmaf(ps, u.w, o.w);
-                    *ui = u;
-                    *reinterpret_cast<float4 *>(Ug + row0 + (size_t)i * rs) = u;
-                    store_o4(Og + row0 + (size_t)i * rs, o);
-                }
+#pragma unroll
+                    for (int t = 0; t < NB; ++t) {
+                        const float ps = pself[ii[t]];
+                        o[t].x = fmaf(ps, u[t].x, o[t].x), o[t].y = fmaf(ps, u[t].y, o[t].y);
+                        o[t].z = fmaf(ps, u[t].z, o[t].z), o[t].w = fmaf(ps, u[t].w, o[t].w);
+                        reinterpret_cast<float4 *>(Ut + ii[t] * D)[lane] = u[t];
+                        *reinterpret_cast<float4 *>(Ug + row0 + (size_t)ii[t] * rs) = u[t];
+                        store_o4(Og + row0 + (size_t)ii[t] * rs, o[t]);
+                    }
+                };
+                int p = m->lvl[lv] + warp;
+#pragma unroll 1
+                for (; p + WT_CWARPS < p1; p += 2 * WT_CWARPS) nodes(std::integral_constant<int, 2>{}, p);
+                if (p < p1) nodes(std::integral_constant<int, 1>{}, p);
                 ptx::named_sync(1, WT_CONS);  // the level's u rows are visible to every warp
             }
             ptx::mbar_arrive_warp(free_qk);  // the o0 tile has been read: the next item's q / k rows may land
