@@ -20,6 +20,10 @@
 // (packed node, value head), the node playing the accepted node and the result going to a
 // separate [T, H_v] array of states instead of back to S0.
 //
+// Trees of more than 64 nodes (the wide-tree calls) have no ancestor masks: there the producer warp
+// keeps the sequence's parent array in shared memory and walks the accepted node's root path
+// through it; everything after that is the same.
+//
 // Paths longer than CP_PCH nodes (deep chains) take the staged rows first and fetch the rest
 // with ordinary loads.  All mbarrier waits are bounded (TREEWY_SEQ_TIMEOUT on give-up).
 #include "ptx_sm100.cuh"
@@ -33,6 +37,7 @@ constexpr int CP_PCH = 16;  // path nodes staged per item
 constexpr int CP_CONSUMERS = 256;
 constexpr int CP_THREADS = CP_CONSUMERS + 32 * CP_STAGES;
 constexpr uint32_t CP_TILE_BYTES = D * D * 2;
+constexpr int CP_WIDE_NODES = TREEWY_MAX_NODES_WIDE;
 
 struct __align__(128) CommitStage {
     __nv_bfloat16 tile[D * D];
@@ -45,10 +50,15 @@ struct __align__(128) CommitStage {
     int store_tile;           // 1: tile goes back to memory (accepted >= 0)
     int b, h;                 // sequence and value head of the item
     int tile_index;           // its state tile: (state slot) * H_v + h
+    // trees of more than 64 nodes have no ancestor masks: the producer walks the accepted node's root path
+    // through the parent array and leaves it here, root first
+    uint8_t path[CP_WIDE_NODES];
 };
 
 struct CommitPipeSmem {
     CommitStage stage[CP_STAGES];
+    int32_t par_scratch[CP_STAGES][CP_WIDE_NODES];
+    uint8_t path_scratch[CP_STAGES][CP_WIDE_NODES];
     uint64_t full[CP_STAGES];
     uint64_t empty[CP_STAGES];
 };
@@ -80,6 +90,9 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         // ------------------------------------------------------------------ producer warp
         const int s = warp - CP_CONSUMERS / 32;
         CommitStage &g = sm.stage[s];
+        // (the parent array of the item being PREPARED lives outside the stage proper: the stage may still
+        // be in the consumers' hands while the next item's path is walked)
+        int32_t *g_par = sm.par_scratch[s];
         for (int kk = s;; kk += CP_STAGES) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
@@ -114,6 +127,7 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 for (int i = lane; i < n; i += 32) {
                     const int p = a.parent[lo + i];
                     bp |= (p < -1 || p >= i);
+                    if (!a.anc_mask) g_par[i] = p;
                 }
                 if (__any_sync(0xffffffffu, bp)) bad = TREEWY_SEQ_BAD_PARENT;
                 else if (acc < -1 || acc >= n) bad = TREEWY_SEQ_BAD_ACCEPTED;
@@ -124,13 +138,27 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
             unsigned long long mask = 0;
             float La = 0.f, wj = 0.f;
             int plen = work ? 0 : -1, cnt = 0, j = 0;
+            uint8_t *g_path = sm.path_scratch[s];
             if (work && acc >= 0) {
-                mask = a.anc_mask[lo + acc];
                 La = a.cum_log_gate[(size_t)(lo + acc) * a.H_v + h];
-                plen = __popcll(mask);
+                if (a.anc_mask) {
+                    mask = a.anc_mask[lo + acc];
+                    plen = __popcll(mask);
+                } else {  // walk up from the accepted node (parent[p] < p: ends), then lay the path out root first
+                    __syncwarp();
+                    if (lane == 0) {
+                        int len = 0;
+                        for (int p = acc; p >= 0; p = g_par[p]) ++len;
+                        int e = len;
+                        for (int p = acc; p >= 0; p = g_par[p]) g_path[--e] = (uint8_t)p;
+                        plen = len;
+                    }
+                    __syncwarp();  // the path is written: every lane may read it
+                    plen = __shfl_sync(0xffffffffu, plen, 0);
+                }
                 cnt = min(plen, CP_PCH);
                 if (lane < cnt) {
-                    j = nth_set_bit(mask, lane);
+                    j = a.anc_mask ? nth_set_bit(mask, lane) : (int)g_path[lane];
                     wj = expf(La - a.cum_log_gate[(size_t)(lo + j) * a.H_v + h]);
                 }
             }
@@ -140,6 +168,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 break;
             }
             if (lane < cnt) g.w[lane] = wj;
+            if (!a.anc_mask && plen > CP_PCH)  // (only a deep path's tail is read from the stage)
+                for (int q = lane; q < plen; q += 32) g.path[q] = g_path[q];
             if (lane == 0) {
                 g.mask = mask, g.La = La, g.ga = expf(La), g.plen = plen;
                 g.store_tile = (acc >= 0);
@@ -211,8 +241,8 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 const int lo = a.node_offsets[b];
                 unsigned long long m = g.mask;
                 for (int q = 0; q < CP_PCH; ++q) m &= m - 1;
-                while (m) {
-                    const int j = __ffsll((long long)m) - 1;
+                for (int q = CP_PCH; q < plen; ++q) {
+                    const int j = a.anc_mask ? __ffsll((long long)m) - 1 : (int)g.path[q];
                     m &= m - 1;
                     const float w = expf(g.La - a.cum_log_gate[(size_t)(lo + j) * a.H_v + h]);
                     float kf[8];
@@ -282,6 +312,7 @@ cudaError_t launch_commit_pipe(const CommitArgs &a, cudaStream_t stream)
     int dev = 0, sms = 0;
     cudaError_t e = current_device_sms(&dev, &sms);
     if (e != cudaSuccess) return e;
+    static_assert(sizeof(CommitPipeSmem) <= 227 * 1024, "shared memory of one CTA");
     const int smem = (int)sizeof(CommitPipeSmem);
     e = ensure_dynamic_smem(reinterpret_cast<const void *>(commit_pipe_kernel), smem, dev);
     if (e != cudaSuccess) return e;

@@ -26,6 +26,14 @@ namespace {
 constexpr int WN = TREEWY_MAX_NODES_WIDE;
 constexpr int WT = 128;  // threads of a verify / prepare CTA
 
+constexpr int WP_HCHUNK = 8;  // value heads per CTA of the prepare kernel (small: the kernel is latency bound and wants many CTAs)
+
+// One CTA per (sequence, chunk of heads).  Node i walks up its root path through the parent array in
+// shared memory for its depth and a two-word ancestor-or-self mask (kept in shared memory only: the
+// wide calls hand no masks to the caller); meanwhile all threads turn the chunk's gates into
+// logf(alpha).  L[i,h] is then the sum of the table's entries over the mask's bits in ascending node
+// order -- the order of the main prepare, so the two agree bit for bit on trees both accept -- with
+// every (i, h) independent of the others.
 __global__ void __launch_bounds__(WT)
 prepare_wide_kernel(int B, int T, int H_v, int max_nodes, const int32_t *__restrict__ node_offsets,
                     const int32_t *__restrict__ parent, const float *__restrict__ alpha, int32_t *__restrict__ depth,
@@ -34,33 +42,53 @@ prepare_wide_kernel(int B, int T, int H_v, int max_nodes, const int32_t *__restr
     __shared__ int s_bad;
     __shared__ int32_t s_parent[WN];
     __shared__ int32_t s_depth[WN];
-    const int b = blockIdx.x;
+    __shared__ unsigned long long s_mask[WN][2];
+    __shared__ float s_log[WN * WP_HCHUNK];
+    const int b = blockIdx.x, h0 = blockIdx.y * WP_HCHUNK;
+    const int hc = min(WP_HCHUNK, H_v - h0);
     const int lo = node_offsets[b];
     const int n = node_offsets[b + 1] - lo;
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
     const int bad = validate_sequence(parent, lo, n, T, max_nodes, &s_bad);
     if (bad) {
-        if (threadIdx.x == 0 && seq_status) atomicOr(&seq_status[b], bad);
+        if (threadIdx.x == 0 && blockIdx.y == 0 && seq_status) atomicOr(&seq_status[b], bad);
         return;
     }
     for (int i = threadIdx.x; i < n; i += WT) s_parent[i] = parent[lo + i];
+    for (int e = threadIdx.x; e < n * hc; e += WT) {
+        const int i = e / hc, h = e - i * hc;
+        s_log[i * WP_HCHUNK + h] = logf(alpha[(size_t)(lo + i) * H_v + h0 + h]);
+    }
     __syncthreads();
     for (int i = threadIdx.x; i < n; i += WT) {
-        int d = 0;
-        for (int p = s_parent[i]; p >= 0; p = s_parent[p]) ++d;  // parent[p] < p: ends
-        s_depth[i] = d;
-        depth[lo + i] = d;
-    }
-    // one thread per head: the running sum along every root path, node after node
-    for (int h = threadIdx.x; h < H_v; h += WT) {
-        for (int i = 0; i < n; ++i) {
-            const int p = s_parent[i];
-            const float up = p < 0 ? 0.f : cum_log_gate[(size_t)(lo + p) * H_v + h];  // written by this thread
-            cum_log_gate[(size_t)(lo + i) * H_v + h] = up + logf(alpha[(size_t)(lo + i) * H_v + h]);
+        unsigned long long m0 = 0ull, m1 = 0ull;
+        int d = -1;
+        for (int p = i; p >= 0; p = s_parent[p]) {  // parent[p] < p: ends
+            if (p < 64) m0 |= 1ull << p;
+            else m1 |= 1ull << (p - 64);
+            ++d;
         }
+        s_depth[i] = d;
+        s_mask[i][0] = m0, s_mask[i][1] = m1;
+        if (blockIdx.y == 0) depth[lo + i] = d;
     }
     __syncthreads();
+    for (int e = threadIdx.x; e < n * hc; e += WT) {
+        const int i = e / hc, h = e - i * hc;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            unsigned long long m = s_mask[i][w];
+            while (m) {
+                const int j = 64 * w + __ffsll((long long)m) - 1;
+                m &= m - 1;
+                acc += s_log[j * WP_HCHUNK + h];
+            }
+        }
+        cum_log_gate[(size_t)(lo + i) * H_v + h0 + h] = acc;
+    }
+    if (blockIdx.y != 0) return;
     for (int i = threadIdx.x; i < n; i += WT) {
         const int di = s_depth[i];
         int rank = 0;
@@ -280,7 +308,7 @@ cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const flo
                                 cudaStream_t stream)
 {
     if (t.B == 0) return cudaSuccess;
-    prepare_wide_kernel<<<t.B, WT, 0, stream>>>(t.B, t.T, t.H_v, max_nodes, t.node_offsets, t.parent, alpha, t.depth,
+    prepare_wide_kernel<<<dim3(t.B, (t.H_v + WP_HCHUNK - 1) / WP_HCHUNK), WT, 0, stream>>>(t.B, t.T, t.H_v, max_nodes, t.node_offsets, t.parent, alpha, t.depth,
                                                 t.cum_log_gate, t.level_order, seq_status);
     return cudaGetLastError();
 }
@@ -310,8 +338,8 @@ cudaError_t launch_verify_wide(const VerifyArgs &a, treewy_dtype_t io, treewy_dt
 cudaError_t launch_commit_wide(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream)
 {
     if (a.B == 0 || a.H_v == 0) return cudaSuccess;
-    if (io == TREEWY_F32) commit_wide_kernel<float><<<dim3(a.H_v, a.B), WC_THREADS, 0, stream>>>(a);
-    else commit_wide_kernel<__nv_bfloat16><<<dim3(a.H_v, a.B), WC_THREADS, 0, stream>>>(a);
+    if (io == TREEWY_BF16) return launch_commit_pipe(a, stream);  // (no masks in `a`: the pipeline walks parents)
+    commit_wide_kernel<float><<<dim3(a.H_v, a.B), WC_THREADS, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
