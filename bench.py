@@ -315,7 +315,7 @@ def kernel_times(sets, dev, stream, reps: int):
     return [sum(e[j].elapsed_time(e[j + 1]) for e in ev) / reps for j in range(3)]
 
 
-def host_cost_per_call(ls: LayerSet, dev, n: int = 300):
+def host_cost_per_call(ls: LayerSet, dev, n: int = 100):
     """Host time of one enqueue (microseconds): n calls of each entry point through its marshalled
     C call, no synchronisation inside, wall clock / n.  The queue is drained between the three."""
     out = {}
@@ -512,6 +512,13 @@ def run_ours(args, rank: int, size: int, local: int):
             wo = wl.make_workload(cid, prefix_device=str(dev))
             rec, osets, _, _ = measure_workload(wo, dev, stream, args.steps, args.warmup)
             rec["value"] = size * wo.T * wo.H_v / (rec["ms_per_step"] * 1e-3)
+            if wo.io_dtype == torch.bfloat16 and wo.max_nodes <= 32:   # the fused round on this workload too
+                fstep = lambda i, s_=osets: (s_[i % 2].prepare(), s_[i % 2].commit_verify())
+                for i in range(max(args.warmup, 3)):
+                    fstep(i)
+                torch.cuda.synchronize(dev)
+                fb, _ = timed_blocks(fstep, args.steps, dev, stream, start=max(args.warmup, 3), min_total_ms=20.0)
+                rec["fused_commit_verify_ms_per_step"] = block_stats(fb, args.steps, dev)["median"]
             rec["config"] = {"B": wo.B, "H_v": wo.H_v, "H_qk": wo.H_qk, "T": wo.T, "max_nodes": wo.max_nodes}
             rec["host_us_per_call"] = host_cost_per_call(osets[0], dev)
             others[wo.name] = rec

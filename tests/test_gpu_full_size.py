@@ -77,23 +77,18 @@ def test_full_size_half_u_is_the_rounded_u():
 
 
 def test_full_size_wide_trees(oracle):
-    """The 128-node workload through the wide-tree calls, sampled sequences against the oracle."""
+    """The 128-node workload through the wide-tree calls, every sequence against the oracle."""
     from tests.test_gpu_wide import run_wide
     w = wl.make_workload(6)
     gpu = run_wide(w, max_nodes=w.max_nodes)
     assert not gpu["status"].any()
     oracle.set_max_nodes(128)
     try:
-        seqs = [0, 17, w.B - 1]
-        sub = w.select_sequences(seqs)
-        tree_ref, ref = pu.run_oracle(oracle, sub)
+        tree_ref, ref = pu.run_oracle(oracle, w)
     finally:
         oracle.set_max_nodes(64)
-    off = w.node_offsets.numpy()
-    rows = np.array([i for b in seqs for i in range(off[b], off[b + 1])], dtype=np.int64)
-    pick = {"depth": gpu["depth"][rows], "anc_mask": tree_ref.anc_mask, "cum_log_gate": gpu["cum_log_gate"][rows],
-            "level_order": gpu["level_order"][rows], "O": gpu["O"][rows], "U": gpu["U"][rows], "S": gpu["S"][seqs],
-            "S32": gpu["S32"][seqs], "status": gpu["status"][seqs]}
-    errs = pu.assert_parity(sub, pick, tree_ref, ref)
-    print(f"workload 6 full size, sequences {seqs}: {errs}")
+    gpu["anc_mask"] = tree_ref.anc_mask        # (the wide calls write no masks: nothing to compare)
+    errs = pu.assert_parity(w, gpu, tree_ref, ref)
+    print(f"workload 6 full size, all {w.B} sequences: {errs}")
     assert torch.isfinite(gpu["O"]).all() and torch.isfinite(gpu["U"]).all()
+    assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any() and not (gpu["O"] == gpu["canary"]).all(dim=-1).any()

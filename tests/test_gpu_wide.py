@@ -105,3 +105,34 @@ def test_wide_limits_are_checked_on_the_host():
     tree = tw.Tree.empty(w.node_offsets.to(dev), w.parent.to(dev), w.H_v, 129)
     with pytest.raises(tw.TreewyError):
         tw.treewy_tree_prepare_wide(tree, w.alpha.to(dev), None)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_wide_batches_shallow_and_deep_trees_side_by_side(wide_oracle, seed):
+    """Random batches of trees of 1..128 nodes whose depth limit is drawn per tree, so that the
+    tensor-core kernel (paths of up to 16 ancestors) and the SIMT kernel (deeper ones) each take their
+    share of one call; heads shared by 1, 2 or 4 value heads."""
+    g = torch.Generator().manual_seed(100 + seed)
+    ri = lambda hi: int(torch.randint(0, hi, (1,), generator=g))
+    trees = []
+    for _ in range(6 + ri(10)):
+        n = (1, 2, 17, 33, 64, 65, 96, 127, 128)[ri(9)]
+        depth_cap = (1, 2, 5, 10, 16, 17, 40, 128)[ri(8)]
+        kind = ri(4)
+        if kind == 0:      # a chain: as deep as it gets (17 nodes = 16 ancestors is the tensor-core kernel's limit)
+            n = (17, 18, 40, 128)[ri(4)]
+            trees.append([i - 1 for i in range(n)])
+        elif kind == 1:    # a chain with a bush of leaves at its end
+            stem = (15, 16, 17, 30)[ri(4)]
+            trees.append([i - 1 for i in range(stem)] + [stem - 1] * (min(n, 128 - stem)))
+        else:
+            trees.append(wl.random_parent_tree(g, n, depth_cap) if n > 1 else [-1])
+    H_v, H_qk = ((4, 4), (4, 2), (4, 1))[seed % 3]
+    acc = [ri(len(t) + 1) - 1 for t in trees]                   # -1 .. n-1
+    w = _custom(trees, H_v=H_v, H_qk=H_qk, seed=200 + seed, accepted=acc)
+    tree_ref, ref = pu.run_oracle(wide_oracle, w)
+    gpu = run_wide(w)
+    assert not gpu["status"].any()
+    gpu["anc_mask"] = tree_ref.anc_mask
+    errs = pu.assert_parity(w, gpu, tree_ref, ref)
+    print(f"seed {seed}: {len(trees)} trees, {errs}")
