@@ -243,11 +243,11 @@ treewy_status_t treewy_commit_half_u(void *S0, const void *U16, const void *k, c
  *   - tree->anc_mask is neither written nor read and may be NULL (a root path is walked through the
  *     parent array instead); depth, cum_log_gate and level_order are written as usual;
  *   - BF16 inputs: the dense contractions (S0 [Q;K]^T and both Gram blocks) run on the tensor cores and the
- *     triangular system is solved level by level on the CUDA cores, for every sequence whose deepest
- *     root path has at most 16 ancestors; a deeper sequence, and every F32 input, takes a plain fp32
- *     SIMT kernel (one CTA per (sequence, value head), an order of magnitude slower per node).  Commit
- *     of BF16 states is the bulk-copy pipeline of treewy_commit with the accepted path found by walking
- *     the parent array.  No block-pool, fused or fp16-U variant.
+ *     triangular system is solved level by level on the CUDA cores; a tree whose deepest root path has
+ *     more than 16 ancestors is accepted and takes a slower route through the same kernel.  Commit of
+ *     BF16 states is the bulk-copy pipeline of treewy_commit with the accepted path found by walking the
+ *     parent array.  F32 inputs take plain fp32 SIMT kernels (one CTA per (sequence, value head)).
+ *     No block-pool, fused or fp16-U variant.
  */
 treewy_status_t treewy_tree_prepare_wide(const treewy_tree_t *tree, const float *alpha, int32_t *seq_status,
                                          void *cuda_stream);

@@ -89,8 +89,8 @@ cudaError_t launch_verify_small(const VerifyArgs &a, const PrevRound *pv, int T,
 cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const float *alpha, int32_t *seq_status,
                                 cudaStream_t stream);
 cudaError_t launch_verify_wide(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od, cudaStream_t stream);
-// ... bf16 inputs, sequences whose deepest path has at most WIDE_TC_MAX_DEPTH ancestors: TMA + tcgen05 for the
-// dense contractions; deeper sequences are left to the SIMT kernel (launch_verify_wide runs both)
+// ... bf16 inputs: TMA + tcgen05 for the dense contractions; trees whose deepest path has at most
+// WIDE_TC_MAX_DEPTH ancestors take its fast route (ancestor lists in shared memory)
 constexpr int WIDE_TC_MAX_DEPTH = 16;
 cudaError_t launch_verify_wide_tc(const VerifyArgs &a, treewy_dtype_t od, cudaStream_t stream);
 cudaError_t launch_commit_wide(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream);

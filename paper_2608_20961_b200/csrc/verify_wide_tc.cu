@@ -26,12 +26,12 @@
 //             and 20 k cycles per item in this phase alone.)
 //
 // The lists keep WT_DCAP entries per node, which covers the trees speculative decoding drafts (wide,
-// a handful of levels).  A sequence with a deeper path is left alone here and taken by the SIMT
-// kernel of wide.cu, which the launcher runs beside this one for exactly those sequences.
+// a handful of levels).  A tree with a deeper path takes a slower route through the same kernel: no
+// lists, every coefficient read from tensor memory when it is needed.
 //
-// Shared memory holds one item.  The o0 tile lies over the q / k tiles (dead once the tensor core has
-// read them); the S0 tile is free again after the MMAs and the v tile once r is formed, so those two
-// are refilled during the solve and only the next item's q / k rows wait for its end.  Every mbarrier
+// Shared memory holds one item.  The q / k tiles are free again as soon as the tensor core has read them,
+// so the next item's q / k rows land during this item's solve; the o0 tile lies over the S0 and v
+// tiles, whose refill waits for the end of the solve (the next MMAs then wait for S0 only).  Every mbarrier
 // wait is bounded by the kernel's deadline (TREEWY_SEQ_TIMEOUT on give-up).
 #include <cuda.h>
 
@@ -61,8 +61,9 @@ constexpr int TM_SQ = 0, TM_SK = WN, TM_GQK = 2 * WN, TM_GKK = 3 * WN;
 struct WtMeta {
     alignas(16) uint32_t mask[WN][4];       // ancestor-or-self (read and written 16 bytes at a time)
     float L[WN], beta[WN], bg[WN], g[WN];   // log-gate, beta, beta g, g per node
-    int n, lo, h, b, maxd;      // n = 0: nothing to verify here (malformed, or left to the SIMT kernel)
-    int lvl[WT_DCAP + 2];       // first position of every level in `order`; lvl[maxd + 1] = n
+    int n, lo, h, b, maxd;      // n = 0: nothing to verify here (malformed sequence)
+    int deep;                   // some path has more than WT_DCAP ancestors: no lists, coefficients on demand
+    int lvl[WN + 2];            // first position of every level in `order`; lvl[maxd + 1] = n
     uint8_t order[WN];          // nodes sorted by (depth, index)
 };
 static_assert(offsetof(WtMeta, mask) % 16 == 0, "mask rows are accessed as uint4");
@@ -75,8 +76,8 @@ constexpr int OFF_AP = OFF_U + WN * D * 4;            // (A, P)[node][d]
 constexpr int OFF_IDX = OFF_AP + WN * WT_DCAP * 8;    // ancestor index [node][d]
 constexpr int OFF_PSELF = OFF_IDX + WN * WT_DCAP;     // q_i . k_i
 constexpr int OFF_PAR = OFF_PSELF + WN * 4;           // producer scratch: the sequence's parent array
-constexpr int OFF_O0 = OFF_QK;                        // o0_i = g_i S0 q_i: [node][c] fp32 over the dead q / k tiles
-static_assert(2 * QK_HALF >= WN * D * 4, "the o0 tile fits over the q / k tiles");
+constexpr int OFF_O0 = OFF_S0;                        // o0_i = g_i S0 q_i: [node][c] fp32 over the S0 and v tiles
+static_assert(OFF_V == OFF_S0 + 2 * S0_HALF && 2 * S0_HALF + WN * D * 2 >= WN * D * 4, "the o0 tile fits over S0 | v");
 constexpr int META_BYTES = ((int)sizeof(WtMeta) + 15) / 16 * 16;
 constexpr int OFF_META = OFF_PAR + WN * 4;
 static_assert(OFF_META % 16 == 0 && META_BYTES % 16 == 0 && OFF_AP % 8 == 0, "alignment of vector accesses");
@@ -101,16 +102,15 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
     extern __shared__ unsigned char smem_dyn[];
     unsigned char *smem = smem_dyn + ((1024u - (ptx::smem_u32(smem_dyn) & 1023u)) & 1023u);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + OFF_BAR);
-    uint64_t *full_qk = bars, *free_qk = bars + 1, *full_v = bars + 2, *free_v = bars + 3;
+    uint64_t *full_qk = bars, *free_qk = bars + 1, *full_v = bars + 2, *free_sv = bars + 3;
     uint64_t *mma_done = bars + 4, *tmem_free = bars + 5, *meta_full = bars + 6, *meta_free = bars + 8;
-    uint64_t *full_s0 = bars + 10, *free_s0 = bars + 11;
+    uint64_t *full_s0 = bars + 10;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + N_BARS);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        ptx::mbar_init(full_qk, 1), ptx::mbar_init(free_qk, WT_CWARPS);
-        ptx::mbar_init(full_s0, 1), ptx::mbar_init(free_s0, 1);
-        ptx::mbar_init(full_v, 1), ptx::mbar_init(free_v, WT_CWARPS);
+        ptx::mbar_init(full_qk, 1), ptx::mbar_init(free_qk, 1);
+        ptx::mbar_init(full_s0, 1), ptx::mbar_init(full_v, 1), ptx::mbar_init(free_sv, WT_CWARPS);
         ptx::mbar_init(mma_done, 1), ptx::mbar_init(tmem_free, WT_CWARPS);
         for (int x = 0; x < 2; ++x) {
             ptx::mbar_init(&meta_full[x], 1);
@@ -195,8 +195,7 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) maxd = max(maxd, __shfl_xor_sync(0xffffffffu, maxd, o));
-                run = maxd <= WT_DCAP;  // a deeper tree is the SIMT kernel's
-                if (run) {
+                {
                     int pos = 0;
 #pragma unroll 1
                     for (int dd = 0; dd <= maxd; ++dd) {  // counting sort by depth; index order inside a level
@@ -221,23 +220,13 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                     }
                 }
             }
-            if (lane == 0) m->n = run ? n : 0, m->lo = lo, m->h = h, m->b = b, m->maxd = maxd;
+            if (lane == 0) m->n = run ? n : 0, m->lo = lo, m->h = h, m->b = b, m->maxd = maxd, m->deep = maxd > WT_DCAP;
             __syncwarp();
             if (run) {
                 const int hq = h / group;
-                // S0 is free once the tensor core has read it, v once r has been formed: both early in the
-                // previous item.  The q / k tiles carry that item's o0 tile until its solve has ended.
-                if (!ptx::mbar_wait(free_s0, (np & 1) ^ 1)) break;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full_s0, TX_S0);
-                    ptx::tma_load_2d(smem + OFF_S0, &tmS0, 0, item * D, full_s0);
-                    ptx::tma_load_2d(smem + OFF_S0 + S0_HALF, &tmS0, 64, item * D, full_s0);
-                }
-                if (!ptx::mbar_wait(free_v, (np & 1) ^ 1)) break;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(full_v, TX_V);
-                    ptx::tma_load_2d(smem + OFF_V, &tmV, h * D, lo, full_v);
-                }
+                // The q / k tiles are free once the tensor core has read them, early in the previous item: its
+                // solve hides their refill.  The S0 and v tiles carry that item's o0 tile until its solve has
+                // ended; S0 is what the next MMAs then wait for, v lands behind them.
                 if (!ptx::mbar_wait(free_qk, (np & 1) ^ 1)) break;
                 if (lane == 0) {
                     ptx::mbar_arrive_expect_tx(full_qk, TX_QK);
@@ -245,6 +234,14 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                     ptx::tma_load_2d(smem + OFF_QK + QK_HALF, &tmQ, hq * D + 64, lo, full_qk);
                     ptx::tma_load_2d(smem + OFF_QK + WN * 128, &tmK, hq * D, lo, full_qk);
                     ptx::tma_load_2d(smem + OFF_QK + QK_HALF + WN * 128, &tmK, hq * D + 64, lo, full_qk);
+                }
+                if (!ptx::mbar_wait(free_sv, (np & 1) ^ 1)) break;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(full_s0, TX_S0);
+                    ptx::tma_load_2d(smem + OFF_S0, &tmS0, 0, item * D, full_s0);
+                    ptx::tma_load_2d(smem + OFF_S0 + S0_HALF, &tmS0, 64, item * D, full_s0);
+                    ptx::mbar_arrive_expect_tx(full_v, TX_V);
+                    ptx::tma_load_2d(smem + OFF_V, &tmV, h * D, lo, full_v);
                 }
                 ++np;
             }
@@ -279,7 +276,7 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                         ptx::umma_bf16(tmem_base + TM_GQK, dq, dk, idesc2, ks > 0);
                         ptx::umma_bf16(tmem_base + TM_GKK, dk, dk, idesc2, ks > 0);
                     }
-                    ptx::umma_commit(free_s0);  // the tiles have been read (q / k now take the o0 tile)
+                    ptx::umma_commit(free_qk);  // the tiles have been read
                     ptx::umma_commit(mma_done);
                 }
                 __syncwarp();
@@ -321,7 +318,8 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                 break;
             }
             ptx::tc_fence_after_sync();
-            {
+            const bool deep = m->deep != 0;
+            if (!deep) {
                 // ---- lists: this thread's Gram row (node c), half of its columns; even groups take
                 // q_c . k_j (P), odd groups k_c . k_j (A)
                 const int i = c, mat = grp & 1, ch = grp >> 1;
@@ -369,39 +367,100 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                     }
                 }
             }
-            ptx::named_sync(1, WT_CONS);  // every line has been read: the tile may take r
             {
-                // ---- r_i[c] and o0_i[c] for the nodes 32 grp .. 32 grp + 31 of this thread's group
+                // ---- r_i[c] and o0_i[c] for the nodes 32 grp .. 32 grp + 31 of this thread's group.  The o0
+                // tile lies over the S0 and v tiles: every v element is in a register before the first o0
+                // row is written (the same barrier says that the lines of the list phase have been read).
                 if (!ptx::mbar_wait(full_v, np & 1)) {
                     if (tid == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                     break;
                 }
                 const int i0 = 32 * grp;
+                float vv[32];
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) vv[jj] = i0 + jj < n ? __bfloat162float(Vt[(i0 + jj) * D + c]) : 0.f;
+                ptx::named_sync(1, WT_CONS);
                 if (i0 < n) {
-                    uint32_t sk[32], sq[32];
-                    ptx::tmem_ld32(tl + TM_SK + i0, sk);
-                    ptx::tmem_ld32(tl + TM_SQ + i0, sq);
+                    uint32_t sx[32];
+                    ptx::tmem_ld32(tl + TM_SK + i0, sx);
                     ptx::tmem_wait_ld();
 #pragma unroll
                     for (int jj = 0; jj < 32; ++jj) {
                         const int i = i0 + jj;
-                        if (i < n) {
-                            const float v = __bfloat162float(Vt[i * D + c]);
-                            Ut[i * D + c] = fmaf(-m->bg[i], __uint_as_float(sk[jj]), m->beta[i] * v);
-                            O0[i * D + c] = m->g[i] * __uint_as_float(sq[jj]);
-                        }
+                        if (i < n) Ut[i * D + c] = fmaf(-m->bg[i], __uint_as_float(sx[jj]), m->beta[i] * vv[jj]);
+                    }
+                    ptx::tmem_ld32(tl + TM_SQ + i0, sx);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const int i = i0 + jj;
+                        if (i < n) O0[i * D + c] = m->g[i] * __uint_as_float(sx[jj]);
                     }
                 }
-                ptx::mbar_arrive_warp(free_v);
-                ptx::tc_fence_before_sync();
-                ptx::mbar_arrive_warp(tmem_free);  // tensor memory has been read out
+                if (!deep) {
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive_warp(tmem_free);  // tensor memory has been read out
+                }
             }
             ptx::named_sync(1, WT_CONS);  // lists, q_i . k_i, r and o0 are in place
             // ---- the solve, level by level, a warp per node, a lane per four elements of d_v
             const int lo = m->lo, h = m->h, maxd = m->maxd;
             const size_t row0 = ((size_t)lo * a.H_v + h) * D + 4 * lane;
+            if (deep) {
+                // A tree with a path of more than WT_DCAP ancestors (a chain, a comb: not what drafting
+                // produces, but a legal input): no lists.  The Gram blocks are still in tensor memory, where
+                // row i is held by lane i % 32 of the warps of quarter i / 32; so a node goes to a warp of its
+                // own quarter, which reads one column at a time and passes the entry round by shuffle.  Slow
+                // (two tensor-memory reads per ancestor), correct for any tree.
 #pragma unroll 1
-            for (int lv = 0; lv <= maxd; ++lv) {
+                for (int lv = 0; lv <= maxd; ++lv) {
+                    const int p1 = m->lvl[lv + 1];
+                    int mine = 0;
+#pragma unroll 1
+                    for (int p = m->lvl[lv]; p < p1; ++p) {
+                        const int i = m->order[p];
+                        if ((i >> 5) != q4) continue;
+                        if ((mine++ & (WT_GROUPS - 1)) != grp) continue;
+                        const uint4 mw = *reinterpret_cast<const uint4 *>(m->mask[i]);
+                        uint32_t pw[4] = {mw.x, mw.y, mw.z, mw.w};
+                        const float Li = m->L[i], bi = m->beta[i];
+                        float4 u = reinterpret_cast<const float4 *>(Ut + i * D)[lane];
+                        float4 o = reinterpret_cast<const float4 *>(O0 + i * D)[lane];
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t word = pw[w];
+                            if (w == (i >> 5)) word &= ~(1u << (i & 31));  // proper ancestors
+#pragma unroll 1
+                            while (word) {
+                                const int j = 32 * w + __ffs((int)word) - 1;
+                                word &= word - 1;
+                                const uint32_t kkv = ptx::tmem_ld1(tl + TM_GKK + j), qkv = ptx::tmem_ld1(tl + TM_GQK + j);
+                                ptx::tmem_wait_ld();
+                                const float kk = __uint_as_float(__shfl_sync(0xffffffffu, kkv, i & 31));
+                                const float qk = __uint_as_float(__shfl_sync(0xffffffffu, qkv, i & 31));
+                                const float e = __expf(Li - m->L[j]), ca = bi * e * kk, cp = e * qk;
+                                const float4 uj = reinterpret_cast<const float4 *>(Ut + j * D)[lane];
+                                u.x = fmaf(-ca, uj.x, u.x), u.y = fmaf(-ca, uj.y, u.y);
+                                u.z = fmaf(-ca, uj.z, u.z), u.w = fmaf(-ca, uj.w, u.w);
+                                o.x = fmaf(cp, uj.x, o.x), o.y = fmaf(cp, uj.y, o.y);
+                                o.z = fmaf(cp, uj.z, o.z), o.w = fmaf(cp, uj.w, o.w);
+                            }
+                        }
+                        const uint32_t psv = ptx::tmem_ld1(tl + TM_GQK + i);
+                        ptx::tmem_wait_ld();
+                        const float ps = __uint_as_float(__shfl_sync(0xffffffffu, psv, i & 31));  // q_i . k_i
+                        o.x = fmaf(ps, u.x, o.x), o.y = fmaf(ps, u.y, o.y), o.z = fmaf(ps, u.z, o.z), o.w = fmaf(ps, u.w, o.w);
+                        reinterpret_cast<float4 *>(Ut + i * D)[lane] = u;
+                        *reinterpret_cast<float4 *>(Ug + row0 + (size_t)i * rs) = u;
+                        store_o4(Og + row0 + (size_t)i * rs, o);
+                    }
+                    ptx::named_sync(1, WT_CONS);  // the level's u rows are visible to every warp
+                }
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive_warp(tmem_free);  // the Gram blocks were read to the end
+            }
+#pragma unroll 1
+            for (int lv = 0; lv <= (deep ? -1 : maxd); ++lv) {
                 const int p1 = m->lvl[lv + 1];
                 // (a node is a chain of dependent shared-memory reads -- order -> lists -> u_j -- so a warp
                 // takes two nodes of the level side by side where the level has them)
@@ -444,7 +503,7 @@ verify_wide_tc_kernel(VerifyArgs a, int n_items, const __grid_constant__ CUtenso
                 if (p < p1) nodes(std::integral_constant<int, 1>{}, p);
                 ptx::named_sync(1, WT_CONS);  // the level's u rows are visible to every warp
             }
-            ptx::mbar_arrive_warp(free_qk);  // the o0 tile has been read: the next item's q / k rows may land
+            ptx::mbar_arrive_warp(free_sv);  // the o0 tile has been read: the next item's S0 tile and v rows may land
             ptx::mbar_arrive_warp(&meta_free[kk & 1]);
             ++np;
         }

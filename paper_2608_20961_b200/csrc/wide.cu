@@ -1,14 +1,14 @@
-// Trees of more than 64 nodes (up to TREEWY_MAX_NODES_WIDE = 128): prepare, verify (Eq. 2 and the
-// read-out) and commit (Eq. 3) without ancestor masks.  A 64-bit mask per node is what the main calls
-// key everything on; here a node's root path is walked through the parent array in shared memory
-// instead, which any tree size allows.  These are plain fp32 SIMT kernels, one CTA per (sequence,
-// value head): a first, correct path for wide draft trees (the paper's window N is a serving
-// parameter, Section 4), not a tuned one -- the blocked solve on the tensor cores that would make it
-// fast is not built.
+// Trees of more than 64 nodes (up to TREEWY_MAX_NODES_WIDE = 128): prepare, and the fp32 paths of verify
+// (Eq. 2 and the read-out) and commit (Eq. 3), without ancestor masks.  A 64-bit mask per node is what
+// the main calls key everything on; here a node's root path is walked through the parent array in
+// shared memory instead, which any tree size allows.  bf16 inputs do not come here: their verify is
+// the tensor-core kernel of verify_wide_tc.cu and their commit the bulk-copy pipeline of
+// commit_pipe.cu.  The verify and commit kernels below are plain fp32 SIMT kernels, one CTA per
+// (sequence, value head), the path fp32 inputs take.
 //
-//   prepare: depth by walking up, L[i,h] = L[parent(i),h] + logf(alpha[i,h]) node after node (the
-//     order a sum over the root path in ascending node index gives, as in the main prepare),
-//     level order by rank; the ancestor masks are not written.
+//   prepare: depth and a two-word ancestor mask by walking up; L[i,h] = sum of logf(alpha[j,h]) over the
+//     mask's bits in ascending node order (the order of the main prepare); level order by rank; the
+//     masks stay in shared memory.
 //   verify, thread c = row c of S0 (kept in registers) = element c of every u_i, o_i:
 //     for node i in index order (parents first):  sk = S0[c,:].k_i, sq = S0[c,:].q_i;
 //     the warps share out the ancestors j of i and reduce k_j.k_i and k_j.q_i over the lanes;
@@ -119,10 +119,8 @@ template <typename TIn> struct WideSmem {
     int bad;
 };
 
-// (deep_only: the tensor-core kernel takes every sequence whose deepest path has at most
-// WIDE_TC_MAX_DEPTH ancestors; this launch then serves the others and leaves those alone)
 template <typename TIn, typename TOut>
-__global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a, int deep_only)
+__global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     WideSmem<TIn> &sm = *reinterpret_cast<WideSmem<TIn> *>(smem_raw);
@@ -138,13 +136,6 @@ __global__ void __launch_bounds__(WT) verify_wide_kernel(VerifyArgs a, int deep_
         return;
     }
     for (int i = c; i < n; i += WT) sm.parent[i] = a.parent[lo + i];
-    if (deep_only) {
-        __syncthreads();
-        int d = 0;
-        if (c < n)
-            for (int p = sm.parent[c]; p >= 0; p = sm.parent[p]) ++d;
-        if (!__syncthreads_or(d > WIDE_TC_MAX_DEPTH)) return;
-    }
     const int hq = h / (a.H_v / a.H_qk);
     const TIn *qg = static_cast<const TIn *>(a.q), *kg = static_cast<const TIn *>(a.k), *vg = static_cast<const TIn *>(a.v);
     for (int i = 0; i < n; ++i) sm.kf[i][c] = kg[((size_t)(lo + i) * a.H_qk + hq) * D + c];
@@ -313,26 +304,20 @@ cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const flo
     return cudaGetLastError();
 }
 
-template <typename TIn, typename TOut> static cudaError_t launch_vw(const VerifyArgs &a, int deep_only, cudaStream_t stream)
+template <typename TIn, typename TOut> static cudaError_t launch_vw(const VerifyArgs &a, cudaStream_t stream)
 {
     const int smem = (int)sizeof(WideSmem<TIn>);
     cudaError_t e = cudaFuncSetAttribute(verify_wide_kernel<TIn, TOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    verify_wide_kernel<TIn, TOut><<<dim3(a.H_v, a.B), WT, smem, stream>>>(a, deep_only);
+    verify_wide_kernel<TIn, TOut><<<dim3(a.H_v, a.B), WT, smem, stream>>>(a);
     return cudaGetLastError();
 }
 
 cudaError_t launch_verify_wide(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od, cudaStream_t stream)
 {
     if (a.B == 0 || a.H_v == 0) return cudaSuccess;
-    if (io == TREEWY_F32)
-        return od == TREEWY_F32 ? launch_vw<float, float>(a, 0, stream) : launch_vw<float, __nv_bfloat16>(a, 0, stream);
-    // bf16: the tensor-core kernel for every sequence it takes (paths of up to WIDE_TC_MAX_DEPTH ancestors),
-    // the SIMT kernel for the deeper ones
-    cudaError_t e = od == TREEWY_F32 ? launch_vw<__nv_bfloat16, float>(a, 1, stream)
-                                     : launch_vw<__nv_bfloat16, __nv_bfloat16>(a, 1, stream);
-    if (e != cudaSuccess) return e;
-    return launch_verify_wide_tc(a, od, stream);
+    if (io == TREEWY_BF16) return launch_verify_wide_tc(a, od, stream);  // TMA + tcgen05
+    return od == TREEWY_F32 ? launch_vw<float, float>(a, stream) : launch_vw<float, __nv_bfloat16>(a, stream);
 }
 
 cudaError_t launch_commit_wide(const CommitArgs &a, treewy_dtype_t io, cudaStream_t stream)
