@@ -65,7 +65,7 @@ def measured_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.002):
+    def __init__(self, index: int, period_s: float = 0.001):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -296,7 +296,8 @@ def block_stats(block_ms, steps: int, dev):
     s = sorted(block_ms)
     med = 0.5 * (s[(len(s) - 1) // 2] + s[len(s) // 2])
     f = lambda x: replicas.max_over_ranks(x, dev) / steps
-    return {"median": f(med), "min": f(s[0]), "max": f(s[-1]), "blocks": len(s)}
+    return {"median": f(med), "min": f(s[0]), "max": f(s[-1]), "blocks": len(s),
+            "series": [round(x / steps, 5) for x in block_ms]}   # this rank's blocks in time order
 
 
 def kernel_times(sets, dev, stream, reps: int):
@@ -336,7 +337,7 @@ def n_launches(w: wl.Workload) -> int:
     return 4 if w.io_dtype == torch.bfloat16 and 32 < w.max_nodes <= 64 else 3
 
 
-def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampler=None):
+def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampler=None, min_total_ms: float = 40.0):
     """The step (prepare + verify + commit, two layer sets rotated) on one workload: block-median time,
     per-kernel times, roofline fractions against the measured and the nominal bandwidth."""
     pb = pass_bytes(w)
@@ -354,7 +355,7 @@ def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampl
     for i in range(warmup):
         step(i)
     torch.cuda.synchronize(dev)
-    blocks, nxt = timed_blocks(step, steps, dev, stream, start=warmup, sampler=sampler)
+    blocks, nxt = timed_blocks(step, steps, dev, stream, start=warmup, sampler=sampler, min_total_ms=min_total_ms)
     st = block_stats(blocks, steps, dev)
     kt = kernel_times(sets, dev, stream, max(3, min(steps, 50)))
     assert not any(int(s_.status.max()) for s_ in sets), "a sequence was flagged"
@@ -363,7 +364,7 @@ def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampl
     nominal_ms = pb.total / (NOMINAL_HBM_GBS * 1e9) * 1e3
     rec = {
         "ms_per_step": st["median"], "ms_per_step_min": st["min"], "ms_per_step_max": st["max"],
-        "blocks": st["blocks"], "steps_per_block": steps,
+        "blocks": st["blocks"], "steps_per_block": steps, "ms_per_step_blocks": st["series"],
         "kernel_ms": {"prepare": kt[0], "verify": kt[1], "commit": kt[2]},
         "kernel_gbs": {"prepare": pb.prepare / kt[0] / 1e6, "verify": pb.verify / kt[1] / 1e6,
                        "commit": pb.commit / kt[2] / 1e6},
@@ -388,7 +389,8 @@ def run_ours(args, rank: int, size: int, local: int):
     w = wl.make_workload(args.config, B=args.batch, prefix_device=str(dev))
     units = w.T * w.H_v
     clocks = ClockSampler(physical_gpu_index(local))
-    main, sets, pb, kt = measure_workload(w, dev, stream, args.steps, args.warmup, sampler=clocks)
+    main, sets, pb, kt = measure_workload(w, dev, stream, args.steps, args.warmup, sampler=clocks,
+                                           min_total_ms=60.0)   # (long enough for a dozen clock samples)
     ms_per_step = main["ms_per_step"]
     value = size * units / (ms_per_step * 1e-3)
 
@@ -537,9 +539,9 @@ def run_ours(args, rank: int, size: int, local: int):
                              "(CUDA events on the launching stream, MAX over ranks)",
                    "parallelism": f"replicas x{size}, no collective"},
         "ms_per_step_min": main["ms_per_step_min"], "ms_per_step_max": main["ms_per_step_max"],
-        "blocks": main["blocks"],
+        "blocks": main["blocks"], "ms_per_step_blocks": main["ms_per_step_blocks"],
         "clocks": clocks.summary(), "e2e": e2e,
-        "gpu_launches": n_launches(w) * args.steps,
+        "gpu_launches": n_launches(w) * args.steps * main["blocks"],   # inside the timed region
         "roofline": roofline,
         "step_roofline": main["step_roofline"],
         "kernel_ms": main["kernel_ms"],
