@@ -93,9 +93,19 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
         // (the parent array of the item being PREPARED lives outside the stage proper: the stage may still
         // be in the consumers' hands while the next item's path is walked)
         int32_t *g_par = sm.par_scratch[s];
+        // The first item of a stage: its state tile depends on nothing but the item's number, so it is
+        // put in flight before the chain accepted -> mask / log-gate -> path gates is walked (three or
+        // four dependent loads, 4 us in a role trace, that would otherwise stand in front of the launch's
+        // first bytes).
+        const bool early = !a.snap_out && !a.state_index && (int)blockIdx.x + s * (int)gridDim.x < n_items;
+        if (early && lane == 0) {
+            ptx::mbar_expect_tx(&sm.full[s], CP_TILE_BYTES);
+            ptx::bulk_g2s(g.tile, S0 + (size_t)(blockIdx.x + s * gridDim.x) * D * D, CP_TILE_BYTES, &sm.full[s]);
+        }
         for (int kk = s;; kk += CP_STAGES) {
             const int item = blockIdx.x + kk * gridDim.x;
             if (item >= n_items) break;
+            const bool tile_issued = early && kk == s;
             int b, h;
             if (a.snap_out) {  // snapshot mode: item = (packed node, head); find the node's sequence
                 const int t = item / a.H_v;
@@ -176,13 +186,14 @@ __global__ void __launch_bounds__(CP_THREADS, 1) commit_pipe_kernel(CommitArgs a
                 g.b = b, g.h = h, g.tile_index = (slot < 0 ? 0 : slot) * a.H_v + h;
             }
             __syncwarp();
-            if (!work) {
+            if (!work) {  // (a tile issued ahead still lands before the phase completes; nobody reads it)
                 if (lane == 0) ptx::mbar_arrive(&sm.full[s]);
                 continue;
             }
             if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(&sm.full[s], CP_TILE_BYTES + cnt * (D * 2 + D * ub));
-                ptx::bulk_g2s(g.tile, S0 + ((size_t)slot * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
+                ptx::mbar_arrive_expect_tx(&sm.full[s], (tile_issued ? 0u : CP_TILE_BYTES) + cnt * (D * 2 + D * ub));
+                if (!tile_issued)
+                    ptx::bulk_g2s(g.tile, S0 + ((size_t)slot * a.H_v + h) * D * D, CP_TILE_BYTES, &sm.full[s]);
             }
             __syncwarp();
             if (lane < cnt) {

@@ -199,6 +199,15 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
             }
             return p;
         };
+        // The first item of a stage: its state tile depends on nothing but the item's number, so it is put
+        // in flight before the item's scalars are fetched.
+        const int item0 = (int)blockIdx.x + s * (int)gridDim.x;
+        const bool early = !a.state_index && item0 < n_items;
+        if (early && lane == 0) {
+            ptx::mbar_expect_tx(&full[s], 2 * VS_HALF);
+            ptx::tma_load_2d(stage + C::OFF_TILE, &tmS0, 0, item0 * D, &full[s]);
+            ptx::tma_load_2d(stage + C::OFF_TILE + VS_HALF, &tmS0, 64, item0 * D, &full[s]);
+        }
         Pre cur = fetch(s);
 #pragma unroll 1
         for (int kk = s;; kk += C::STAGES) {
@@ -217,7 +226,7 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
             if (lane == 0) *reinterpret_cast<volatile int *>(&meta->item) = p.item;
             if (lane == 0) meta->n = p.bad ? 0 : p.n, meta->lo = p.lo, meta->srow = p.srow, meta->plen = p.plen, meta->ga = expf(p.La);
             const int cnt = p.plen > 0 ? p.plen : 0;
-            const bool need_tile = !p.bad || p.plen >= 0;  // the state tile serves verify, commit or both
+            const bool need_tile = (!p.bad || p.plen >= 0) && !(early && kk == s);  // the state tile serves verify, commit or both
             const uint32_t tx = (need_tile ? 2 * VS_HALF : 0) + (p.bad ? 0 : 2 * VS_QK_HALF + VS_N * D * 2) + cnt * (D * 2 + D * 4);
             const int hq = p.h / group_heads;
             if (lane == 0 && need_tile) {
