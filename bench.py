@@ -155,6 +155,17 @@ class LayerSet:
                                   self.tree, w.H_qk, self.acc, None, self.status)
         self._half = self._fused = None
         self._flip = 0
+        self._wide = wide
+
+    def raw_step_calls(self):
+        """The three calls as plain binding calls on the CURRENT stream (for capture in a CUDA graph)."""
+        tw, w = self.tw, self.w
+        prep = tw.treewy_tree_prepare_wide if self._wide else tw.treewy_tree_prepare
+        ver = tw.treewy_verify_wide if self._wide else tw.treewy_verify
+        com = tw.treewy_commit_wide if self._wide else tw.treewy_commit
+        return (lambda: prep(self.tree, self.alpha, self.status),
+                lambda: ver(self.S0, self.q, self.k, self.v, self.beta, self.tree, w.H_qk, self.O, self.U, self.status),
+                lambda: com(self.S0, self.U, self.k, self.tree, w.H_qk, self.acc, None, self.status))
 
     def _half_calls(self):
         """verify / commit with the pseudo-values kept in fp16 (own buffer)."""
@@ -331,6 +342,40 @@ def host_cost_per_call(ls: LayerSet, dev, n: int = 100):
     return out
 
 
+def graph_replay_ms_per_step(sets, dev, steps: int) -> float:
+    """The same step captured in a CUDA graph and replayed: what a caller sees whose host does not have
+    to enqueue the launches one by one (the paper's chain path runs under a CUDA graph, Section 4)."""
+    calls = [s_.raw_step_calls() for s_ in sets]
+
+    def raw_step(i: int):
+        a, b = calls[i % 2], calls[(i + 1) % 2]
+        a[0](), a[1](), b[2]()
+
+    n = 2 * ((steps + 1) // 2)            # an even number of steps: a replay leaves the rotation where it was
+    side = torch.cuda.Stream(dev)
+    side.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(side):
+        raw_step(0), raw_step(1)
+    torch.cuda.current_stream(dev).wait_stream(side)
+    torch.cuda.synchronize(dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(n):
+            raw_step(i)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(3, int(40.0 / max(1e-3, n * 0.05)) // 10)
+    stream = torch.cuda.current_stream(dev)
+    e0.record(stream)
+    for _ in range(reps):
+        graph.replay()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    return e0.elapsed_time(e1) / (reps * n)
+
+
 def n_launches(w: wl.Workload) -> int:
     """Kernels per prepare + verify + commit step: a bf16 batch whose trees may exceed 32 nodes verifies
     in two launches (one per size class)."""
@@ -358,6 +403,7 @@ def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampl
     blocks, nxt = timed_blocks(step, steps, dev, stream, start=warmup, sampler=sampler, min_total_ms=min_total_ms)
     st = block_stats(blocks, steps, dev)
     kt = kernel_times(sets, dev, stream, max(3, min(steps, 50)))
+    graph_ms = graph_replay_ms_per_step(sets, dev, steps)
     assert not any(int(s_.status.max()) for s_ in sets), "a sequence was flagged"
     hbm, tf, which = measured_peaks()
     roof_ms = max(pb.total / (hbm * 1e9), pb.tensor_flops / (tf * 1e12)) * 1e3
@@ -372,6 +418,7 @@ def measure_workload(w: wl.Workload, dev, stream, steps: int, warmup: int, sampl
                           "frac": roof_ms / st["median"], "peak_source": f"of {which}",
                           "frac_of_nominal_8tbs": nominal_ms / st["median"]},
         "gpu_launches_per_step": n_launches(w),
+        "graph_replay_ms_per_step": graph_ms,   # the same steps replayed from a CUDA graph
     }
     return rec, sets, pb, kt
 
@@ -547,6 +594,7 @@ def run_ours(args, rank: int, size: int, local: int):
         "kernel_ms": main["kernel_ms"],
         "kernel_gbs": main["kernel_gbs"],
         "host_us_per_call": host_us,
+        "graph_replay_ms_per_step": main["graph_replay_ms_per_step"],
         "footprint": footprint.footprint_report(w.max_nodes, w.H_v, w.H_qk),
         "snapshot_comparator": storeall,
         "fused_commit_verify": fused, "half_u": half_u,
