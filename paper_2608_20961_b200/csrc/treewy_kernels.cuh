@@ -85,7 +85,9 @@ cudaError_t launch_commit_verify_sm100(const VerifyArgs &a, const PrevRound &pv,
 constexpr int SMALL_MAX_NODES = 8;
 cudaError_t launch_verify_small(const VerifyArgs &a, const PrevRound *pv, int T, treewy_dtype_t od,
                                 cudaStream_t stream);
-// trees of up to TREEWY_MAX_NODES_WIDE nodes: fp32 SIMT kernels that walk parent chains (no masks)
+// trees of up to TREEWY_MAX_NODES_WIDE nodes, no ancestor masks (root paths are walked through the parent array):
+// prepare; verify and commit dispatch on the input type -- bf16 takes the tensor-core kernel below and the
+// bulk-copy commit pipeline in its parent-walk mode (CommitArgs::anc_mask == NULL), fp32 the SIMT kernels
 cudaError_t launch_prepare_wide(const treewy_tree_t &t, int max_nodes, const float *alpha, int32_t *seq_status,
                                 cudaStream_t stream);
 cudaError_t launch_verify_wide(const VerifyArgs &a, treewy_dtype_t io, treewy_dtype_t od, cudaStream_t stream);
