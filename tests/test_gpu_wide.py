@@ -136,3 +136,14 @@ def test_random_wide_batches_shallow_and_deep_trees_side_by_side(wide_oracle, se
     gpu["anc_mask"] = tree_ref.anc_mask
     errs = pu.assert_parity(w, gpu, tree_ref, ref)
     print(f"seed {seed}: {len(trees)} trees, {errs}")
+
+
+def test_wide_calls_on_a_tiny_batch(wide_oracle):
+    """Fewer packed nodes than one load box has rows (T = 4 against boxes of 128 rows): the loads read
+    zeros past the arrays' end and nothing outside a sequence's rows is written."""
+    w = _custom([[-1], [-1, 0, 0]], H_v=2, H_qk=1, seed=31, accepted=[0, 2])
+    tree_ref, ref = pu.run_oracle(wide_oracle, w)
+    gpu = run_wide(w)
+    assert not gpu["status"].any()
+    gpu["anc_mask"] = tree_ref.anc_mask
+    pu.assert_parity(w, gpu, tree_ref, ref)
