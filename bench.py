@@ -640,8 +640,8 @@ def run_ours(args, rank: int, size: int, local: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, help="workload id (2 = the metric's)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch size (profiling captures on a small case)")
