@@ -31,6 +31,11 @@
  * Matrix products are written as the triple loops of their definition.  The only
  * algebra applied to Eq. 1 is associativity of  S (k k^T) = (S k) k^T.
  *
+ * Malformed sequences -- a node range that is not a range inside the T packed nodes, a node count
+ * outside 1..max, a parent that is not an earlier node, an accepted node outside the tree -- are
+ * flagged with the library's status bits and skipped (the packed layout and these rules are the
+ * library's; the paper packs nothing).
+ *
  * Parity status of the functions here: all pinned (see tests/test_oracle_pins.py:
  * literal-matrix chain recurrence, beta = 0 closed form, orthonormal-key
  * overwrite, N = 1 by hand, brute-force path enumeration, fp64 closed form of
@@ -58,6 +63,7 @@ void treewy_oracle_set_max_nodes(int32_t n)
 #define ORACLE_SEQ_BAD_PARENT 1
 #define ORACLE_SEQ_TOO_MANY_NODES 2
 #define ORACLE_SEQ_BAD_ACCEPTED 4
+#define ORACLE_SEQ_BAD_OFFSETS 32 /* the sequence's node range is not a range inside 0..T */
 
 int treewy_oracle_num_threads(void)
 {
@@ -69,9 +75,13 @@ int treewy_oracle_num_threads(void)
 }
 
 /* 0 when sequence b is well formed, else the status bits describing why not. */
-static int check_sequence(const int32_t *node_offsets, const int32_t *parent, int32_t b)
+static int check_sequence(const int32_t *node_offsets, const int32_t *parent, int32_t b, int32_t T)
 {
     const int32_t lo = node_offsets[b], n = node_offsets[b + 1] - lo;
+    /* packed layout (the library's; the paper packs nothing): a range that is negative, runs backwards
+       or ends past the T packed nodes is malformed, and nothing of it is addressed */
+    if (lo < 0 || n < 0 || (int64_t)lo + n > (int64_t)T)
+        return ORACLE_SEQ_BAD_OFFSETS;
     if (n < 1 || n > oracle_max_nodes)
         return ORACLE_SEQ_TOO_MANY_NODES;
     for (int32_t i = 0; i < n; ++i) {
@@ -87,13 +97,13 @@ static int check_sequence(const int32_t *node_offsets, const int32_t *parent, in
  * depth [T], anc_mask [T], L [T, H_v], level_order [T] are written for well-formed sequences and
  * left untouched for malformed ones, whose seq_status[b] gets the reason OR-ed in.
  */
-int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
+int treewy_oracle_prepare(int32_t B, int32_t T, int32_t H_v, const int32_t *node_offsets,
                           const int32_t *parent, const double *alpha, int32_t *depth,
                           uint64_t *anc_mask, double *L, uint8_t *level_order,
                           int32_t *seq_status)
 {
     for (int32_t b = 0; b < B; ++b) {
-        const int bad = check_sequence(node_offsets, parent, b);
+        const int bad = check_sequence(node_offsets, parent, b, T);
         if (bad) {
             if (seq_status)
                 seq_status[b] |= bad;
@@ -140,7 +150,7 @@ int treewy_oracle_prepare(int32_t B, int32_t H_v, const int32_t *node_offsets,
  * -1..N-1) are skipped: their outputs are left untouched and seq_status[b] gets
  * the reason OR-ed in.
  */
-int treewy_oracle_verify_commit(int32_t B, int32_t H_v, int32_t H_qk, int32_t d_k, int32_t d_v,
+int treewy_oracle_verify_commit(int32_t B, int32_t T, int32_t H_v, int32_t H_qk, int32_t d_k, int32_t d_v,
                                 const int32_t *node_offsets, const int32_t *parent,
                                 const double *S0, const double *q, const double *k,
                                 const double *v, const double *alpha, const double *beta,
@@ -153,7 +163,7 @@ int treewy_oracle_verify_commit(int32_t B, int32_t H_v, int32_t H_qk, int32_t d_
     const size_t state = (size_t)d_v * d_k;
 
     for (int32_t b = 0; b < B; ++b) {
-        int bad = check_sequence(node_offsets, parent, b);
+        int bad = check_sequence(node_offsets, parent, b, T);
         if (!bad && accepted) {
             const int32_t n = node_offsets[b + 1] - node_offsets[b];
             if (accepted[b] < -1 || accepted[b] >= n)
@@ -168,7 +178,7 @@ int treewy_oracle_verify_commit(int32_t B, int32_t H_v, int32_t H_qk, int32_t d_
     for (int32_t b = 0; b < B; ++b) {
         for (int32_t h = 0; h < H_v; ++h) {
             const int32_t lo = node_offsets[b], n = node_offsets[b + 1] - lo;
-            if (check_sequence(node_offsets, parent, b))
+            if (check_sequence(node_offsets, parent, b, T))
                 continue;
             if (accepted && (accepted[b] < -1 || accepted[b] >= n))
                 continue;

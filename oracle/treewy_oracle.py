@@ -25,6 +25,7 @@ _LIB = os.path.join(_HERE, "libtreewy_oracle.so")
 SEQ_BAD_PARENT = 1
 SEQ_TOO_MANY_NODES = 2
 SEQ_BAD_ACCEPTED = 4
+SEQ_BAD_OFFSETS = 32
 
 _lib = None
 
@@ -87,8 +88,10 @@ class OracleResult:
     Snap: np.ndarray | None  # float64 [T, H_v, d_v, d_k] when requested
 
 
-def prepare(node_offsets, parent, alpha) -> OracleTree:
-    """depth, ancestor-or-self masks and cumulative log-gates of a packed batch of trees."""
+def prepare(node_offsets, parent, alpha, T_declared: int | None = None) -> OracleTree:
+    """depth, ancestor-or-self masks and cumulative log-gates of a packed batch of trees.
+    T_declared: the packed node count the tree declares (default: the arrays' length); a sequence whose
+    node range leaves 0..T_declared is flagged and skipped."""
     lib = _load()
     off = _arr(node_offsets, np.int32)
     par = _arr(parent, np.int32)
@@ -101,7 +104,9 @@ def prepare(node_offsets, parent, alpha) -> OracleTree:
     L = np.zeros((T, H_v), np.float64)
     order = np.zeros(T, np.uint8)
     status = np.zeros(B, np.int32)
-    rc = lib.treewy_oracle_prepare(ctypes.c_int32(B), ctypes.c_int32(H_v), _ptr(off), _ptr(par),
+    Td = T if T_declared is None else int(T_declared)
+    assert 0 <= Td <= T
+    rc = lib.treewy_oracle_prepare(ctypes.c_int32(B), ctypes.c_int32(Td), ctypes.c_int32(H_v), _ptr(off), _ptr(par),
                                    _ptr(al), _ptr(depth), _ptr(mask), _ptr(L), _ptr(order),
                                    _ptr(status))
     assert rc == 0
@@ -109,7 +114,7 @@ def prepare(node_offsets, parent, alpha) -> OracleTree:
 
 
 def verify_commit(node_offsets, parent, S0, q, k, v, alpha, beta, accepted,
-                  want_snapshots: bool = False) -> OracleResult:
+                  want_snapshots: bool = False, T_declared: int | None = None) -> OracleResult:
     """Outputs, pseudo-values and the committed state by walking Eq. 1 along every path."""
     lib = _load()
     off = _arr(node_offsets, np.int32)
@@ -133,7 +138,8 @@ def verify_commit(node_offsets, parent, S0, q, k, v, alpha, beta, accepted,
     Snap = np.zeros((T, H_v, d_v, d_k), np.float64) if want_snapshots else None
     status = np.zeros(B, np.int32)
     rc = lib.treewy_oracle_verify_commit(
-        ctypes.c_int32(B), ctypes.c_int32(H_v), ctypes.c_int32(H_qk), ctypes.c_int32(d_k),
+        ctypes.c_int32(B), ctypes.c_int32(T if T_declared is None else int(T_declared)),
+        ctypes.c_int32(H_v), ctypes.c_int32(H_qk), ctypes.c_int32(d_k),
         ctypes.c_int32(d_v), _ptr(off), _ptr(par), _ptr(S0), _ptr(q), _ptr(k), _ptr(v), _ptr(al),
         _ptr(be), _ptr(acc), _ptr(O), _ptr(U), _ptr(Sc), _ptr(Snap), _ptr(status))
     if rc != 0:

@@ -64,7 +64,7 @@ PATHS = {
 
 
 @pytest.mark.parametrize("name", sorted(PATHS))
-def test_offsets_past_the_declared_node_count_are_flagged_and_skipped(name):
+def test_offsets_past_the_declared_node_count_are_flagged_and_skipped(oracle, name):
     from paper_2608_20961_b200 import binding as tw
     cid, kw, hint = PATHS[name]
     w = wl.make_workload(cid, **kw)
@@ -77,6 +77,14 @@ def test_offsets_past_the_declared_node_count_are_flagged_and_skipped(name):
     got = _run(w, path, T_decl=T_decl, hint=hint)
     bad = [b for b in range(w.B) if off[b + 1] > T_decl]
     assert bad and bad[0] >= cut
+    # the oracle restates the rule: same status words
+    oracle.set_max_nodes(128 if name == "wide" else 64)
+    try:
+        ref = oracle.verify_commit(w.node_offsets.numpy(), w.parent.numpy(), pu.f64(w.S0), pu.f64(w.q), pu.f64(w.k),
+                                   pu.f64(w.v), pu.f64(w.alpha), pu.f64(w.beta), w.accepted.numpy(), T_declared=T_decl)
+    finally:
+        oracle.set_max_nodes(64)
+    assert list(ref.seq_status) == list(got["status"])
     for b in range(w.B):
         sl = slice(off[b], off[b + 1])
         if b in bad:

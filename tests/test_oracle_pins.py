@@ -325,6 +325,28 @@ def test_malformed_sequences_are_flagged_and_skipped(oracle):
     assert list(tr.seq_status) == [oracle.SEQ_TOO_MANY_NODES]
 
 
+def test_node_ranges_outside_the_packed_arrays_are_flagged_and_skipped(oracle):
+    """The packed layout's own rule (the paper packs nothing): a sequence whose range of node_offsets is
+    negative, runs backwards or ends past the T packed nodes the tree declares is malformed; the
+    sequences around it are computed as if it were not there."""
+    r = rng(17)
+    trees = [[-1, 0, 1], [-1, 0, 0, 1], [-1, 0]]
+    w = draw(r, trees, 1, 1, 4, 4)
+    good = oracle.verify_commit(**w)
+    cut = oracle.verify_commit(**w, T_declared=8)              # sequence 2 = [7, 9) sticks out of 8 nodes
+    assert list(cut.seq_status) == [0, 0, oracle.SEQ_BAD_OFFSETS]
+    assert np.array_equal(cut.O[:7], good.O[:7]) and np.all(cut.O[7:] == 0) and np.all(cut.S_commit[2] == 0)
+    assert np.array_equal(cut.S_commit[:2], good.S_commit[:2])
+    tr = oracle.prepare(w["node_offsets"], w["parent"], w["alpha"], T_declared=8)
+    assert list(tr.seq_status) == [0, 0, oracle.SEQ_BAD_OFFSETS] and np.all(tr.depth[7:] == -1)
+    back = dict(w, node_offsets=np.array([0, 3, 2, 9], np.int32))   # sequence 1 runs backwards
+    res = oracle.verify_commit(**back)
+    assert res.seq_status[1] == oracle.SEQ_BAD_OFFSETS and res.seq_status[0] == 0
+    assert np.array_equal(res.O[:3], good.O[:3])
+    neg = dict(w, node_offsets=np.array([-1, 3, 7, 9], np.int32))
+    assert oracle.verify_commit(**neg).seq_status[0] == oracle.SEQ_BAD_OFFSETS
+
+
 # ------------------------------------------------------------------ trees of more than 64 nodes
 
 def test_wide_trees_chain_and_closed_form(oracle):
