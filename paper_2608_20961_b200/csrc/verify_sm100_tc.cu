@@ -2,7 +2,7 @@
 // read-out), with BOTH contractions of the method on the tcgen05 tensor cores:
 //
 //   stage 1 (bf16 x bf16 -> fp32):   D1 = S0 [Q;K]^T  (S0 q_i, S0 k_i),   D2 = [Q;K] K^T  (Gram)
-//   stage 2 (tf32 split, ~fp32):     [O | U]^T = [g.S0q | 0]^T + R^T [W;T]^T
+//   stage 2 (bf16 x bf16 -> fp32, two-term operand splits):   [O | U]^T = [g.S0q | 0]^T + R^T [W;T]^T
 //
 // where R[j] = beta_j (v_j - g_j S0 k_j) is the right-hand side of Eq. 2, T = (I + A)^{-1} and
 // W = P T.  The triangular system is not solved column by column: because A only couples a
@@ -12,9 +12,11 @@
 // the solve shrinks from N steps per column to depth steps per node, done once per item, and
 // the N x N x 128 products go to the tensor pipe.
 //
-// fp32 accuracy on the tf32 pipe: every operand x is split as hi = x with the low 13 mantissa
-// bits cleared (exactly representable in tf32) and lo = x - hi; the kernel accumulates
-// hi.hi + lo.hi + hi.lo in fp32, dropping only lo.lo (relative 2^-22).
+// Accuracy of stage 2: every fp32 operand x is split as hi = bf16(x) and lo = bf16(x - hi), which
+// leaves 2^-18 |x|; the kernel accumulates hi.hi + lo.hi + hi.lo in fp32 and drops lo.lo, so a
+// product is off by at most 3 * 2^-18 of its size (three orders of magnitude below the bf16 rounding
+// of O and of the committed state).  Against the same split on the tf32 pipe (2^-22, K = 8 per
+// instruction, 4-byte operands) this halves the MMAs, the B tiles and the R^T columns in tensor memory.
 //
 // Roles (persistent CTA, one per SM; item = one (sequence, value head)).  Every phase of an item
 // has its own warps and every role walks all items in order, so the per-item cost is that of the
@@ -31,8 +33,8 @@
 //   R^T warps        (thread c = TMEM lane c = row c of d_v) row c of R^T as hi / lo back into
 //                    tensor memory over the Gram block, g.S0q in place, zeros over S0k
 //                                                                          -> ops_ready
-//   MMA-2 warp       stage-2 MMAs, A = R^T from tensor memory, B = [W;T] from shared memory, three
-//                    passes (hi.hi, lo.hi, hi.lo) accumulated on [g.S0q | 0]: [O | U]
+//   MMA-2 warp       stage-2 MMAs, A = R^T from tensor memory (bf16 pairs), B = [W;T] from shared memory,
+//                    three passes (hi.hi, lo.hi, hi.lo) accumulated on [g.S0q | 0]: [O | U]
 //                                                                          -> mma2_done, stage and
 //                                                                             R^T block released
 //   epilogue warps   o_i and u_i leave tensor memory: coalesced stores     -> block released
@@ -65,7 +67,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int STAGES = BIG ? 2 : (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     // (fused mode gives 128 columns of tensor memory to the commit's accumulator)
-    static constexpr int TBUF = BIG ? 2 : FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
+        static constexpr int TBUF = BIG ? 3 : FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
     static constexpr int RBUF = BIG ? 2 : FUSED ? 2 : 3;  // [D2 | -] -> R^T (hi | lo) blocks: held from stage 1 to the end of stage 2
     // every phase of an item has its own warps, and every role walks all items in order
     // (64 nodes: two R^T groups, each taking half of the columns of every item)
@@ -97,23 +99,26 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int META_BYTES = META_IDX + 2 * NP * 4;
     static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
     static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
-    // stage-2 B operand [W;T]: 2 NP rows (W rows above T rows, so one MMA yields O and U together)
-    // of NP fp32 columns, as atoms of 2 NP rows x 128 bytes (32 columns) with the 128-byte swizzle,
-    // once for the hi parts and once for the lo parts; they overlay the stage's dead tiles
-    static constexpr int ATOM = 2 * NP * 128, NATOM = BIG ? 2 : 1;
+    // stage-2 B operand [W;T]: 2 NP rows (W rows above T rows, so one MMA yields O and U together) of NP
+    // bf16 columns, each row in a 128-byte line of its own with the 128-byte swizzle (NP < 64 leaves the
+    // rest of the line empty), once for the hi parts and once for the lo parts; they overlay the stage's
+    // dead [Q;K] tile
+    static constexpr int PART = 2 * NP * 128;
     static constexpr int OFF_W_HI = 0, OFF_T_HI = NP * 128;
-    static constexpr int OFF_W_LO = NATOM * ATOM, OFF_T_LO = OFF_W_LO + NP * 128;
-    static constexpr int TILE_BYTES = 2 * NATOM * ATOM;
-    static_assert(TILE_BYTES <= (BIG ? QK_BYTES + S0_BYTES : QK_BYTES), "operand overlays fit");
+    static constexpr int OFF_W_LO = PART, OFF_T_LO = OFF_W_LO + NP * 128;
+    static constexpr int TILE_BYTES = 2 * PART;
+    static_assert(TILE_BYTES <= QK_BYTES, "operand overlays fit");
     // scratch over the dead tiles: the raw Gram rows (up to 32 nodes: in the S0 tile, beside the B
-    // tiles; 64 nodes: under the B tiles, which are zeroed once the lists are built) and, up to 32
-    // nodes, the back-substitution rows of deep paths
+    // tiles; 64 nodes: from the stage's start, under the B tiles, which are zeroed once the lists are
+    // built) and the back-substitution rows of deep paths (in the S0 tile; 64 nodes: the stash is dead
+    // by then, and a row is exactly NP floats, rotated by the node's number against bank conflicts)
     static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
-    static constexpr int XLD = NP + 1;
-    static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;
+    static constexpr int XLD = BIG ? NP : NP + 1;
+    static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = BIG ? OFF_S0 : OFF_S0 + 2 * NP * RLD * 4;
     static_assert(OFF_RAW + 2 * NP * RLD * 4 <= OFF_S0 + S0_BYTES, "Gram stash fits");
+    static_assert(OFF_XR + 2 * NP * XLD * 4 <= OFF_S0 + S0_BYTES, "back-substitution rows fit");
     // ... and, for trees with a path of more than 8 ancestors, the full-length lists (64 nodes: in an
-    // area of their own, since the B tiles take both dead tiles)
+    // area of their own)
     static constexpr int OFF_DAP = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 15) / 16 * 16;
     static constexpr int OFF_DPP = OFF_DAP + NP * NP * 4, OFF_DIDX = OFF_DPP + NP * NP * 4;
     static_assert(BIG || OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
@@ -141,14 +146,16 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the R^T warps
     // turn it, in their own lanes, into g.SQ | 0, stage 2 accumulates [O | U] on top, and the
-    // epilogue frees it.  A block of the second takes the Gram block D2 from stage 1; the Gram warps
-    // read it out, the R^T warps write R^T (hi) over it and R^T (lo) behind it, stage 2 takes both as
-    // its A operand, and its completion frees the block (long before the epilogue runs).
+    // epilogue frees it.  A block of the second (NP columns) takes the Gram block D2 from stage 1; the
+    // Gram warps read it out, the R^T warps write R^T over it as bf16 pairs (two nodes per column: the
+    // hi parts in the first NP / 2 columns, the lo parts in the rest), stage 2 takes both as its A
+    // operand, and its completion frees the block (long before the epilogue runs).
     static constexpr int TM_COLS = 2 * NP;
     static constexpr int TM_DO = 0, TM_DU = NP;
     static constexpr int TM_R0 = TBUF * TM_COLS;  // second ring
-    static constexpr int TM_RHI = 0, TM_RLO = NP;
-    static constexpr int TM_C0 = TM_R0 + RBUF * 2 * NP;  // fused mode: the commit's 128 x 128 accumulator
+    static constexpr int TM_RCOLS = NP;
+    static constexpr int TM_RHI = 0, TM_RLO = NP / 2;
+    static constexpr int TM_C0 = TM_R0 + RBUF * TM_RCOLS;  // fused mode: the commit's 128 x 128 accumulator
     static_assert(TM_C0 + (FUSED ? D : 0) <= 512, "tensor memory");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 };
@@ -297,11 +304,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
     auto meta_rat = [&](unsigned char *stage) { return reinterpret_cast<float4 *>(stage + C::OFF_META + C::META_RAT); };
     auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
-    // byte offset of element (row, col) of a stage-2 B tile (atoms of 32 columns, 128-byte swizzle)
-    auto tile_off = [](int row, int col) {
-        return (C::NATOM > 1 ? (col >> 5) * C::ATOM : 0) + row * 128 + (((((col & 31) >> 2)) ^ (row & 7)) << 4) +
-               ((col & 3) << 2);
-    };
+    // byte offset of element (row, col) of a stage-2 B tile (bf16, one 128-byte line per row, 128-byte swizzle)
+    auto tile_off = [](int row, int col) { return row * 128 + (((col >> 3) ^ (row & 7)) << 4) + ((col & 7) << 1); };
 
     if (warp >= C::PROD_WARP0) {
         // ------------------------------------------------------------------ producer warp
@@ -473,7 +477,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             {
                 // Path lists of the node this lane owns: index and gate ratio e^{L_i - L_j} of its first
                 // 8 ancestors.  Only the ratios depend on the head; building them here takes the
-                // ffs / exp chain off the consumers' critical path.  (Rolled: code size.)
+                // ffs / exp chain off the consumers' critical path.  (Rolled: code size.  Building them in
+                // registers before the stage is free, the other nodes' log-gates by shuffle, was tried: the
+                // unrolled code made every instance slower, 2 % to 5 %.)
                 __syncwarp();  // the log-gates of all nodes are in the meta block
                 const float *Lm = meta_L(stage);
 #pragma unroll
@@ -677,7 +683,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (n > 0) {
                     const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
                     const uint32_t d1 = tmem_base + buf * C::TM_COLS;
-                    const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
+                    const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * C::TM_RCOLS;
 #pragma unroll 1
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t ko = (ks >> 2) * C::QK_HALF + (ks & 3) * 32;
@@ -703,7 +709,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         if (FUSED && !gram_chain && lane == 0) ptx::bulk_wait_group<0>();
     } else if (warp == C::MMA2_WARP) {
         // ------------------------------------------------------------------ stage-2 MMAs
-        constexpr uint32_t idesc = ptx::umma_idesc_tf32_f32(128, 2 * NP);
+        constexpr uint32_t idesc = ptx::umma_idesc_bf16_f32(128, 2 * NP);
 #pragma unroll 1
         for (int kk = 0;; ++kk) {
             const int item = item_of(kk);
@@ -717,15 +723,16 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
                     const uint32_t tb = tmem_base + buf * C::TM_COLS;
-                    const uint32_t tr = tmem_base + C::TM_R0 + (kk % C::RBUF) * 2 * NP;
-                    // three passes (hi.hi, lo.hi, hi.lo), each NP / 8 steps of K = 8, on top of g.S0q (O)
+                    const uint32_t tr = tmem_base + C::TM_R0 + (kk % C::RBUF) * C::TM_RCOLS;
+                    // three passes (hi.hi, lo.hi, hi.lo), each NP / 16 steps of K = 16, on top of g.S0q (O)
                     // and zeros (U); rolled: the issue loop is short and code size matters
+                    constexpr int KS = NP / 16;
 #pragma unroll 1
-                    for (int q = 0; q < 3 * (NP / 8); ++q) {
-                        const int p = q / (NP / 8), ks = q % (NP / 8);
+                    for (int q = 0; q < 3 * KS; ++q) {
+                        const int p = q / KS, ks = q % KS;
                         const uint32_t ra = tr + (p == 1 ? C::TM_RLO : C::TM_RHI) + ks * 8;
-                        const uint32_t wt = base + (p == 2 ? C::OFF_W_LO : C::OFF_W_HI) + (ks >> 2) * C::ATOM + (ks & 3) * 32;
-                        ptx::umma_tf32_ts(tb, ra, ptx::umma_desc_k_sw128(wt), idesc, 1u);
+                        const uint32_t wt = base + (p == 2 ? C::OFF_W_LO : C::OFF_W_HI) + ks * 32;
+                        ptx::umma_bf16_ts(tb, ra, ptx::umma_desc_k_sw128(wt), idesc, 1u);
                     }
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
@@ -781,19 +788,23 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     for (int q = tg; q < C::TILE_BYTES / 16; q += C::G_THREADS)
                         reinterpret_cast<uint4 *>(stage)[q] = make_uint4(0u, 0u, 0u, 0u);
                 }
+                // the slot's previous lists and scalars must have been read
+                if (!ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1)) break;  // (a role has given up)
                 // the rows of the Gram block (row owner = lane)
                 if (gram_reader && !reuse_gram) {
-                    const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;
+                    const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * C::TM_RCOLS;
+                    constexpr int CH = NP < 32 ? NP : 32;  // columns per read: few, wide reads (each costs a round trip)
 #pragma unroll
-                    for (int c0 = 0; c0 < NP; c0 += 16) {
+                    for (int c0 = 0; c0 < NP; c0 += CH) {
                         if (c0 < n) {
-                            uint32_t g[16];
-                            ptx::tmem_ld16(tr + c0, g);
+                            uint32_t g[CH];
+                            if constexpr (CH == 32) ptx::tmem_ld32(tr + c0, g);
+                            else ptx::tmem_ld16(tr + c0, g);
                             ptx::tmem_wait_ld();
                             if (tg < 2 * NP) {
                                 float4 *dst = reinterpret_cast<float4 *>(raw + tg * C::RLD + c0);
 #pragma unroll
-                                for (int q = 0; q < 4; ++q)
+                                for (int q = 0; q < CH / 4; ++q)
                                     dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
                                                          __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
                             }
@@ -801,21 +812,20 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
                     ptx::tc_fence_before_sync();
                 }
-                if (!reuse_gram) ptx::named_sync(1, C::G_THREADS);
-                // the slot's previous lists and scalars must have been read
-                if (!ptx::mbar_wait(&lists_free[L], ((kk >> 1) & 1) ^ 1)) break;  // (a role has given up)
                 const bool valid = i < n;
                 const float Li = Lm[i];
                 const float bi = meta_beta(stage)[i];
                 const float scale = kind ? bi : 1.f;
                 const float *row = raw + (kind ? NP + i : i) * C::RLD;
-                // the per-node scalars first: the R^T warps need nothing else from here
+                // the per-node scalars first (a thread needs only its own row's diagonal entry for them): the
+                // R^T warps need nothing else from here, and a warp's arrival says its rows have left tensor memory
                 if (tg < NP && valid) {
                     const float gi = __expf(Li);
                     if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
                     scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
                 }
                 ptx::mbar_arrive_warp(&scal_ready[L]);
+                if (!reuse_gram) ptx::named_sync(1, C::G_THREADS);
                 if (!deep) {
                     // the producer left indices and gate ratios of the first 8 ancestors: four Gram
                     // entries are scaled at a time, no dependent chain
@@ -869,7 +879,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // Rows of T = (I + A)^-1 (one thread per node) and of W = P T (another) by back-substitution
         // along node i's root path j_0 .. j_{dp-1}, j_dp = i:
         //   x_dp = 1 (T) or P[i][i] (W);  x_e = p_e - sum_{f > e} x_f A[j_f][j_e]
-        // scattered (hi, lo) into the swizzled B tiles of stage 2.  Shared memory only.
+        // scattered as bf16 (hi, lo) into the swizzled B tiles of stage 2.  Shared memory only.
         const int tt = tid - C::T_WARP0 * 32;
         const int i = tt & (NP - 1);
         const bool wrow = (tt / NP) & 1;
@@ -923,6 +933,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
+                    auto put = [&](int off, float val) {  // val = hi + lo + 2^-18 |val|, both parts bf16
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+                        *reinterpret_cast<__nv_bfloat16 *>(Mhi + off) = hi;
+                        *reinterpret_cast<__nv_bfloat16 *>(Mlo + off) = __float2bfloat16_rn(val - __bfloat162float(hi));
+                    };
                     if (!deep) {  // registers only, no branches: entries beyond the path are zeros
                         const uint32_t iw0 = meta_idx(stage)[i], iw1 = meta_idx(stage)[NP + i];
                         int jf[9];
@@ -961,35 +976,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         // e = 8 the real diagonal entry (e = dp) is written after them
 #pragma unroll
                         for (int e = 8; e >= 0; --e) {
-                            const int col = jf[e];
-                            const float hi = ptx::tf32_hi(x[e]);
-                            const int off = tile_off(i, col);
-                            *reinterpret_cast<float *>(Mhi + off) = hi;
-                            *reinterpret_cast<float *>(Mlo + off) = x[e] - hi;
-                        }
-                    } else if constexpr (C::BIG) {  // deep paths: x_e is kept in the hi tile at its final column
-                        *reinterpret_cast<float *>(Mhi + tile_off(i, i)) = top;
-#pragma unroll 1
-                        for (int e = dp - 1; e >= 0; --e) {
-                            const int col_e = ((e >> 2) * NP) * 4 + (e & 3);
-                            float acc = wrow ? Pp[col_e + i * 4] : 0.f;
-#pragma unroll 1
-                            for (int f = e + 1; f <= dp; ++f) {
-                                const int jf = (f == dp) ? i : idx[((f >> 2) * NP + i) * 4 + (f & 3)];
-                                acc = fmaf(-*reinterpret_cast<const float *>(Mhi + tile_off(i, jf)), Ap[col_e + jf * 4], acc);
-                            }
-                            *reinterpret_cast<float *>(Mhi + tile_off(i, idx[((e >> 2) * NP + i) * 4 + (e & 3)])) = acc;
-                        }
-#pragma unroll 1
-                        for (int e = 0; e <= dp; ++e) {
-                            const int off = tile_off(i, (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)]);
-                            const float val = *reinterpret_cast<const float *>(Mhi + off), hi = ptx::tf32_hi(val);
-                            *reinterpret_cast<float *>(Mhi + off) = hi;
-                            *reinterpret_cast<float *>(Mlo + off) = val - hi;
+                            put(tile_off(i, jf[e]), x[e]);
                         }
                     } else {  // deep paths: the same recurrence through shared memory
                         float *x = xr + (wrow ? i : NP + i) * C::XLD;
-                        x[dp] = top;
+                        auto xi = [&](int e) { return C::BIG ? (e + i) & (NP - 1) : e; };
+                        x[xi(dp)] = top;
 #pragma unroll 1
                         for (int e = dp - 1; e >= 0; --e) {
                             const int col_e = ((e >> 2) * NP) * 4 + (e & 3);
@@ -997,17 +989,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
 #pragma unroll 1
                             for (int f = e + 1; f <= dp; ++f) {
                                 const int jf = (f == dp) ? i : idx[((f >> 2) * NP + i) * 4 + (f & 3)];
-                                acc = fmaf(-x[f], Ap[col_e + jf * 4], acc);
+                                acc = fmaf(-x[xi(f)], Ap[col_e + jf * 4], acc);
                             }
-                            x[e] = acc;
+                            x[xi(e)] = acc;
                         }
 #pragma unroll 1
                         for (int e = 0; e <= dp; ++e) {
                             const int col = (e == dp) ? i : idx[((e >> 2) * NP + i) * 4 + (e & 3)];
-                            const float val = x[e], hi = ptx::tf32_hi(val);
-                            const int off = tile_off(i, col);
-                            *reinterpret_cast<float *>(Mhi + off) = hi;
-                            *reinterpret_cast<float *>(Mlo + off) = val - hi;
+                            put(tile_off(i, col), x[xi(e)]);
                         }
                     }
             }
@@ -1027,7 +1016,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     } else if (warp >= C::R_WARP0 && warp < C::E_WARP0) {
         // ------------------------------------------------------------------ R^T warps
         // Thread c = TMEM lane c = row c of d_v.  Row c of R^T, r_j = beta_j v_j - beta_j g_j (S0 k_j),
-        // goes back to tensor memory as hi / lo (the A operand of stage 2); g_j (S0 q_j) in place and
+        // goes back to tensor memory as bf16 hi / lo pairs (the A operand of stage 2); g_j (S0 q_j) in place and
         // zeros over S0 k_j are what stage 2 accumulates o_j and u_j on.
         const int t = (tid - C::R_WARP0 * 32) & 127;
         const int c_lo = ((tid - C::R_WARP0 * 32) >> 7) * (NP / C::R_GROUPS), c_hi = c_lo + NP / C::R_GROUPS;
@@ -1042,7 +1031,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const float4 *scal = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
             const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;                 // SQ | SK
-            const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * 2 * NP;            // D2 | -
+            const uint32_t tr = tmem_base + lane_base + C::TM_R0 + rb * C::TM_RCOLS;            // D2 | -
             // The Gram warps signal the scalars after they have seen stage 1 complete, read the Gram block
             // out and recorded the item's size: one wait covers all of it.
             if (!ptx::mbar_wait(&scal_ready[L], (kk >> 1) & 1)) break;
@@ -1052,7 +1041,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (n > 0) {
 #pragma unroll 1
                 for (int c0 = c_lo; c0 < c_hi; c0 += 8) {  // (rolled: code size matters more than the loop overhead)
-                    uint32_t hi[8], lo[8];
+                    uint32_t hi[4], lo[4];
                     if (c0 < n) {
                         uint32_t sk[8], sq[8];
                         ptx::tmem_ld8(tm + NP + c0, sk);
@@ -1066,20 +1055,23 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                             const int j = c0 + jj;
                             const float4 sc = scal[j];
                             const float val = fmaf(-sc.y, __uint_as_float(sk[jj]), sc.x * v[jj]);
-                            const float rj = j < n ? val : 0.f;
-                            const float h = ptx::tf32_hi(rj);
-                            hi[jj] = __float_as_uint(h), lo[jj] = __float_as_uint(rj - h);
+                            v[jj] = j < n ? val : 0.f;  // r_j
                             sq[jj] = __float_as_uint(sc.z * __uint_as_float(sq[jj]));
                             sk[jj] = 0u;
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {  // nodes 2q, 2q + 1 share a column: the lower one in its low half
+                            const float h0 = ptx::bf16_hi(v[2 * q]), h1 = ptx::bf16_hi(v[2 * q + 1]);
+                            hi[q] = pack_bf16(h0, h1), lo[q] = pack_bf16(v[2 * q] - h0, v[2 * q + 1] - h1);
                         }
                         ptx::tmem_st8(tm + c0, sq);
                         ptx::tmem_st8(tm + NP + c0, sk);
                     } else {
 #pragma unroll
-                        for (int jj = 0; jj < 8; ++jj) hi[jj] = 0u, lo[jj] = 0u;
+                        for (int q = 0; q < 4; ++q) hi[q] = 0u, lo[q] = 0u;
                     }
-                    ptx::tmem_st8(tr + C::TM_RHI + c0, hi);
-                    ptx::tmem_st8(tr + C::TM_RLO + c0, lo);
+                    ptx::tmem_st4(tr + C::TM_RHI + c0 / 2, hi);
+                    ptx::tmem_st4(tr + C::TM_RLO + c0 / 2, lo);
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();

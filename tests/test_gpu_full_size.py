@@ -41,9 +41,11 @@ def test_tensor_core_and_simt_kernels_agree_at_full_size():
     w = wl.make_workload(2, B=64)
     a = pu.run_gpu(w, torch.float32, generic=False, want_s32=False)
     b = pu.run_gpu(w, torch.float32, generic=True, want_s32=False)
+    # the tensor-core kernel's second product takes its operands as two-term bf16 splits and drops the
+    # lo.lo term: 3 * 2^-18 = 1.1e-5 of |r_j| |T_ij| per product at worst, summed over a root path
     scale = float(b["O"].abs().max())
-    assert float((a["O"] - b["O"]).abs().max()) <= 1e-5 * scale
-    assert float((a["U"] - b["U"]).abs().max()) <= 1e-5 * float(b["U"].abs().max())
+    assert float((a["O"] - b["O"]).abs().max()) <= 5e-5 * scale
+    assert float((a["U"] - b["U"]).abs().max()) <= 5e-5 * float(b["U"].abs().max())
 
 
 def test_full_size_half_u_is_the_rounded_u():
