@@ -112,10 +112,14 @@ template <int NP, bool FUSED> struct VtCfg {
     // tiles; 64 nodes: from the stage's start, under the B tiles, which are zeroed once the lists are
     // built) and the back-substitution rows of deep paths (in the S0 tile; 64 nodes: the stash is dead
     // by then, and a row is exactly NP floats, rotated by the node's number against bank conflicts)
-    static constexpr int RLD = NP + 4;  // row stride of the raw Gram stash (floats)
+    // (64 nodes: the stash is exactly the [Q;K] tile, rows of NP floats with their 16-byte columns swizzled
+    // by the row number, so that the S0 tile is dead once stage 1 has read it and goes back to the
+    // producer right then, a stage-2 time before the rest of the stage; deep trees keep it for their rows)
+    static constexpr bool S0_EARLY = BIG;
+    static constexpr int RLD = BIG ? NP : NP + 4;  // row stride of the raw Gram stash (floats)
     static constexpr int XLD = BIG ? NP : NP + 1;
     static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = BIG ? OFF_S0 : OFF_S0 + 2 * NP * RLD * 4;
-    static_assert(OFF_RAW + 2 * NP * RLD * 4 <= OFF_S0 + S0_BYTES, "Gram stash fits");
+    static_assert(OFF_RAW + 2 * NP * RLD * 4 <= (BIG ? QK_BYTES : OFF_S0 + S0_BYTES), "Gram stash fits");
     static_assert(OFF_XR + 2 * NP * XLD * 4 <= OFF_S0 + S0_BYTES, "back-substitution rows fit");
     // ... and, for trees with a path of more than 8 ancestors, the full-length lists (64 nodes: in an
     // area of their own)
@@ -141,7 +145,7 @@ template <int NP, bool FUSED> struct VtCfg {
     // work list of a launch that takes one size class of a mixed batch: the CTA's units of that class
     // (up to CT_CAP of them; a longer list is walked whole), then 32 warp counts
     static constexpr int CT_CAP = 1024;
-    static constexpr int OFF_CTAB = OFF_BAR + (3 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16;
+    static constexpr int OFF_CTAB = OFF_BAR + (4 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16;
     static constexpr int SMEM_BYTES = OFF_CTAB + CT_CAP * 2 + 32 * 4 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the R^T warps
@@ -200,7 +204,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *scal_ready = lists_free + C::SLOTS;      // Gram warps -> R^T warps: per-node scalars written
     uint64_t *upd_done = scal_ready + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
     uint64_t *cmma_done = upd_done + C::STAGES;        // fused mode: the commit's rank-P product has finished
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(cmma_done + 1);
+    uint64_t *s0_empty = cmma_done + 1;                // 64 nodes: the S0 tile of a stage may be refilled
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s0_empty + C::STAGES);
     int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -245,7 +250,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&lists_free[g], (C::R_THREADS + C::T_THREADS) / 32);
             ptx::mbar_init(&scal_ready[g], C::G_THREADS / 32);
         }
-        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32);
+        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32), ptx::mbar_init(&s0_empty[s], 1);
         ptx::mbar_init(cmma_done, 1);
         ptx::fence_barrier_init();
     }
@@ -304,6 +309,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
     auto meta_rat = [&](unsigned char *stage) { return reinterpret_cast<float4 *>(stage + C::OFF_META + C::META_RAT); };
     auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
+    // element (row, col) of the raw Gram stash
+    auto raw_at = [](int row, int col) {
+        return C::BIG ? row * C::RLD + ((((col >> 2) ^ (row & 15)) << 2) | (col & 3)) : row * C::RLD + col;
+    };
     // byte offset of element (row, col) of a stage-2 B tile (bf16, one 128-byte line per row, 128-byte swizzle)
     auto tile_off = [](int row, int col) { return row * 128 + (((col >> 3) ^ (row & 7)) << 4) + ((col & 7) << 1); };
 
@@ -416,11 +425,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, item0 * D, &full[s]);
         }  // (the q / k rows as well, one load away, was tried: the step got 0.2 % slower, workload 3 1 %)
         Pre cur = fetch(s);
+        bool s0_issued = early;  // the state tile of `cur` is in flight already
 #pragma unroll 1
         for (int kk = s;; kk += C::STAGES) {
             if (cur.item >= n_items) break;
             if (cur.item == a.skip_item) {  // test hook: this item's loads and their arrival never happen
                 cur = fetch(kk + C::STAGES);
+                s0_issued = false;
                 continue;
             }
             const Pre p = cur;
@@ -446,7 +457,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             // The copies are issued first and announced (expect_tx, with the warp's one arrival) last:
             // the phase cannot complete before that arrival, and the path lists below are written
             // while the data is on its way.
-            const bool tile_issued = early && kk == s;
+            const bool tile_issued = s0_issued;
             const bool need_tile = (!p.bad || p.plen >= 0) && !tile_issued;  // the state tile serves verify, commit or both
             const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
             if (lane == 0) {
@@ -503,6 +514,22 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 else ptx::mbar_arrive_expect_tx(&full[s], tx);
             }
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
+            s0_issued = false;
+            if constexpr (C::S0_EARLY) {
+                // the next item's state tile: the stage's S0 tile is free as soon as stage 1 has read it
+                if (cur.item < n_items && cur.item != a.skip_item && !cur.bad) {
+                    if (!ptx::mbar_wait(&s0_empty[s], (kk / C::STAGES) & 1)) {
+                        if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[cur.b], TREEWY_SEQ_TIMEOUT);
+                        break;
+                    }
+                    if (lane == 0) {
+                        ptx::mbar_expect_tx(&full[s], C::S0_BYTES);
+                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, cur.srow * D, &full[s]);
+                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, cur.srow * D, &full[s]);
+                    }
+                    s0_issued = true;
+                }
+            }
         }
     } else if (FUSED && warp >= C::COMMIT_WARP0 && warp < C::MMA1_WARP) {
         // ------------------------------------------------------------------ commit group (fused mode)
@@ -699,9 +726,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     // store must have read it by then)
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::umma_commit(&mma1_done[buf]);
+                    if (C::S0_EARLY && !gram_chain && meta_nlo(stage)[2] == 0) ptx::umma_commit(&s0_empty[s]);
                 } else {
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::mbar_arrive(&mma1_done[buf]);
+                    if (C::S0_EARLY && !gram_chain && meta_nlo(stage)[2] == 0) ptx::mbar_arrive(&s0_empty[s]);
                 }
             }
             __syncwarp();
@@ -719,6 +748,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (!ptx::mbar_wait(&ops_ready[buf], (kk / C::TBUF) & 1)) break;
             ptx::tc_fence_after_sync();
             const int n = meta_nlo(stage)[0];
+            const bool keeps_s0 = C::S0_EARLY && meta_nlo(stage)[2] != 0;  // a deep tree: its S0 tile goes back only now
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
@@ -736,10 +766,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
+                    if (keeps_s0) ptx::umma_commit(&s0_empty[s]);
                     ptx::umma_commit(&r_free[kk % C::RBUF]);
                 } else {
                     ptx::mbar_arrive(&mma2_done[buf]);
                     ptx::mbar_arrive(&empty[s]);
+                    if (keeps_s0) ptx::mbar_arrive(&s0_empty[s]);
                     ptx::mbar_arrive(&r_free[kk % C::RBUF]);
                 }
             }
@@ -802,10 +834,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                             else ptx::tmem_ld16(tr + c0, g);
                             ptx::tmem_wait_ld();
                             if (tg < 2 * NP) {
-                                float4 *dst = reinterpret_cast<float4 *>(raw + tg * C::RLD + c0);
 #pragma unroll
                                 for (int q = 0; q < CH / 4; ++q)
-                                    dst[q] = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
+                                    *reinterpret_cast<float4 *>(raw + raw_at(tg, c0 + 4 * q)) = make_float4(__uint_as_float(g[4 * q]), __uint_as_float(g[4 * q + 1]),
                                                          __uint_as_float(g[4 * q + 2]), __uint_as_float(g[4 * q + 3]));
                             }
                         }
@@ -816,12 +847,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const float Li = Lm[i];
                 const float bi = meta_beta(stage)[i];
                 const float scale = kind ? bi : 1.f;
-                const float *row = raw + (kind ? NP + i : i) * C::RLD;
+                const int rrow = kind ? NP + i : i;
                 // the per-node scalars first (a thread needs only its own row's diagonal entry for them): the
                 // R^T warps need nothing else from here, and a warp's arrival says its rows have left tensor memory
                 if (tg < NP && valid) {
                     const float gi = __expf(Li);
-                    if (!reuse_gram) gram_diag = raw[i * C::RLD + i];
+                    if (!reuse_gram) gram_diag = raw[raw_at(i, i)];
                     scal[i] = make_float4(bi, bi * gi, gi, gram_diag);
                 }
                 ptx::mbar_arrive_warp(&scal_ready[L]);
@@ -836,7 +867,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         const float4 rt = meta_rat(stage)[hf * NP + i];
                         if (!reuse_gram) {
                             const uint32_t iw = meta_idx(stage)[hf * NP + i];
-                            gram4[q] = make_float4(row[iw & 255u], row[(iw >> 8) & 255u], row[(iw >> 16) & 255u], row[iw >> 24]);
+                            gram4[q] = make_float4(raw[raw_at(rrow, iw & 255u)], raw[raw_at(rrow, (iw >> 8) & 255u)],
+                                                   raw[raw_at(rrow, (iw >> 16) & 255u)], raw[raw_at(rrow, iw >> 24)]);
                         }
                         float4 val;
                         val.x = scale * rt.x * gram4[q].x, val.y = scale * rt.y * gram4[q].y;
@@ -856,7 +888,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     for (int d = 0; m; ++d) {
                         const int j = m_ffs(m);
                         m &= m - 1;
-                        const float val = scale * __expf(Li - Lm[j]) * row[j];
+                        const float val = scale * __expf(Li - Lm[j]) * raw[raw_at(rrow, j)];
                         const int at = ((d >> 2) * NP + i) * 4 + (d & 3);
                         if (kind) Ap[at] = val;
                         else Pp[at] = val, idx[at] = (unsigned char)j;
