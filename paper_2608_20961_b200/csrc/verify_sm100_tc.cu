@@ -97,7 +97,13 @@ template <int NP, bool FUSED> struct VtCfg {
     // the ancestors' indices as [d / 4][node] words of four bytes
     static constexpr int META_RAT = NP * 16 + 16, META_IDX = META_RAT + 2 * NP * 16;
     static constexpr int META_BYTES = META_IDX + 2 * NP * 4;
-    static constexpr int OFF_PMETA = OFF_META + META_BYTES;  // PathMeta of the previous round's commit
+    // 64 nodes: the meta blocks are not part of the stage but a ring of their own, twice as deep, so that
+    // the producer writes an item's block (the path lists are 4 k cycles of one warp's time) while the
+    // stage is still busy with the item before, not after it has been handed back.  (The fused mode has
+    // room for such a ring too; it was tried and changed nothing there: its loads take as long as its lists.)
+    static constexpr bool META_RING = BIG;
+    static constexpr int OFF_PMETA = OFF_META + (META_RING ? 0 : META_BYTES);  // PathMeta of the previous round's commit
+    static constexpr int META_SLOTS = META_RING ? 2 * STAGES : STAGES, META_STRIDE = (META_BYTES + 15) / 16 * 16;
     static constexpr int STAGE_BYTES = (OFF_PMETA + (FUSED ? 128 : 0) + 1023) / 1024 * 1024;
     // stage-2 B operand [W;T]: 2 NP rows (W rows above T rows, so one MMA yields O and U together) of NP
     // bf16 columns, each row in a 128-byte line of its own with the 128-byte swizzle (NP < 64 leaves the
@@ -135,7 +141,8 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_DEEP = OFF_GP + SLOTS * GP_BYTES;  // 64 nodes: full-length lists of deep trees
-    static constexpr int OFF_EINFO = OFF_DEEP + DEEP_BYTES;      // (n, first node) of the item in a TMEM block
+    static constexpr int OFF_MRING = OFF_DEEP + DEEP_BYTES;      // 64 nodes: the ring of meta blocks
+    static constexpr int OFF_EINFO = OFF_MRING + (META_RING ? META_SLOTS * META_STRIDE : 0);  // (n, first node) of the item in a TMEM block
     // fused mode: operands of the commit's rank-P product, K-major without swizzle, K = 8 path nodes:
     // core matrices of 8 rows x 16 bytes, the two K halves COPS_LBO apart
     static constexpr int COPS_LBO = D * 16, COPS_TILE = 2 * COPS_LBO;
@@ -303,12 +310,17 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         K = kept;
     }
 
-    auto meta_mask = [&](unsigned char *stage) { return reinterpret_cast<unsigned long long *>(stage + C::OFF_META); };
-    auto meta_L = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 8); };
-    auto meta_beta = [&](unsigned char *stage) { return reinterpret_cast<float *>(stage + C::OFF_META + NP * 12); };
-    auto meta_nlo = [&](unsigned char *stage) { return reinterpret_cast<int *>(stage + C::OFF_META + NP * 16); };
-    auto meta_rat = [&](unsigned char *stage) { return reinterpret_cast<float4 *>(stage + C::OFF_META + C::META_RAT); };
-    auto meta_idx = [&](unsigned char *stage) { return reinterpret_cast<uint32_t *>(stage + C::OFF_META + C::META_IDX); };
+    // the meta block of item kk of this CTA
+    auto meta_of = [&](int kk) {
+        return C::META_RING ? smem + C::OFF_MRING + (kk % C::META_SLOTS) * C::META_STRIDE
+                            : smem + (kk % C::STAGES) * C::STAGE_BYTES + C::OFF_META;
+    };
+    auto meta_mask = [&](unsigned char *mt) { return reinterpret_cast<unsigned long long *>(mt); };
+    auto meta_L = [&](unsigned char *mt) { return reinterpret_cast<float *>(mt + NP * 8); };
+    auto meta_beta = [&](unsigned char *mt) { return reinterpret_cast<float *>(mt + NP * 12); };
+    auto meta_nlo = [&](unsigned char *mt) { return reinterpret_cast<int *>(mt + NP * 16); };
+    auto meta_rat = [&](unsigned char *mt) { return reinterpret_cast<float4 *>(mt + C::META_RAT); };
+    auto meta_idx = [&](unsigned char *mt) { return reinterpret_cast<uint32_t *>(mt + C::META_IDX); };
     // element (row, col) of the raw Gram stash
     auto raw_at = [](int row, int col) {
         return C::BIG ? row * C::RLD + ((((col >> 2) ^ (row & 15)) << 2) | (col & 3)) : row * C::RLD + col;
@@ -424,6 +436,37 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, item0 * D, &full[s]);
             ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, item0 * D, &full[s]);
         }  // (the q / k rows as well, one load away, was tried: the step got 0.2 % slower, workload 3 1 %)
+        // An item's meta block: node scalars, size and place, and the path lists of the node(s) a lane owns
+        // (index and gate ratio e^{L_i - L_j} of the first 8 ancestors; only the ratios depend on the head).
+        // Building the lists here takes the ffs / exp chain off the consumers' critical path.  (Rolled:
+        // code size.  Building them in registers, the other nodes' log-gates by shuffle, was tried: the
+        // unrolled code made every instance slower, 2 % to 5 %.)
+        auto write_meta = [&](const Pre &p, unsigned char *mt) {
+#pragma unroll
+            for (int r = 0; r < C::NPL; ++r) {
+                const int i = lane + 32 * r;
+                if (i < NP) meta_mask(mt)[i] = p.mk[r], meta_L(mt)[i] = p.Lv[r], meta_beta(mt)[i] = p.bv[r];
+            }
+            if (lane == 0)
+                meta_nlo(mt)[0] = p.bad ? 0 : p.n, meta_nlo(mt)[1] = p.lo, meta_nlo(mt)[2] = p.deep,
+                meta_nlo(mt)[3] = p.srow;
+            __syncwarp();  // the log-gates of all nodes are in the meta block
+            const float *Lm = meta_L(mt);
+#pragma unroll
+            for (int r = 0; r < C::NPL; ++r) {
+                const int i = lane + 32 * r;
+                mask_t m = (mask_t)p.mk[r] & ~((mask_t)1 << i);
+                float *ratp = reinterpret_cast<float *>(meta_rat(mt)) + i * 4;
+                unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(mt)) + i * 4;
+#pragma unroll 1
+                for (int d = 0; d < 8; ++d) {
+                    const int j = m ? m_ffs(m) : 0;
+                    const float rt = m ? __expf(p.Lv[r] - Lm[j]) : 0.f;
+                    if (i < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = rt, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
+                    m &= m - 1;
+                }
+            }
+        };
         Pre cur = fetch(s);
         bool s0_issued = early;  // the state tile of `cur` is in flight already
 #pragma unroll 1
@@ -435,20 +478,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 continue;
             }
             const Pre p = cur;
+            unsigned char *mt = meta_of(kk);
+            if constexpr (C::META_RING) write_meta(p, mt);  // the block of item kk - 2 * STAGES: long read
             if (p.bad && p.flag && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.bad);
             if (FUSED && p.pbad && p.h == 0 && lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], p.pbad);
             if (!ptx::mbar_wait(&empty[s], ((kk / C::STAGES) & 1) ^ 1)) {
                 if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[p.b], TREEWY_SEQ_TIMEOUT);
                 break;
             }
-#pragma unroll
-            for (int r = 0; r < C::NPL; ++r) {
-                const int i = lane + 32 * r;
-                if (i < NP) meta_mask(stage)[i] = p.mk[r], meta_L(stage)[i] = p.Lv[r], meta_beta(stage)[i] = p.bv[r];
-            }
-            if (lane == 0)
-                meta_nlo(stage)[0] = p.bad ? 0 : p.n, meta_nlo(stage)[1] = p.lo, meta_nlo(stage)[2] = p.deep,
-                meta_nlo(stage)[3] = p.srow;
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
@@ -485,29 +522,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                                   D * 4, &full[s]);
                 }
             }
-            {
-                // Path lists of the node this lane owns: index and gate ratio e^{L_i - L_j} of its first
-                // 8 ancestors.  Only the ratios depend on the head; building them here takes the
-                // ffs / exp chain off the consumers' critical path.  (Rolled: code size.  Building them in
-                // registers before the stage is free, the other nodes' log-gates by shuffle, was tried: the
-                // unrolled code made every instance slower, 2 % to 5 %.)
-                __syncwarp();  // the log-gates of all nodes are in the meta block
-                const float *Lm = meta_L(stage);
-#pragma unroll
-                for (int r = 0; r < C::NPL; ++r) {
-                    const int i = lane + 32 * r;
-                    mask_t m = (mask_t)p.mk[r] & ~((mask_t)1 << i);
-                    float *ratp = reinterpret_cast<float *>(meta_rat(stage)) + i * 4;
-                    unsigned char *idxp = reinterpret_cast<unsigned char *>(meta_idx(stage)) + i * 4;
-#pragma unroll 1
-                    for (int d = 0; d < 8; ++d) {
-                        const int j = m ? m_ffs(m) : 0;
-                        const float rt = m ? __expf(p.Lv[r] - Lm[j]) : 0.f;
-                        if (i < NP) ratp[(d >> 2) * NP * 4 + (d & 3)] = rt, idxp[(d >> 2) * NP * 4 + (d & 3)] = (unsigned char)j;
-                        m &= m - 1;
-                    }
-                }
-            }
+            if constexpr (!C::META_RING) write_meta(p, mt);  // (while the data is on its way)
             __syncwarp();
             if (lane == 0) {
                 if (tx == 0) ptx::mbar_arrive(&full[s]);
@@ -557,6 +572,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) {
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                 break;
@@ -685,15 +701,16 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) break;
-            const bool reuse_gram = pair_mode && (kk & 1) && meta_nlo(stage)[2] == 0;
-            const int n = gram_chain && reuse_gram ? 0 : meta_nlo(stage)[0];
+            const bool reuse_gram = pair_mode && (kk & 1) && meta_nlo(mt)[2] == 0;
+            const int n = gram_chain && reuse_gram ? 0 : meta_nlo(mt)[0];
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
             bool stored = false;
             if constexpr (FUSED) {
                 // the new state goes back to global memory while verification proceeds from this copy
                 if (!gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
-                    const int srow = meta_nlo(stage)[3];
+                    const int srow = meta_nlo(mt)[3];
                     ptx::tma_store_2d(&tmS0, 0, srow * D, stage + C::OFF_S0);
                     ptx::tma_store_2d(&tmS0, 64, srow * D, stage + C::OFF_S0 + C::S0_HALF);
                     ptx::bulk_commit_group();
@@ -726,11 +743,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     // store must have read it by then)
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::umma_commit(&mma1_done[buf]);
-                    if (C::S0_EARLY && !gram_chain && meta_nlo(stage)[2] == 0) ptx::umma_commit(&s0_empty[s]);
+                    if (C::S0_EARLY && !gram_chain && meta_nlo(mt)[2] == 0) ptx::umma_commit(&s0_empty[s]);
                 } else {
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::mbar_arrive(&mma1_done[buf]);
-                    if (C::S0_EARLY && !gram_chain && meta_nlo(stage)[2] == 0) ptx::mbar_arrive(&s0_empty[s]);
+                    if (C::S0_EARLY && !gram_chain && meta_nlo(mt)[2] == 0) ptx::mbar_arrive(&s0_empty[s]);
                 }
             }
             __syncwarp();
@@ -745,10 +762,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             if (!ptx::mbar_wait(&ops_ready[buf], (kk / C::TBUF) & 1)) break;
             ptx::tc_fence_after_sync();
-            const int n = meta_nlo(stage)[0];
-            const bool keeps_s0 = C::S0_EARLY && meta_nlo(stage)[2] != 0;  // a deep tree: its S0 tile goes back only now
+            const int n = meta_nlo(mt)[0];
+            const bool keeps_s0 = C::S0_EARLY && meta_nlo(mt)[2] != 0;  // a deep tree: its S0 tile goes back only now
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
@@ -796,6 +814,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
             float4 *Ap4 = reinterpret_cast<float4 *>(gp + C::GP_AP);
             float4 *Pp4 = reinterpret_cast<float4 *>(gp + C::GP_PP);
@@ -806,12 +825,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             ptx::tc_fence_after_sync();
             ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1);  // already complete: acquires the meta block
-            const int n = meta_nlo(stage)[0];
-            if (tg == 0) einfo[buf] = make_int2(n, meta_nlo(stage)[1]);
+            const int n = meta_nlo(mt)[0];
+            if (tg == 0) einfo[buf] = make_int2(n, meta_nlo(mt)[1]);
             if (n > 0) {
-                const float *Lm = meta_L(stage);
+                const float *Lm = meta_L(mt);
                 float *raw = reinterpret_cast<float *>(stage + C::OFF_RAW);
-                const bool deep = meta_nlo(stage)[2] != 0;  // some path of this tree has more than 8 ancestors
+                const bool deep = meta_nlo(mt)[2] != 0;  // some path of this tree has more than 8 ancestors
                 // second item of a pair: same tree, same [Q;K] rows; the Gram entries are in registers
                 const bool reuse_gram = pair_mode && (kk & 1) && !deep;
                 // zero the stage-2 B tiles (they overlay the dead [Q;K] tile; with 64 nodes they also cover
@@ -845,7 +864,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
                 const bool valid = i < n;
                 const float Li = Lm[i];
-                const float bi = meta_beta(stage)[i];
+                const float bi = meta_beta(mt)[i];
                 const float scale = kind ? bi : 1.f;
                 const int rrow = kind ? NP + i : i;
                 // the per-node scalars first (a thread needs only its own row's diagonal entry for them): the
@@ -864,9 +883,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
 #pragma unroll
                     for (int q = 0; q < HN; ++q) {
                         const int hf = tg / (2 * NP) + q * HSTEP;
-                        const float4 rt = meta_rat(stage)[hf * NP + i];
+                        const float4 rt = meta_rat(mt)[hf * NP + i];
                         if (!reuse_gram) {
-                            const uint32_t iw = meta_idx(stage)[hf * NP + i];
+                            const uint32_t iw = meta_idx(mt)[hf * NP + i];
                             gram4[q] = make_float4(raw[raw_at(rrow, iw & 255u)], raw[raw_at(rrow, (iw >> 8) & 255u)],
                                                    raw[raw_at(rrow, (iw >> 16) & 255u)], raw[raw_at(rrow, iw >> 24)]);
                         }
@@ -883,7 +902,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     float *Ap = reinterpret_cast<float *>(dl);
                     float *Pp = reinterpret_cast<float *>(dl + NP * NP * 4);
                     unsigned char *idx = dl + 2 * NP * NP * 4;
-                    mask_t m = valid ? (mask_t)meta_mask(stage)[i] & ~((mask_t)1 << i) : (mask_t)0;
+                    mask_t m = valid ? (mask_t)meta_mask(mt)[i] & ~((mask_t)1 << i) : (mask_t)0;
 #pragma unroll 1
                     for (int d = 0; m; ++d) {
                         const int j = m_ffs(m);
@@ -944,6 +963,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
             const float4 *Ap4 = reinterpret_cast<const float4 *>(gp + C::GP_AP);
             const float4 *Pp4 = reinterpret_cast<const float4 *>(gp + C::GP_PP);
@@ -953,15 +973,15 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 gave_up = true;
                 break;
             }
-            const int n = meta_nlo(stage)[0];  // (the Gram warps read the meta block before they signalled)
+            const int n = meta_nlo(mt)[0];  // (the Gram warps read the meta block before they signalled)
             if (n > 0 && tt < 2 * NP && i < n) {
-                const bool deep = meta_nlo(stage)[2] != 0;
+                const bool deep = meta_nlo(mt)[2] != 0;
                 const unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;  // full-length lists
                 const float *Ap = reinterpret_cast<const float *>(dl);
                 const float *Pp = reinterpret_cast<const float *>(dl + NP * NP * 4);
                 const unsigned char *idx = dl + 2 * NP * NP * 4;
                 float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
-                const int dp = m_popc((mask_t)meta_mask(stage)[i]) - 1;  // ancestors of node i
+                const int dp = m_popc((mask_t)meta_mask(mt)[i]) - 1;  // ancestors of node i
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
                     unsigned char *Mlo = stage + (wrow ? C::OFF_W_LO : C::OFF_T_LO);
@@ -971,7 +991,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         *reinterpret_cast<__nv_bfloat16 *>(Mlo + off) = __float2bfloat16_rn(val - __bfloat162float(hi));
                     };
                     if (!deep) {  // registers only, no branches: entries beyond the path are zeros
-                        const uint32_t iw0 = meta_idx(stage)[i], iw1 = meta_idx(stage)[NP + i];
+                        const uint32_t iw0 = meta_idx(mt)[i], iw1 = meta_idx(mt)[NP + i];
                         int jf[9];
                         float x[9], pe[8], co[9][8];
 #pragma unroll
@@ -1059,6 +1079,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (item >= n_items) break;
             const int s = kk % C::STAGES, buf = kk % C::TBUF, rb = kk % C::RBUF, L = kk & 1;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
+            unsigned char *mt = meta_of(kk);
             unsigned char *gp = smem + C::OFF_GP + L * C::GP_BYTES;
             const float4 *scal = reinterpret_cast<const float4 *>(gp + C::GP_SCAL);
             const __nv_bfloat16 *vs = reinterpret_cast<const __nv_bfloat16 *>(gp + C::GP_VS);
