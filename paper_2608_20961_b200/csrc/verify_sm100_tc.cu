@@ -220,22 +220,27 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     // share a q/k head, a CTA takes the heads two by two: both items of a pair have the same tree
     // and the same [Q;K] rows, so the second reuses the first one's Gram entries.
     const bool pair_mode = ((a.H_v / a.H_qk) & 1) == 0;
-    // The CTA's units (items, or pairs of them) are blockIdx.x, blockIdx.x + gridDim.x, ...: K of them.
-    // A launch that takes one size class of a mixed batch walks only the units of its class (ctab).
+    // The CTA's units (items, or pairs of them) are numbers blockIdx.x, blockIdx.x + gridDim.x, ... of the
+    // launch's units.  A launch that takes one size class of a mixed batch numbers only the units of the
+    // sequences of its class (ctab lists those sequences, for the whole batch, so that every CTA gets the
+    // same share of them whatever their places in the batch); a batch of more than CT_CAP sequences is
+    // walked whole.
     const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
-    int K = ((pair_mode ? n_items / 2 : n_items) - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const bool compact = CLASS && K <= C::CT_CAP;
+    const bool compact = CLASS && a.B <= C::CT_CAP;
+    const int ups = pair_mode ? a.H_v >> 1 : a.H_v;  // units per sequence
+    // g / ups = umulhi(g, magic) for ups >= 2 and g < 2^32 / ups (a division per item in every thread cost 4 %)
+    const uint32_t ups_magic = ups < 2 ? 0u : (uint32_t)((0x100000000ull + (uint32_t)ups - 1u) / (uint32_t)ups);
+    int n_units = pair_mode ? n_items / 2 : n_items;  // (compact: set once the class's sequences are counted)
     auto item_of = [&](int kk) {
+        const int g = (int)blockIdx.x + (pair_mode ? kk >> 1 : kk) * (int)gridDim.x;
         if constexpr (CLASS) {
-            int ku = pair_mode ? kk >> 1 : kk;
-            if (ku >= K) return n_items;
-            if (compact) ku = ctab[ku];
-            const int unit = (int)blockIdx.x + ku * (int)gridDim.x;
-            return pair_mode ? 2 * unit + (kk & 1) : unit;
-        } else {
-            return pair_mode ? 2 * ((int)blockIdx.x + (kk >> 1) * (int)gridDim.x) + (kk & 1)
-                             : (int)blockIdx.x + kk * (int)gridDim.x;
+            if (g >= n_units) return n_items;
+            if (compact) {
+                const int sq = ups < 2 ? g : (int)__umulhi((uint32_t)g, ups_magic), u = g - sq * ups;
+                return (int)ctab[sq] * a.H_v + (pair_mode ? 2 * u + (kk & 1) : u);
+            }
         }
+        return pair_mode ? 2 * g + (kk & 1) : g;
     };
 
     if (tid == 0) {
@@ -278,18 +283,15 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     const uint32_t tmem_base = *tmem_slot;
     if (CLASS && compact) {
         // Every role would otherwise hand every unit of the other classes through the whole pipeline
-        // just to drop it (a third of the time of a ragged batch).  All threads: one unit each per
-        // round, kept units numbered by warp ballots and a prefix over the warps' counts.
+        // just to drop it (a third of the time of a ragged batch).  All threads: one sequence each per
+        // round, kept sequences numbered by warp ballots and a prefix over the warps' counts.
         uint16_t *tab = reinterpret_cast<uint16_t *>(smem + C::OFF_CTAB);
         int *wcount = reinterpret_cast<int *>(smem + C::OFF_CTAB + C::CT_CAP * 2);
-        const int K_all = K;
         int kept = 0;
-        for (int base = 0; base < K_all; base += C::THREADS) {
-            const int ku = base + tid;
+        for (int base = 0; base < a.B; base += C::THREADS) {
+            const int b = base + tid;
             bool keep = false;
-            if (ku < K_all) {
-                const int unit = (int)blockIdx.x + ku * (int)gridDim.x;
-                const int b = (pair_mode ? 2 * unit : unit) / a.H_v;
+            if (b < a.B) {
                 const int lo = a.node_offsets[b], n = a.node_offsets[b + 1] - lo;
                 // another class's well-formed sequence goes; whatever has to be flagged stays
                 keep = !(n >= 1 && n <= a.max_nodes && (n <= a.cls_lo || n > a.cls_hi || n > NP)) || bad_offsets(lo, n, a.T) ||
@@ -303,11 +305,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 const int c = wcount[w2];
                 before += w2 < warp ? c : 0, total += c;
             }
-            if (keep) tab[kept + before + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)ku;
+            if (keep) tab[kept + before + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)b;
             kept += total;
             __syncthreads();
         }
-        K = kept;
+        n_units = kept * ups;
     }
 
     // the meta block of item kk of this CTA
@@ -1239,20 +1241,21 @@ cudaError_t launch_verify_sm100(const VerifyArgs &a, int T, treewy_dtype_t od, c
     if (a.B == 0 || a.H_v == 0 || T == 0) return cudaSuccess;
     if (a.max_nodes <= SMALL_MAX_NODES) return launch_verify_small(a, nullptr, T, od, stream);
     const PrevRound none = {};
-    VerifyArgs small = a;
-    small.cls_lo = 0, small.cls_hi = a.max_nodes < 32 ? a.max_nodes : 32;
-    cudaError_t e;
-    if (small.cls_hi <= 16)
-        e = od == TREEWY_F32 ? launch_vt<16, float, false>(small, none, T, stream)
-                             : launch_vt<16, __nv_bfloat16, false>(small, none, T, stream);
-    else
-        e = od == TREEWY_F32 ? launch_vt<32, float, false>(small, none, T, stream)
-                             : launch_vt<32, __nv_bfloat16, false>(small, none, T, stream);
-    if (e != cudaSuccess || a.max_nodes <= 32) return e;
-    VerifyArgs large = a;
-    large.cls_lo = 32, large.cls_hi = a.max_nodes;
-    return od == TREEWY_F32 ? launch_vt<64, float, false>(large, none, T, stream)
-                            : launch_vt<64, __nv_bfloat16, false>(large, none, T, stream);
+    auto run = [&](int np, int lo, int hi) {
+        VerifyArgs c = a;
+        c.cls_lo = lo, c.cls_hi = hi;
+        const bool f32 = od == TREEWY_F32;
+        if (np == 16) return f32 ? launch_vt<16, float, false>(c, none, T, stream) : launch_vt<16, __nv_bfloat16, false>(c, none, T, stream);
+        if (np == 32) return f32 ? launch_vt<32, float, false>(c, none, T, stream) : launch_vt<32, __nv_bfloat16, false>(c, none, T, stream);
+        return f32 ? launch_vt<64, float, false>(c, none, T, stream) : launch_vt<64, __nv_bfloat16, false>(c, none, T, stream);
+    };
+    if (a.max_nodes <= 16) return run(16, 0, a.max_nodes);
+    if (a.max_nodes <= 32) return run(32, 0, a.max_nodes);
+    // (a third class for trees of up to 8 nodes, through the small-tree kernel, which takes half the time
+    // per tree, or up to 16 nodes through the 16-node instance, was tried on the ragged workload: the extra
+    // launch costs more than it saves)
+    const cudaError_t e = run(32, 0, 32);
+    return e != cudaSuccess ? e : run(64, 32, a.max_nodes);
 }
 
 // commit of the previous round + verify of this one, one kernel; this round's trees have <= 32 nodes

@@ -212,3 +212,19 @@ def test_prepare_from_log_gates(oracle):
     tw.treewy_tree_prepare(lin, w.alpha.to(dev), status)
     torch.cuda.synchronize()
     np.testing.assert_allclose(tree.cum_log_gate.cpu().numpy(), lin.cum_log_gate.cpu().numpy(), rtol=0, atol=2e-6)
+
+
+@pytest.mark.parametrize("H_v,H_qk", [(1, 1), (2, 1), (3, 3), (6, 1), (4, 2), (5, 1)])
+def test_mixed_size_batches_across_head_layouts(oracle, H_v, H_qk):
+    """A batch that holds trees on both sides of 32 nodes gets one launch per size class, each numbering
+    the units of its class's sequences (one, several, an odd number of units per sequence; heads taken
+    singly or in pairs): every sequence must be verified exactly once, whatever its place in the batch."""
+    g = torch.Generator().manual_seed(100 + 7 * H_v + H_qk)
+    sizes = [40, 3, 64, 17, 1, 33, 32, 8, 50, 20, 64, 2, 36]
+    trees = [wl.random_parent_tree(g, n, 6) for n in sizes]
+    w = _custom(trees, H_v=H_v, H_qk=H_qk, seed=9, accepted=[n // 2 for n in sizes])
+    gpu = pu.run_gpu(w, torch.float32, max_nodes=64)
+    assert not gpu["status"].any()
+    assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any()
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    pu.assert_parity(w, gpu, tree_ref, ref)
