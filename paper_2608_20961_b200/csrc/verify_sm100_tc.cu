@@ -142,7 +142,7 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int OFF_GP = STAGES * STAGE_BYTES;
     static constexpr int OFF_DEEP = OFF_GP + SLOTS * GP_BYTES;  // 64 nodes: full-length lists of deep trees
     static constexpr int OFF_MRING = OFF_DEEP + DEEP_BYTES;      // 64 nodes: the ring of meta blocks
-    static constexpr int OFF_EINFO = OFF_MRING + (META_RING ? META_SLOTS * META_STRIDE : 0);  // (n, first node) of the item in a TMEM block
+    static constexpr int OFF_EINFO = OFF_MRING + (META_RING ? META_SLOTS * META_STRIDE : 0);  // (n, first output row) of the item in a TMEM block
     // fused mode: operands of the commit's rank-P product, K-major without swizzle, K = 8 path nodes:
     // core matrices of 8 rows x 16 bytes, the two K halves COPS_LBO apart
     static constexpr int COPS_LBO = D * 16, COPS_TILE = 2 * COPS_LBO;
@@ -178,6 +178,7 @@ struct PathMeta {
     float La, ga;             // its log-gate and e^{La}
     int plen;                 // path length; -1 = no commit for this item
     int lo;                   // first packed node of the sequence in the previous tree
+    int h;                    // the item's value head
 };
 static_assert(sizeof(PathMeta) <= 128, "path meta block");
 
@@ -450,7 +451,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (i < NP) meta_mask(mt)[i] = p.mk[r], meta_L(mt)[i] = p.Lv[r], meta_beta(mt)[i] = p.bv[r];
             }
             if (lane == 0)
-                meta_nlo(mt)[0] = p.bad ? 0 : p.n, meta_nlo(mt)[1] = p.lo, meta_nlo(mt)[2] = p.deep,
+                meta_nlo(mt)[0] = p.bad ? 0 : p.n, meta_nlo(mt)[1] = p.lo * a.H_v + p.h, meta_nlo(mt)[2] = p.deep,
                 meta_nlo(mt)[3] = p.srow;
             __syncwarp();  // the log-gates of all nodes are in the meta block
             const float *Lm = meta_L(mt);
@@ -491,7 +492,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if constexpr (FUSED) {
                 PathMeta *pm = reinterpret_cast<PathMeta *>(stage + C::OFF_PMETA);
                 if (lane < p.cnt) pm->w[lane] = p.wj;
-                if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = __expf(p.La), pm->plen = p.plen, pm->lo = p.plo;
+                if (lane == 0) pm->mask = p.pmask, pm->La = p.La, pm->ga = __expf(p.La), pm->plen = p.plen, pm->lo = p.plo, pm->h = p.h;
             }
             // The copies are issued first and announced (expect_tx, with the warp's one arrival) last:
             // the phase cannot complete before that arrival, and the path lists below are written
@@ -582,7 +583,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const PathMeta *pm = reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA);
             const int plen = pm->plen;
             if (plen >= 0) {
-                const int h = item % a.H_v;
+                const int h = pm->h;
                 const __nv_bfloat16 *kp = reinterpret_cast<const __nv_bfloat16 *>(stage + C::OFF_KP);
                 const float *up = reinterpret_cast<const float *>(stage + C::OFF_UP);
                 const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(pv.k);
@@ -1146,7 +1147,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         for (int kk = 0;; ++kk) {
             const int item = item_of(kk);
             if (item >= n_items) break;
-            const int buf = kk % C::TBUF, h = item % a.H_v;
+            const int buf = kk % C::TBUF;
             const uint32_t tm = tmem_base + lane_base + buf * C::TM_COLS;
             if (!ptx::mbar_wait(&mma2_done[buf], (kk / C::TBUF) & 1)) {
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
@@ -1154,9 +1155,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             }
             ptx::tc_fence_after_sync();
             const int2 info = einfo[buf];
-            const int n = info.x, lo = info.y;
+            const int n = info.x;
             if (n > 0) {
-                const size_t row0 = ((size_t)lo * a.H_v + h) * D + t;
+                const size_t row0 = (size_t)info.y * D + t;  // (the producer left the item's first row: a modulo here is 2 % of the kernel's instructions)
                 TU *Ub = static_cast<TU *>(a.U) + row0;
                 TOut *Ob = Og + row0;
 #pragma unroll 1
