@@ -53,7 +53,7 @@ static_assert(VS_N == 8, "the thread maps below are written for 8 nodes");
 struct VsMeta {
     int item;  // the item the stage holds or is being filled with (-1 before the first)
     int n;     // nodes to verify; 0 = nothing to verify (skipped or malformed sequence)
-    int lo;    // first packed node of the sequence
+    int row;   // the item's first output row: (first packed node of the sequence) * H_v + head
     int srow;  // state tile: (state slot) * H_v + head
     int plen;  // fused mode: nodes on the accepted path of the previous round; -1 = nothing to commit
     float ga;  //             e^{L_a}
@@ -224,7 +224,7 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
             VsMeta *meta = reinterpret_cast<VsMeta *>(smem + C::OFF_META + s * C::META_BYTES);
             if (lane < VS_N) meta->mask[lane] = p.mk, meta->L[lane] = p.Lv, meta->beta[lane] = p.bv, meta->w[lane] = p.wj;
             if (lane == 0) *reinterpret_cast<volatile int *>(&meta->item) = p.item;
-            if (lane == 0) meta->n = p.bad ? 0 : p.n, meta->lo = p.lo, meta->srow = p.srow, meta->plen = p.plen, meta->ga = expf(p.La);
+            if (lane == 0) meta->n = p.bad ? 0 : p.n, meta->row = p.lo * a.H_v + p.h, meta->srow = p.srow, meta->plen = p.plen, meta->ga = expf(p.La);
             const int cnt = p.plen > 0 ? p.plen : 0;
             const bool need_tile = (!p.bad || p.plen >= 0) && !(early && kk == s);  // the state tile serves verify, commit or both
             const uint32_t tx = (need_tile ? 2 * VS_HALF : 0) + (p.bad ? 0 : 2 * VS_QK_HALF + VS_N * D * 2) + cnt * (D * 2 + D * 4);
@@ -292,9 +292,8 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                 break;
             }
-            const int n = meta->n, lo = meta->lo, srow = meta->srow;
+            const int n = meta->n, row0 = meta->row, srow = meta->srow;
             const int plen = FUSED ? meta->plen : -1;
-            const int h = item % a.H_v;
             if constexpr (FUSED) {
                 if (plen >= 0) {
                     // Eq. 3 on the tile: thread (r0, cc) takes the 16-byte chunk cc of rows r0, r0 + 8, ...
@@ -466,8 +465,8 @@ verify_small_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_consta
                 }
                 ptx::tc_fence_before_sync();
                 float u[VS_N];
-                const size_t urow = ((size_t)lo * a.H_v + h) * D + t;
-                TOut *Og = static_cast<TOut *>(a.O) + ((size_t)lo * a.H_v + h) * D + t;
+                const size_t urow = (size_t)row0 * D + t;
+                TOut *Og = static_cast<TOut *>(a.O) + urow;
                 const size_t rs = (size_t)a.H_v * D;
 #pragma unroll
                 for (int j = 0; j < VS_N; ++j) {
