@@ -228,3 +228,19 @@ def test_mixed_size_batches_across_head_layouts(oracle, H_v, H_qk):
     assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any()
     tree_ref, ref = pu.run_oracle(oracle, w)
     pu.assert_parity(w, gpu, tree_ref, ref)
+
+
+def test_mixed_size_batch_larger_than_the_class_table(oracle):
+    """More sequences than a class launch lists in shared memory (1024): both class launches walk the
+    whole batch and drop the other class's sequences one by one."""
+    g = torch.Generator().manual_seed(77)
+    sizes = [1 + int(torch.randint(0, 3, (1,), generator=g)) for _ in range(1040)]
+    for at, n in ((5, 64), (333, 40), (700, 33), (1030, 57)):
+        sizes[at] = n
+    trees = [wl.random_parent_tree(g, n, 5) for n in sizes]
+    w = _custom(trees, H_v=1, H_qk=1, seed=12, accepted=[n - 1 for n in sizes])
+    gpu = pu.run_gpu(w, torch.float32, max_nodes=64)
+    assert not gpu["status"].any()
+    assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any()
+    tree_ref, ref = pu.run_oracle(oracle, w)
+    pu.assert_parity(w, gpu, tree_ref, ref)
