@@ -182,6 +182,24 @@ struct PathMeta {
 };
 static_assert(sizeof(PathMeta) <= 128, "path meta block");
 
+// How a class launch numbers its units (see the kernel's prologue): unit g of the launch is unit
+// g % ups of sequence tab[g / ups] (compact) or of sequence g / ups (a batch too large for the table).
+struct ClassMap {
+    const uint16_t *tab;
+    int n_units, n_items, ups, H_v;
+    uint32_t magic;  // g / ups = umulhi(g, magic) for ups >= 2 and g < 2^32 / ups (a division per item in every thread cost 4 %)
+    bool pair, compact;
+};
+static __shared__ ClassMap s_class_map;  // written by thread 0 before the roles start
+static __device__ __noinline__ int class_item_of(int g, int odd)
+{
+    const ClassMap &m = s_class_map;
+    if (g >= m.n_units) return m.n_items;
+    if (!m.compact) return m.pair ? 2 * g + odd : g;
+    const int sq = m.ups < 2 ? g : (int)__umulhi((uint32_t)g, m.magic), u = g - sq * m.ups;
+    return (int)m.tab[sq] * m.H_v + (m.pair ? 2 * u + odd : u);
+}
+
 // (CLASS: the launch takes one size class of a mixed batch and walks a compacted work list; TU: the
 // type U is stored in, float or __half.  Both are template parameters because the code they add
 // costs the other launches instruction-cache hits: 2 % of the headline kernel's time for either.)
@@ -226,18 +244,21 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     // sequences of its class (ctab lists those sequences, for the whole batch, so that every CTA gets the
     // same share of them whatever their places in the batch); a batch of more than CT_CAP sequences is
     // walked whole.
-    const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
+    // (a class launch: see ClassMap; n_units is set once the class's sequences are counted)
     const bool compact = CLASS && a.B <= C::CT_CAP;
     const int ups = pair_mode ? a.H_v >> 1 : a.H_v;  // units per sequence
-    // g / ups = umulhi(g, magic) for ups >= 2 and g < 2^32 / ups (a division per item in every thread cost 4 %)
-    const uint32_t ups_magic = ups < 2 ? 0u : (uint32_t)((0x100000000ull + (uint32_t)ups - 1u) / (uint32_t)ups);
     int n_units = pair_mode ? n_items / 2 : n_items;  // (compact: set once the class's sequences are counted)
+    const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
     auto item_of = [&](int kk) {
         const int g = (int)blockIdx.x + (pair_mode ? kk >> 1 : kk) * (int)gridDim.x;
-        if constexpr (CLASS) {
+        if constexpr (CLASS && C::BIG) {
+            // out of line in the 64-node instance (eleven call sites: 1 % through the instruction cache);
+            // the smaller instances, with a third of the time per item, lose 5 % to the calls
+            return class_item_of(g, kk & 1);
+        } else if constexpr (CLASS) {
             if (g >= n_units) return n_items;
             if (compact) {
-                const int sq = ups < 2 ? g : (int)__umulhi((uint32_t)g, ups_magic), u = g - sq * ups;
+                const int sq = ups < 2 ? g : (int)__umulhi((uint32_t)g, a.ups_magic), u = g - sq * ups;
                 return (int)ctab[sq] * a.H_v + (pair_mode ? 2 * u + (kk & 1) : u);
             }
         }
@@ -311,6 +332,15 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             __syncthreads();
         }
         n_units = kept * ups;
+    }
+    if constexpr (CLASS && C::BIG) {
+        if (tid == 0) {
+            s_class_map.tab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
+            s_class_map.n_units = n_units;
+            s_class_map.n_items = n_items, s_class_map.ups = ups, s_class_map.H_v = a.H_v;
+            s_class_map.magic = a.ups_magic, s_class_map.pair = pair_mode, s_class_map.compact = compact;
+        }
+        __syncthreads();
     }
 
     // the meta block of item kk of this CTA
@@ -1202,12 +1232,16 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     int dev = 0, sms = 0;
     cudaError_t e = current_device_sms(&dev, &sms);
     if (e != cudaSuccess) return e;
-    const long long units = (a.H_v / a.H_qk) % 2 == 0 ? n_items / 2 : n_items;  // the kernel takes heads in pairs
+    const bool pairs = (a.H_v / a.H_qk) % 2 == 0;  // the kernel takes heads in pairs
+    const long long units = pairs ? n_items / 2 : n_items;
     const int grid = (int)(units < sms ? units : sms);
+    VerifyArgs a2 = a;
+    const uint32_t ups = (uint32_t)(pairs ? a.H_v / 2 : a.H_v);
+    a2.ups_magic = ups < 2 ? 0u : (uint32_t)((0x100000000ull + ups - 1u) / ups);
     auto go = [&](auto kernel) {
         cudaError_t e2 = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), C::SMEM_BYTES, dev);
         if (e2 != cudaSuccess) return e2;
-        return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a, pv, (int)n_items, m.S0, m.Q,
+        return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a2, pv, (int)n_items, m.S0, m.Q,
                                 m.K, m.V);
     };
     if constexpr (FUSED) {
