@@ -500,16 +500,15 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 }
             }
         };
-        Pre cur = fetch(s);
+        // (One call site for the fetch: it is the largest piece of code a producer runs.  The loop's first
+        // round, kk = s - STAGES, only fetches; a round processes the item fetched by the round before.)
+        Pre cur = {};
         bool s0_issued = early;  // the state tile of `cur` is in flight already
 #pragma unroll 1
-        for (int kk = s;; kk += C::STAGES) {
-            if (cur.item >= n_items) break;
-            if (cur.item == a.skip_item) {  // test hook: this item's loads and their arrival never happen
-                cur = fetch(kk + C::STAGES);
-                s0_issued = false;
-                continue;
-            }
+        for (int kk = s - C::STAGES;; kk += C::STAGES) {
+            // (test hook: the skipped item's loads and their arrival never happen)
+            if (kk >= s && cur.item >= n_items) break;
+            if (kk >= s && cur.item != a.skip_item) {
             const Pre p = cur;
             unsigned char *mt = meta_of(kk);
             if constexpr (C::META_RING) write_meta(p, mt);  // the block of item kk - 2 * STAGES: long read
@@ -561,11 +560,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (tx == 0) ptx::mbar_arrive(&full[s]);
                 else ptx::mbar_arrive_expect_tx(&full[s], tx);
             }
+            }
+            const bool processed = kk >= s && cur.item != a.skip_item;
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
-            s0_issued = false;
+            if (kk >= s) s0_issued = false;
             if constexpr (C::S0_EARLY) {
                 // the next item's state tile: the stage's S0 tile is free as soon as stage 1 has read it
-                if (cur.item < n_items && cur.item != a.skip_item && !cur.bad) {
+                if (processed && cur.item < n_items && cur.item != a.skip_item && !cur.bad) {
                     if (!ptx::mbar_wait(&s0_empty[s], (kk / C::STAGES) & 1)) {
                         if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[cur.b], TREEWY_SEQ_TIMEOUT);
                         break;
