@@ -61,10 +61,15 @@ constexpr uint32_t VT_TMEM_COLS = 512;
 
 template <int NP, bool FUSED> struct VtCfg {
     static_assert(NP == 16 || NP == 32 || (NP == 64 && !FUSED), "up to 64 nodes; the fused mode up to 32");
-    static constexpr bool BIG = NP == 64;  // 33..64 nodes: shared memory and tensor memory hold two items
+    static constexpr bool BIG = NP == 64;  // 33..64 nodes: shared memory and tensor memory hold three items
+    // 64 nodes: the S0 tiles are not part of the stages but a ring of their own, S0_SLOTS deep, filled by
+    // a warp of its own in item order.  A state tile lives from its copy to the end of stage 1, half as
+    // long as the [Q;K] tile and what overlays it, so two tiles serve three stages.
+    static constexpr bool S0_RING = BIG;
+    static constexpr int S0_SLOTS = 2;
     static constexpr int NPL = (NP + 31) / 32;  // nodes per producer lane
     static constexpr int SLOTS = 2;  // list / scalar / v-row buffers alternate between consecutive items
-    static constexpr int STAGES = BIG ? 2 : (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
+    static constexpr int STAGES = BIG ? 3 : (FUSED ? 3 : 4) + (NP == 16 ? 1 : 0);  // as many as shared memory holds
     static constexpr int CGROUP = FUSED ? 128 : 0;  // threads of the commit group (fused mode)
     // (fused mode gives 128 columns of tensor memory to the commit's accumulator)
         static constexpr int TBUF = BIG ? 3 : FUSED ? 4 : 5;  // [SQ | SK] -> [O | U] blocks: held from stage 1 to the epilogue
@@ -81,17 +86,18 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int MMA1B_WARP = MMA1_WARP + 1;  // the Gram chain of stage 1 has its own issuing warp
     static constexpr int MMA2_WARP = MMA1B_WARP + 1;
     static constexpr int PROD_WARP0 = MMA2_WARP + 1;
-    static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 96 + 32 * STAGES;
+    static constexpr int S0P_WARP = PROD_WARP0 + STAGES;  // (S0_RING) the warp that fills the ring of S0 tiles
+    static constexpr int THREADS = COMMIT_WARP0 * 32 + CGROUP + 96 + 32 * STAGES + (S0_RING ? 32 : 0);
     // stage: [Q;K] tile | S0 tile | (fused: previous round's path rows of k and U) | meta | (fused: path meta)
     // (the v rows go to the slots below, two items ahead)
     static constexpr int QK_HALF = 2 * NP * 128;
     static constexpr int QK_BYTES = 2 * QK_HALF;
     static constexpr int S0_HALF = D * 128;
     static constexpr int S0_BYTES = 2 * S0_HALF;
-    static constexpr int OFF_S0 = QK_BYTES;
+    static constexpr int OFF_S0 = QK_BYTES;  // (not S0_RING)
     static constexpr int PCH = 8;  // previous-round path nodes staged per item (fused mode)
     static constexpr int OFF_KP = OFF_S0 + S0_BYTES, OFF_UP = OFF_KP + PCH * D * 2;
-    static constexpr int OFF_META = FUSED ? OFF_UP + PCH * D * 4 : OFF_S0 + S0_BYTES;
+    static constexpr int OFF_META = FUSED ? OFF_UP + PCH * D * 4 : S0_RING ? QK_BYTES : OFF_S0 + S0_BYTES;
     // mask u64, L f32, beta f32 per node; n, lo, deep; then the producer-built path lists of the
     // first 8 ancestors of every node: gate ratios e^{L_i - L_j} as [d / 4][node][d % 4] floats and
     // the ancestors' indices as [d / 4][node] words of four bytes
@@ -115,33 +121,31 @@ template <int NP, bool FUSED> struct VtCfg {
     static constexpr int TILE_BYTES = 2 * PART;
     static_assert(TILE_BYTES <= QK_BYTES, "operand overlays fit");
     // scratch over the dead tiles: the raw Gram rows (up to 32 nodes: in the S0 tile, beside the B
-    // tiles; 64 nodes: from the stage's start, under the B tiles, which are zeroed once the lists are
-    // built) and the back-substitution rows of deep paths (in the S0 tile; 64 nodes: the stash is dead
-    // by then, and a row is exactly NP floats, rotated by the node's number against bank conflicts)
-    // (64 nodes: the stash is exactly the [Q;K] tile, rows of NP floats with their 16-byte columns swizzled
-    // by the row number, so that the S0 tile is dead once stage 1 has read it and goes back to the
-    // producer right then, a stage-2 time before the rest of the stage; deep trees keep it for their rows)
-    static constexpr bool S0_EARLY = BIG;
+    // tiles; 64 nodes: the stash IS the [Q;K] tile, rows of NP floats with their 16-byte columns swizzled
+    // by the row number, and the B tiles, zeroed once the lists are built, take its place), so that with
+    // 64 nodes a state tile is dead once stage 1 has read it.  Trees with a path of more than 8
+    // ancestors ("deep") need more: their back-substitution rows and full-length lists.  Up to 32 nodes
+    // both are in the S0 tile; with 64 nodes a deep tree keeps its S0 tile until stage 2 ends, the lists
+    // A and P (NP x NP floats each) fill it exactly, the ancestors' indices take the place of the slot's
+    // short lists, and the rows live in the solver threads' local memory.
     static constexpr int RLD = BIG ? NP : NP + 4;  // row stride of the raw Gram stash (floats)
-    static constexpr int XLD = BIG ? NP : NP + 1;
-    static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = BIG ? OFF_S0 : OFF_S0 + 2 * NP * RLD * 4;
+    static constexpr int XLD = NP + 1;
+    static constexpr int OFF_RAW = BIG ? 0 : OFF_S0, OFF_XR = OFF_S0 + 2 * NP * RLD * 4;  // (OFF_XR: up to 32 nodes)
     static_assert(OFF_RAW + 2 * NP * RLD * 4 <= (BIG ? QK_BYTES : OFF_S0 + S0_BYTES), "Gram stash fits");
-    static_assert(OFF_XR + 2 * NP * XLD * 4 <= OFF_S0 + S0_BYTES, "back-substitution rows fit");
-    // ... and, for trees with a path of more than 8 ancestors, the full-length lists (64 nodes: in an
-    // area of their own)
-    static constexpr int OFF_DAP = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 15) / 16 * 16;
+    static constexpr int OFF_DAP = OFF_S0 + (2 * NP * RLD * 4 + 2 * NP * XLD * 4 + 15) / 16 * 16;  // (up to 32 nodes)
     static constexpr int OFF_DPP = OFF_DAP + NP * NP * 4, OFF_DIDX = OFF_DPP + NP * NP * 4;
     static_assert(BIG || OFF_DIDX + NP * NP <= OFF_S0 + S0_BYTES, "scratch fits in the S0 tile");
-    static constexpr int DEEP_BYTES = BIG ? 2 * NP * NP * 4 + NP * NP : 0;
+    static_assert(!BIG || 2 * NP * NP * 4 == S0_BYTES, "64 nodes: the full-length lists fill a state tile");
     static constexpr int V_BYTES = NP * D * 2;
     // a slot (consecutive items alternate between the two): path lists of the first 8 ancestors,
     // per-node scalars, and the item's v rows [NP][128] bf16
     static constexpr int GP_AP = 0, GP_PP = 2 * NP * 16, GP_SCAL = 4 * NP * 16;
     static constexpr int GP_VS = (GP_SCAL + NP * 16 + 127) / 128 * 128;
     static constexpr int GP_BYTES = GP_VS + V_BYTES;
-    static constexpr int OFF_GP = STAGES * STAGE_BYTES;
-    static constexpr int OFF_DEEP = OFF_GP + SLOTS * GP_BYTES;  // 64 nodes: full-length lists of deep trees
-    static constexpr int OFF_MRING = OFF_DEEP + DEEP_BYTES;      // 64 nodes: the ring of meta blocks
+    static_assert(!BIG || GP_SCAL >= NP * NP, "64 nodes: a deep tree's ancestor indices fit over the slot's short lists");
+    static constexpr int OFF_S0R = STAGES * STAGE_BYTES;  // (S0_RING) the ring of state tiles
+    static constexpr int OFF_GP = OFF_S0R + (S0_RING ? S0_SLOTS * S0_BYTES : 0);
+    static constexpr int OFF_MRING = OFF_GP + SLOTS * GP_BYTES;  // 64 nodes: the ring of meta blocks
     static constexpr int OFF_EINFO = OFF_MRING + (META_RING ? META_SLOTS * META_STRIDE : 0);  // (n, first output row) of the item in a TMEM block
     // fused mode: operands of the commit's rank-P product, K-major without swizzle, K = 8 path nodes:
     // core matrices of 8 rows x 16 bytes, the two K halves COPS_LBO apart
@@ -152,7 +156,7 @@ template <int NP, bool FUSED> struct VtCfg {
     // work list of a launch that takes one size class of a mixed batch: the CTA's units of that class
     // (up to CT_CAP of them; a longer list is walked whole), then 32 warp counts
     static constexpr int CT_CAP = 1024;
-    static constexpr int OFF_CTAB = OFF_BAR + (4 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16;
+    static constexpr int OFF_CTAB = OFF_BAR + (5 * STAGES + 4 * TBUF + RBUF + 5 * SLOTS + 1) * 8 + 16;
     static constexpr int SMEM_BYTES = OFF_CTAB + CT_CAP * 2 + 32 * 4 + 1024;
     static constexpr uint32_t TX_BYTES = S0_BYTES + QK_BYTES;
     // Tensor memory holds two rings.  A block of the first takes SQ | SK from stage 1; the R^T warps
@@ -230,8 +234,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     uint64_t *scal_ready = lists_free + C::SLOTS;      // Gram warps -> R^T warps: per-node scalars written
     uint64_t *upd_done = scal_ready + C::SLOTS;        // fused mode: the state tile of a stage carries the commit
     uint64_t *cmma_done = upd_done + C::STAGES;        // fused mode: the commit's rank-P product has finished
-    uint64_t *s0_empty = cmma_done + 1;                // 64 nodes: the S0 tile of a stage may be refilled
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s0_empty + C::STAGES);
+    uint64_t *s0_empty = cmma_done + 1;                // 64 nodes: a tile of the S0 ring may be refilled
+    uint64_t *s0_full = s0_empty + C::STAGES;          //           ... has landed
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s0_full + C::STAGES);
     int2 *einfo = reinterpret_cast<int2 *>(smem + C::OFF_EINFO);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -284,7 +289,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             ptx::mbar_init(&lists_free[g], (C::R_THREADS + C::T_THREADS) / 32);
             ptx::mbar_init(&scal_ready[g], C::G_THREADS / 32);
         }
-        for (int s = 0; s < C::STAGES; ++s) ptx::mbar_init(&upd_done[s], 128 / 32), ptx::mbar_init(&s0_empty[s], 1);
+        for (int s = 0; s < C::STAGES; ++s)
+            ptx::mbar_init(&upd_done[s], 128 / 32), ptx::mbar_init(&s0_empty[s], 1), ptx::mbar_init(&s0_full[s], 1);
         ptx::mbar_init(cmma_done, 1);
         ptx::fence_barrier_init();
     }
@@ -343,6 +349,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         __syncthreads();
     }
 
+    // the state tile of item kk of this CTA
+    auto s0_of = [&](int kk) {
+        return C::S0_RING ? smem + C::OFF_S0R + (kk % C::S0_SLOTS) * C::S0_BYTES
+                          : smem + (kk % C::STAGES) * C::STAGE_BYTES + C::OFF_S0;
+    };
     // the meta block of item kk of this CTA
     auto meta_of = [&](int kk) {
         return C::META_RING ? smem + C::OFF_MRING + (kk % C::META_SLOTS) * C::META_STRIDE
@@ -361,7 +372,33 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     // byte offset of element (row, col) of a stage-2 B tile (bf16, one 128-byte line per row, 128-byte swizzle)
     auto tile_off = [](int row, int col) { return row * 128 + (((col >> 3) ^ (row & 7)) << 4) + ((col & 7) << 1); };
 
-    if (warp >= C::PROD_WARP0) {
+    if (C::S0_RING && warp == C::S0P_WARP) {
+        // ------------------------------------------------------------------ state-tile warp (64 nodes)
+        // Fills the ring of S0 tiles in item order: a tile's address depends on nothing but the item's
+        // number (and the sequence's state slot), so this warp validates nothing; an item the pipeline
+        // skips gets its tile all the same (stage 1 waits for it before it hands the slot back).
+#pragma unroll 1
+        for (int kk = 0;; ++kk) {
+            const int item = item_of(kk);
+            if (item >= n_items) break;
+            if (item == a.skip_item) continue;  // test hook: this item's loads and their arrival never happen
+            const int b = item / a.H_v, h = item - b * a.H_v;
+            const int slot = state_slot(a.state_index, a.n_states, b);
+            const int srow = (slot < 0 ? 0 : slot) * a.H_v + h;
+            const int z = kk % C::S0_SLOTS;
+            if (!ptx::mbar_wait(&s0_empty[z], ((kk / C::S0_SLOTS) & 1) ^ 1)) {
+                if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[b], TREEWY_SEQ_TIMEOUT);
+                break;
+            }
+            if (lane == 0) {
+                unsigned char *tile = s0_of(kk);
+                ptx::mbar_arrive_expect_tx(&s0_full[z], C::S0_BYTES);
+                ptx::tma_load_2d(tile, &tmS0, 0, srow * D, &s0_full[z]);
+                ptx::tma_load_2d(tile + C::S0_HALF, &tmS0, 64, srow * D, &s0_full[z]);
+            }
+            __syncwarp();
+        }
+    } else if (warp >= C::PROD_WARP0) {
         // ------------------------------------------------------------------ producer warp
         const int s = warp - C::PROD_WARP0;
         unsigned char *stage = smem + s * C::STAGE_BYTES;
@@ -463,7 +500,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         // in flight before the item's scalars are fetched (two dependent loads, 2 us in a role trace, that
         // would otherwise stand in front of the launch's first bytes).
         const int item0 = item_of(s);
-        const bool early = !a.state_index && item0 < n_items && item0 != a.skip_item;
+        const bool early = !C::S0_RING && !a.state_index && item0 < n_items && item0 != a.skip_item;
         if (early && lane == 0) {
             ptx::mbar_expect_tx(&full[s], C::S0_BYTES);
             ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, item0 * D, &full[s]);
@@ -527,7 +564,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             // the phase cannot complete before that arrival, and the path lists below are written
             // while the data is on its way.
             const bool tile_issued = s0_issued;
-            const bool need_tile = (!p.bad || p.plen >= 0) && !tile_issued;  // the state tile serves verify, commit or both
+            // the state tile serves verify, commit or both (64 nodes: it comes through the ring of its own)
+            const bool need_tile = !C::S0_RING && (!p.bad || p.plen >= 0) && !tile_issued;
             const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
             if (lane == 0) {
                 if (tx != 0) {
@@ -561,24 +599,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 else ptx::mbar_arrive_expect_tx(&full[s], tx);
             }
             }
-            const bool processed = kk >= s && cur.item != a.skip_item;
             cur = fetch(kk + C::STAGES);  // in flight while this stage is being consumed
             if (kk >= s) s0_issued = false;
-            if constexpr (C::S0_EARLY) {
-                // the next item's state tile: the stage's S0 tile is free as soon as stage 1 has read it
-                if (processed && cur.item < n_items && cur.item != a.skip_item && !cur.bad) {
-                    if (!ptx::mbar_wait(&s0_empty[s], (kk / C::STAGES) & 1)) {
-                        if (lane == 0 && a.seq_status) atomicOr(&a.seq_status[cur.b], TREEWY_SEQ_TIMEOUT);
-                        break;
-                    }
-                    if (lane == 0) {
-                        ptx::mbar_expect_tx(&full[s], C::S0_BYTES);
-                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, cur.srow * D, &full[s]);
-                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, cur.srow * D, &full[s]);
-                    }
-                    s0_issued = true;
-                }
-            }
         }
     } else if (FUSED && warp >= C::COMMIT_WARP0 && warp < C::MMA1_WARP) {
         // ------------------------------------------------------------------ commit group (fused mode)
@@ -755,11 +777,14 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                 if (!ptx::mbar_wait(&r_free[kk % C::RBUF], ((kk / C::RBUF) & 1) ^ 1)) break;
             } else {
                 if (!ptx::mbar_wait(&tmem_free[buf], ((kk / C::TBUF) & 1) ^ 1)) break;
+                // (64 nodes: the item's state tile has landed -- also when the item is skipped: the slot
+                // goes back below, and its copy must be over by then)
+                if (C::S0_RING && !ptx::mbar_wait(&s0_full[kk % C::S0_SLOTS], (kk / C::S0_SLOTS) & 1)) break;
             }
             ptx::tc_fence_after_sync();
             if (lane == 0) {
                 if (n > 0) {
-                    const uint32_t qk = ptx::smem_u32(stage), s0 = qk + C::OFF_S0;
+                    const uint32_t qk = ptx::smem_u32(stage), s0 = ptx::smem_u32(s0_of(kk));
                     const uint32_t d1 = tmem_base + buf * C::TM_COLS;
                     const uint32_t d2 = tmem_base + C::TM_R0 + (kk % C::RBUF) * C::TM_RCOLS;
 #pragma unroll 1
@@ -777,11 +802,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     // store must have read it by then)
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::umma_commit(&mma1_done[buf]);
-                    if (C::S0_EARLY && !gram_chain && meta_nlo(mt)[2] == 0) ptx::umma_commit(&s0_empty[s]);
+                    if (C::S0_RING && !gram_chain && meta_nlo(mt)[2] == 0) ptx::umma_commit(&s0_empty[kk % C::S0_SLOTS]);
                 } else {
                     if (stored) ptx::bulk_wait_group_read<0>();
                     ptx::mbar_arrive(&mma1_done[buf]);
-                    if (C::S0_EARLY && !gram_chain && meta_nlo(mt)[2] == 0) ptx::mbar_arrive(&s0_empty[s]);
+                    if (C::S0_RING && !gram_chain && meta_nlo(mt)[2] == 0) ptx::mbar_arrive(&s0_empty[kk % C::S0_SLOTS]);
                 }
             }
             __syncwarp();
@@ -800,7 +825,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (!ptx::mbar_wait(&ops_ready[buf], (kk / C::TBUF) & 1)) break;
             ptx::tc_fence_after_sync();
             const int n = meta_nlo(mt)[0];
-            const bool keeps_s0 = C::S0_EARLY && meta_nlo(mt)[2] != 0;  // a deep tree: its S0 tile goes back only now
+            const bool keeps_s0 = C::S0_RING && meta_nlo(mt)[2] != 0;  // a deep tree: its S0 tile goes back only now
             if (lane == 0) {
                 if (n > 0) {
                     const uint32_t base = ptx::smem_u32(stage);
@@ -818,12 +843,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                     }
                     ptx::umma_commit(&mma2_done[buf]);
                     ptx::umma_commit(&empty[s]);  // the stage's operand overlays have been consumed
-                    if (keeps_s0) ptx::umma_commit(&s0_empty[s]);
+                    if (keeps_s0) ptx::umma_commit(&s0_empty[kk % C::S0_SLOTS]);
                     ptx::umma_commit(&r_free[kk % C::RBUF]);
                 } else {
                     ptx::mbar_arrive(&mma2_done[buf]);
                     ptx::mbar_arrive(&empty[s]);
-                    if (keeps_s0) ptx::mbar_arrive(&s0_empty[s]);
+                    if (keeps_s0) ptx::mbar_arrive(&s0_empty[kk % C::S0_SLOTS]);
                     ptx::mbar_arrive(&r_free[kk % C::RBUF]);
                 }
             }
@@ -928,14 +953,13 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         val.z = scale * rt.z * gram4[q].z, val.w = scale * rt.w * gram4[q].w;
                         (kind ? Ap4 : Pp4)[hf * NP + i] = val;
                     }
-                } else if (tg < 2 * NP) {  // full-length lists, in scratch memory
-                    if constexpr (C::BIG) {  // one area for both slots: the previous item's solve must be over
-                        if (kk >= 1 && !ptx::mbar_wait(&lists_free[(kk - 1) & 1], ((kk - 1) >> 1) & 1)) break;
-                    }
-                    unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;
+                } else if (tg < 2 * NP) {
+                    // full-length lists, in scratch memory (64 nodes: A and P fill the item's state tile, which
+                    // a deep tree keeps until stage 2 ends; the indices take the place of the slot's short lists)
+                    unsigned char *dl = C::BIG ? s0_of(kk) : stage + C::OFF_DAP;
                     float *Ap = reinterpret_cast<float *>(dl);
                     float *Pp = reinterpret_cast<float *>(dl + NP * NP * 4);
-                    unsigned char *idx = dl + 2 * NP * NP * 4;
+                    unsigned char *idx = C::BIG ? gp + C::GP_AP : dl + 2 * NP * NP * 4;
                     mask_t m = valid ? (mask_t)meta_mask(mt)[i] & ~((mask_t)1 << i) : (mask_t)0;
 #pragma unroll 1
                     for (int d = 0; m; ++d) {
@@ -1010,11 +1034,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int n = meta_nlo(mt)[0];  // (the Gram warps read the meta block before they signalled)
             if (n > 0 && tt < 2 * NP && i < n) {
                 const bool deep = meta_nlo(mt)[2] != 0;
-                const unsigned char *dl = C::BIG ? smem + C::OFF_DEEP : stage + C::OFF_DAP;  // full-length lists
+                const unsigned char *dl = C::BIG ? s0_of(kk) : stage + C::OFF_DAP;  // full-length lists (deep trees)
                 const float *Ap = reinterpret_cast<const float *>(dl);
                 const float *Pp = reinterpret_cast<const float *>(dl + NP * NP * 4);
-                const unsigned char *idx = dl + 2 * NP * NP * 4;
-                float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);
+                const unsigned char *idx = C::BIG ? gp + C::GP_AP : dl + 2 * NP * NP * 4;
+                float *xr = reinterpret_cast<float *>(stage + C::OFF_XR);  // (up to 32 nodes)
                 const int dp = m_popc((mask_t)meta_mask(mt)[i]) - 1;  // ancestors of node i
                     const float top = wrow ? scal[i].w : 1.f;
                     unsigned char *Mhi = stage + (wrow ? C::OFF_W_HI : C::OFF_T_HI);
@@ -1064,9 +1088,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
                         for (int e = 8; e >= 0; --e) {
                             put(tile_off(i, jf[e]), x[e]);
                         }
-                    } else {  // deep paths: the same recurrence through shared memory
-                        float *x = xr + (wrow ? i : NP + i) * C::XLD;
-                        auto xi = [&](int e) { return C::BIG ? (e + i) & (NP - 1) : e; };
+                    } else {  // deep paths: the same recurrence through shared memory (64 nodes: local memory)
+                        float xloc[C::BIG ? NP : 1];
+                        float *x = C::BIG ? xloc : xr + (wrow ? i : NP + i) * C::XLD;
+                        auto xi = [](int e) { return e; };
                         x[xi(dp)] = top;
 #pragma unroll 1
                         for (int e = dp - 1; e >= 0; --e) {
