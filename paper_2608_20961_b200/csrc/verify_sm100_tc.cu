@@ -24,6 +24,8 @@
 // for lists / scalars / v rows) let consecutive items overlap:
 //   producer warps   TMA tensor-map loads of S0 and [Q;K] into a stage ring; node scalars and the
 //                    path lists (index and gate ratio of every node's first 8 ancestors)
+//   state-tile warp  (64-node instance) the S0 tiles have a ring of their own, shorter-lived than
+//                    the stages, filled in item order by this warp
 //   MMA-1 warp       stage-1 MMAs: SQ | SK into a block of the first TMEM ring, the Gram block
 //                    into a block of the second                            -> mma1_done
 //   Gram warps       Gram rows -> stash -> scaled ancestor lists (A, P), per-node scalars; zero the
