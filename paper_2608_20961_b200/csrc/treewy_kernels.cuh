@@ -30,7 +30,6 @@ struct VerifyArgs {
     // size class of this launch: sequences with cls_lo < N_b <= cls_hi are processed, the others are
     // left to the launch of their class (N_b outside 1..max_nodes is flagged where cls_lo == 0)
     int cls_lo, cls_hi;
-    uint32_t ups_magic;  // class launches of the role pipeline: ceil(2^32 / units per sequence), 0 when that is 1
 };
 
 // the previous decoding round, whose accepted node the fused kernel commits before verifying

@@ -188,24 +188,6 @@ struct PathMeta {
 };
 static_assert(sizeof(PathMeta) <= 128, "path meta block");
 
-// How a class launch numbers its units (see the kernel's prologue): unit g of the launch is unit
-// g % ups of sequence tab[g / ups] (compact) or of sequence g / ups (a batch too large for the table).
-struct ClassMap {
-    const uint16_t *tab;
-    int n_units, n_items, ups, H_v;
-    uint32_t magic;  // g / ups = umulhi(g, magic) for ups >= 2 and g < 2^32 / ups (a division per item in every thread cost 4 %)
-    bool pair, compact;
-};
-static __shared__ ClassMap s_class_map;  // written by thread 0 before the roles start
-static __device__ __noinline__ int class_item_of(int g, int odd)
-{
-    const ClassMap &m = s_class_map;
-    if (g >= m.n_units) return m.n_items;
-    if (!m.compact) return m.pair ? 2 * g + odd : g;
-    const int sq = m.ups < 2 ? g : (int)__umulhi((uint32_t)g, m.magic), u = g - sq * m.ups;
-    return (int)m.tab[sq] * m.H_v + (m.pair ? 2 * u + odd : u);
-}
-
 // (CLASS: the launch takes one size class of a mixed batch and walks a compacted work list; TU: the
 // type U is stored in, float or __half.  Both are template parameters because the code they add
 // costs the other launches instruction-cache hits: 2 % of the headline kernel's time for either.)
@@ -248,27 +230,23 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     const bool pair_mode = ((a.H_v / a.H_qk) & 1) == 0;
     // The CTA's units (items, or pairs of them) are numbers blockIdx.x, blockIdx.x + gridDim.x, ... of the
     // launch's units.  A launch that takes one size class of a mixed batch numbers only the units of the
-    // sequences of its class (ctab lists those sequences, for the whole batch, so that every CTA gets the
-    // same share of them whatever their places in the batch); a batch of more than CT_CAP sequences is
-    // walked whole.
-    // (a class launch: see ClassMap; n_units is set once the class's sequences are counted)
-    const bool compact = CLASS && a.B <= C::CT_CAP;
+    // sequences of its class, over the whole batch, so that every CTA gets the same share of them whatever
+    // their places in the batch; its own units are then listed in ctab (see the prologue below).  A batch of
+    // more than CT_CAP sequences is walked whole.
     const int ups = pair_mode ? a.H_v >> 1 : a.H_v;  // units per sequence
-    int n_units = pair_mode ? n_items / 2 : n_items;  // (compact: set once the class's sequences are counted)
+    const bool compact = CLASS && a.B <= C::CT_CAP && (a.B * ups + (int)gridDim.x - 1) / (int)gridDim.x <= C::CT_CAP;
+    int K = 0;  // compact: the CTA's units (set by the prologue)
     const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
     auto item_of = [&](int kk) {
-        const int g = (int)blockIdx.x + (pair_mode ? kk >> 1 : kk) * (int)gridDim.x;
-        if constexpr (CLASS && C::BIG) {
-            // out of line in the 64-node instance (eleven call sites: 1 % through the instruction cache);
-            // the smaller instances, with a third of the time per item, lose 5 % to the calls
-            return class_item_of(g, kk & 1);
-        } else if constexpr (CLASS) {
-            if (g >= n_units) return n_items;
+        const int ku = pair_mode ? kk >> 1 : kk;
+        if constexpr (CLASS) {
             if (compact) {
-                const int sq = ups < 2 ? g : (int)__umulhi((uint32_t)g, a.ups_magic), u = g - sq * ups;
-                return (int)ctab[sq] * a.H_v + (pair_mode ? 2 * u + (kk & 1) : u);
+                if (ku >= K) return n_items;
+                const int unit = ctab[ku];  // sequence * ups + unit of the sequence
+                return pair_mode ? 2 * unit + (kk & 1) : unit;
             }
         }
+        const int g = (int)blockIdx.x + ku * (int)gridDim.x;
         return pair_mode ? 2 * g + (kk & 1) : g;
     };
 
@@ -313,8 +291,12 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     const uint32_t tmem_base = *tmem_slot;
     if (CLASS && compact) {
         // Every role would otherwise hand every unit of the other classes through the whole pipeline
-        // just to drop it (a third of the time of a ragged batch).  All threads: one sequence each per
-        // round, kept sequences numbered by warp ballots and a prefix over the warps' counts.
+        // just to drop it (a third of the time of a ragged batch).  First the sequences of the class, over
+        // the whole batch: all threads, one sequence each per round, kept sequences numbered by warp
+        // ballots and a prefix over the warps' counts (scratch: the first stage, idle until the roles
+        // start).  Then this CTA's units, numbers blockIdx.x, blockIdx.x + gridDim.x, ... of the kept
+        // sequences' units, into ctab: a role finds its item with one load.
+        uint16_t *seq = reinterpret_cast<uint16_t *>(smem);
         uint16_t *tab = reinterpret_cast<uint16_t *>(smem + C::OFF_CTAB);
         int *wcount = reinterpret_cast<int *>(smem + C::OFF_CTAB + C::CT_CAP * 2);
         int kept = 0;
@@ -331,22 +313,20 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (lane == 0) wcount[warp] = __popc(bal);
             __syncthreads();
             int before = 0, total = 0;
+#pragma unroll 1
             for (int w2 = 0; w2 < C::THREADS / 32; ++w2) {
                 const int c = wcount[w2];
                 before += w2 < warp ? c : 0, total += c;
             }
-            if (keep) tab[kept + before + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)b;
+            if (keep) seq[kept + before + __popc(bal & ((1u << lane) - 1u))] = (uint16_t)b;
             kept += total;
             __syncthreads();
         }
-        n_units = kept * ups;
-    }
-    if constexpr (CLASS && C::BIG) {
-        if (tid == 0) {
-            s_class_map.tab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
-            s_class_map.n_units = n_units;
-            s_class_map.n_items = n_items, s_class_map.ups = ups, s_class_map.H_v = a.H_v;
-            s_class_map.magic = a.ups_magic, s_class_map.pair = pair_mode, s_class_map.compact = compact;
+        const int n_units = kept * ups;  // (at most CT_CAP * 64 = 65536: a unit's number fits 16 bits)
+        K = n_units > (int)blockIdx.x ? (n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+        for (int ku = tid; ku < K; ku += C::THREADS) {
+            const int g = (int)blockIdx.x + ku * (int)gridDim.x, sq = g / ups;
+            tab[ku] = (uint16_t)((int)seq[sq] * ups + (g - sq * ups));
         }
         __syncthreads();
     }
@@ -1263,13 +1243,10 @@ cudaError_t launch_vt(const VerifyArgs &a, const PrevRound &pv, int T, cudaStrea
     const bool pairs = (a.H_v / a.H_qk) % 2 == 0;  // the kernel takes heads in pairs
     const long long units = pairs ? n_items / 2 : n_items;
     const int grid = (int)(units < sms ? units : sms);
-    VerifyArgs a2 = a;
-    const uint32_t ups = (uint32_t)(pairs ? a.H_v / 2 : a.H_v);
-    a2.ups_magic = ups < 2 ? 0u : (uint32_t)((0x100000000ull + ups - 1u) / ups);
     auto go = [&](auto kernel) {
         cudaError_t e2 = ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), C::SMEM_BYTES, dev);
         if (e2 != cudaSuccess) return e2;
-        return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a2, pv, (int)n_items, m.S0, m.Q,
+        return launch_dependent(kernel, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, stream, a, pv, (int)n_items, m.S0, m.Q,
                                 m.K, m.V);
     };
     if constexpr (FUSED) {

@@ -101,11 +101,6 @@ prepare_wide_kernel(int B, int T, int H_v, int max_nodes, const int32_t *__restr
 }
 
 __device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
-__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p)
-{
-    const uint2 x = *reinterpret_cast<const uint2 *>(p);
-    return make_float4(bf16lo(x.x), bf16hi(x.x), bf16lo(x.y), bf16hi(x.y));
-}
 
 template <typename TIn> struct WideSmem {
     alignas(16) TIn kf[WN][D];     // k rows of the sequence (this head's q/k head), as stored: bf16 rows
