@@ -484,9 +484,10 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
         const int item0 = item_of(s);
         const bool early = !C::S0_RING && !a.state_index && item0 < n_items && item0 != a.skip_item;
         if (early && lane == 0) {
-            ptx::mbar_expect_tx(&full[s], C::S0_BYTES);
-            ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, item0 * D, &full[s]);
-            ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, item0 * D, &full[s]);
+            uint64_t *bar0 = FUSED ? &s0_full[s] : &full[s];
+            ptx::mbar_expect_tx(bar0, C::S0_BYTES);
+            ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, item0 * D, bar0);
+            ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, item0 * D, bar0);
         }  // (the q / k rows as well, one load away, was tried: the step got 0.2 % slower, workload 3 1 %)
         // An item's meta block: node scalars, size and place, and the path lists of the node(s) a lane owns
         // (index and gate ratio e^{L_i - L_j} of the first 8 ancestors; only the ratios depend on the head).
@@ -548,31 +549,39 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const bool tile_issued = s0_issued;
             // the state tile serves verify, commit or both (64 nodes: it comes through the ring of its own)
             const bool need_tile = !C::S0_RING && (!p.bad || p.plen >= 0) && !tile_issued;
-            const uint32_t tx = (need_tile ? C::S0_BYTES : 0) + (p.bad ? 0 : C::QK_BYTES) + p.cnt * (D * 2 + D * 4);
-            if (lane == 0) {
-                if (tx != 0) {
-                    const int hq = p.h / group;
-                    if (need_tile) {
-                        ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.srow * D, &full[s]);
-                        ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.srow * D, &full[s]);
-                    }
-                    if (!p.bad) {
-                        ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
-                        ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
-                        ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
-                        ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
-                    }
-                }
+            // Fused mode: what the commit group waits for (state tile, the previous round's path rows, the
+            // path meta block) is announced on a barrier of its own, as soon as it has been issued: the
+            // group starts when THAT has landed, not when the last of the q / k rows has (the copies of a
+            // stage are accepted one after the other, ~200 cycles each).
+            uint64_t *cbar = FUSED ? &s0_full[s] : &full[s];
+            const uint32_t tx_c = (need_tile ? C::S0_BYTES : 0) + p.cnt * (D * 2 + D * 4);
+            const uint32_t tx_q = p.bad ? 0 : C::QK_BYTES;
+            const uint32_t tx = FUSED ? tx_q : tx_c + tx_q;
+            const int hq = p.h / group;
+            if (lane == 0 && need_tile) {
+                ptx::tma_load_2d(stage + C::OFF_S0, &tmS0, 0, p.srow * D, cbar);
+                ptx::tma_load_2d(stage + C::OFF_S0 + C::S0_HALF, &tmS0, 64, p.srow * D, cbar);
             }
             if constexpr (FUSED) {
                 __syncwarp();
                 if (lane < p.cnt) {  // the accepted path's k and U rows of the previous round
                     const __nv_bfloat16 *kp = static_cast<const __nv_bfloat16 *>(pv.k);
                     ptx::bulk_g2s(stage + C::OFF_KP + lane * D * 2,
-                                  kp + ((size_t)(p.plo + p.pj) * a.H_qk + p.h / group) * D, D * 2, &full[s]);
+                                  kp + ((size_t)(p.plo + p.pj) * a.H_qk + hq) * D, D * 2, cbar);
                     ptx::bulk_g2s(stage + C::OFF_UP + lane * D * 4, pv.U + ((size_t)(p.plo + p.pj) * a.H_v + p.h) * D,
-                                  D * 4, &full[s]);
+                                  D * 4, cbar);
                 }
+                __syncwarp();
+                if (lane == 0) {
+                    if (tx_c == 0) ptx::mbar_arrive(cbar);
+                    else ptx::mbar_arrive_expect_tx(cbar, tx_c);
+                }
+            }
+            if (lane == 0 && !p.bad) {
+                ptx::tma_load_2d(stage, &tmQ, hq * D, p.lo, &full[s]);
+                ptx::tma_load_2d(stage + C::QK_HALF, &tmQ, hq * D + 64, p.lo, &full[s]);
+                ptx::tma_load_2d(stage + NP * 128, &tmK, hq * D, p.lo, &full[s]);
+                ptx::tma_load_2d(stage + C::QK_HALF + NP * 128, &tmK, hq * D + 64, p.lo, &full[s]);
             }
             if constexpr (!C::META_RING) write_meta(p, mt);  // (while the data is on its way)
             __syncwarp();
@@ -611,7 +620,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             const int s = kk % C::STAGES;
             unsigned char *stage = smem + s * C::STAGE_BYTES;
             unsigned char *mt = meta_of(kk);
-            if (!ptx::mbar_wait(&full[s], (kk / C::STAGES) & 1)) {
+            if (!ptx::mbar_wait(&s0_full[s], (kk / C::STAGES) & 1)) {  // state tile, path rows, path meta
                 if (t == 0 && a.seq_status) atomicOr(&a.seq_status[item / a.H_v], TREEWY_SEQ_TIMEOUT);
                 break;
             }
@@ -747,6 +756,8 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             bool stored = false;
             if constexpr (FUSED) {
                 // the new state goes back to global memory while verification proceeds from this copy
+                // (issued in front of the MMAs: behind them, the wait for the store to have read the tile
+                // delays stage 1's completion signal, 2 % of the launch)
                 if (!gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
                     const int srow = meta_nlo(mt)[3];
                     ptx::tma_store_2d(&tmS0, 0, srow * D, stage + C::OFF_S0);
