@@ -755,10 +755,11 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             if (FUSED && !ptx::mbar_wait(&upd_done[s], (kk / C::STAGES) & 1)) break;  // tile carries the commit
             bool stored = false;
             if constexpr (FUSED) {
-                // the new state goes back to global memory while verification proceeds from this copy
-                // (issued in front of the MMAs: behind them, the wait for the store to have read the tile
-                // delays stage 1's completion signal, 2 % of the launch)
-                if (!gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
+                // the new state goes back to global memory while verification proceeds from this copy.  The
+                // Gram chain's warp issues the store (its chain is the shorter one, and idle for the second
+                // head of a pair), in front of its MMAs: behind them, the wait for the store to have read the
+                // tile delays stage 1's completion signal, 2 % of the launch.
+                if (gram_chain && lane == 0 && reinterpret_cast<const PathMeta *>(stage + C::OFF_PMETA)->plen >= 0) {
                     const int srow = meta_nlo(mt)[3];
                     ptx::tma_store_2d(&tmS0, 0, srow * D, stage + C::OFF_S0);
                     ptx::tma_store_2d(&tmS0, 64, srow * D, stage + C::OFF_S0 + C::S0_HALF);
