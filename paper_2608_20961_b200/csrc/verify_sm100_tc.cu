@@ -234,7 +234,9 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
     // their places in the batch; its own units are then listed in ctab (see the prologue below).  A batch of
     // more than CT_CAP sequences is walked whole.
     const int ups = pair_mode ? a.H_v >> 1 : a.H_v;  // units per sequence
-    const bool compact = CLASS && a.B <= C::CT_CAP && (a.B * ups + (int)gridDim.x - 1) / (int)gridDim.x <= C::CT_CAP;
+    // (a unit's number has to fit the table's 16 bits, and a CTA's units the table)
+    const bool compact = CLASS && a.B <= C::CT_CAP && a.B * ups <= 65536 &&
+                         (a.B * ups + (int)gridDim.x - 1) / (int)gridDim.x <= C::CT_CAP;
     int K = 0;  // compact: the CTA's units (set by the prologue)
     const uint16_t *ctab = reinterpret_cast<const uint16_t *>(smem + C::OFF_CTAB);
     auto item_of = [&](int kk) {
@@ -322,7 +324,7 @@ verify_sm100_tc_kernel(VerifyArgs a, PrevRound pv, int n_items, const __grid_con
             kept += total;
             __syncthreads();
         }
-        const int n_units = kept * ups;  // (at most CT_CAP * 64 = 65536: a unit's number fits 16 bits)
+        const int n_units = kept * ups;  // (at most 65536: a unit's number fits 16 bits)
         K = n_units > (int)blockIdx.x ? (n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
         for (int ku = tid; ku < K; ku += C::THREADS) {
             const int g = (int)blockIdx.x + ku * (int)gridDim.x, sq = g / ups;

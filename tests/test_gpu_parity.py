@@ -244,3 +244,23 @@ def test_mixed_size_batch_larger_than_the_class_table(oracle):
     assert not (gpu["U"] == gpu["canary"]).all(dim=-1).any()
     tree_ref, ref = pu.run_oracle(oracle, w)
     pu.assert_parity(w, gpu, tree_ref, ref)
+
+
+def test_mixed_size_batch_with_many_heads_per_sequence():
+    """More units than a class launch's 16-bit unit table can number (sequences x heads > 65536; here
+    520 x 128 unpaired heads, 2 GB of states): both class launches walk the whole batch instead.  Checked
+    against the SIMT kernel on the same inputs (every row written exactly where that kernel writes)."""
+    g = torch.Generator().manual_seed(78)
+    sizes = [1 + int(torch.randint(0, 2, (1,), generator=g)) for _ in range(520)]
+    for at, n in ((7, 40), (519, 64)):
+        sizes[at] = n
+    trees = [wl.random_parent_tree(g, n, 4) for n in sizes]
+    w = _custom(trees, H_v=128, H_qk=128, seed=13, accepted=[n - 1 for n in sizes])
+    fast = pu.run_gpu(w, torch.float32, max_nodes=64, want_s32=False)
+    slow = pu.run_gpu(w, torch.float32, max_nodes=64, want_s32=False, generic=True)
+    assert not fast["status"].any() and not slow["status"].any()
+    assert not (fast["U"] == fast["canary"]).all(dim=-1).any()
+    for name in ("O", "U"):
+        scale = float(slow[name].abs().max())
+        assert float((fast[name] - slow[name]).abs().max()) <= 5e-5 * scale, name
+    assert torch.equal(fast["S"], slow["S"]) or float((fast["S"].float() - slow["S"].float()).abs().max()) <= 2 ** -7 * float(slow["S"].float().abs().max())
